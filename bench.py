@@ -1,0 +1,349 @@
+#!/usr/bin/env python
+"""Benchmark of the attention-backward hot path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
+
+One step = one ``lt_attn_bwd`` call (delta preprocess, main tensor-core kernel, dQ finalise)
+on one seeded synthetic batch.  The metric is attention-backward TFLOP/s with causal FLOPs
+(5 * B * Hq * S^2 * D).  Rank 0 prints one JSON line.  With N > 1 (launched by torchrun, one
+process per GPU) every rank runs its own replica of the workload: the path has no exchange
+step, so the only collectives are the timing barrier and the max over ranks.
+
+``--impl reference`` times the CPU oracle, as it stands, on a bounded sample of the same
+workload on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+from pathlib import Path
+
+import torch
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+from paper_2606_10415_b200 import workloads  # noqa: E402
+
+METRIC = "attention-backward TFLOP/s (causal FLOPs)"
+UNIT = "TFLOP/s"
+NOMINAL_FP16_TFLOPS = 2250.0  # datasheet dense figure, context only
+FALLBACK_PEAK_TFLOPS = 1590.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default="llama2_7b", choices=sorted(workloads.CONFIGS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the timed oracle leg (debugging)")
+    return ap.parse_args()
+
+
+def describe(cfg) -> str:
+    return (f"{cfg.name}: B={cfg.B} Hq={cfg.Hq} Hkv={cfg.Hkv} S={cfg.S} D={cfg.D} "
+            f"{'causal' if cfg.causal else 'full'} fp16")
+
+
+def measured_peak():
+    path = ROOT / "MEASURED_PEAKS.json"
+    if path.exists():
+        d = json.loads(path.read_text())
+        return float(d["bf16_tflops"]), float(d.get("hbm_gbs", 0.0)), "measured"
+    return FALLBACK_PEAK_TFLOPS, 6650.0, "fallback"
+
+
+# ------------------------------------------------------------------ CPU oracle legs
+
+def oracle_sample(cfg, n_heads):
+    """The first kv groups of batch 0, enough to cover about `n_heads` query heads."""
+    G = cfg.Hq // cfg.Hkv
+    n_groups = max(1, min(cfg.Hkv, (n_heads + G - 1) // G))
+    sub = workloads.custom(1, n_groups * G, n_groups, cfg.S, cfg.D, cfg.causal, cfg.qkv_std, cfg.do_std, cfg.seed,
+                           name=cfg.name + "_sample")
+    Q, K, V, dO = workloads.make_inputs(cfg)
+    arrs = [Q[:1, :n_groups * G], K[:1, :n_groups], V[:1, :n_groups], dO[:1, :n_groups * G]]
+    return sub, [a.double().numpy() for a in arrs]
+
+
+def time_oracle(cfg, n_heads, steps, warmup):
+    import oracle
+    sub, arrs = oracle_sample(cfg, n_heads)
+    times = []
+    for it in range(warmup + steps):
+        t0 = time.perf_counter()
+        oracle.attn_bwd(*arrs, sub.causal, sub.scale)
+        dt = time.perf_counter() - t0
+        if it >= warmup:
+            times.append(dt)
+    return sub, times, oracle.num_threads()
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    threads = oracle.num_threads()
+    n_heads = max(1, min(cfg.Hq, threads))
+    # keep the whole run within a few minutes: shrink the sample if one head is slow
+    t0 = time.perf_counter()
+    sub1, arrs1 = oracle_sample(cfg, 1)
+    oracle.attn_bwd(*arrs1, sub1.causal, sub1.scale)
+    per_head = time.perf_counter() - t0
+    waves = max(1.0, n_heads / threads)
+    budget = 180.0
+    while n_heads > 1 and per_head * waves * (args.steps + args.warmup) > budget:
+        n_heads = max(1, n_heads // 2)
+        waves = max(1.0, n_heads / threads)
+    sub, times, threads = time_oracle(cfg, n_heads, args.steps, args.warmup)
+    total = sum(times)
+    value = sub.flops * len(times) / total / 1e12
+    sample = f"{sub.Hq} query heads ({sub.Hkv} kv groups) of batch 0, full S={cfg.S}, per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": describe(cfg), "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------ clocks
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_id: str):
+        self.proc = None
+        self.path = None
+        self.device_id = device_id
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.device_id}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "50"],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        clocks, maxes, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in Path(self.path).read_text().splitlines():
+            parts = [x.strip() for x in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                clocks.append(float(parts[0]))
+                maxes.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        os.unlink(self.path)
+        if clocks:
+            out.update(sm_mhz=statistics.median(clocks), sm_max_mhz=max(maxes), reasons=sorted(reasons),
+                       samples=len(clocks))
+        return out
+
+
+# ------------------------------------------------------------------ GPU arm
+
+def run_ours(args, cfg):
+    from paper_2606_10415_b200 import binding as lt
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the attention path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    Qh, Kh, Vh, dOh = workloads.make_inputs(cfg)
+    Q, K, V, dO = (t.cuda() for t in (Qh, Kh, Vh, dOh))
+    O = torch.empty_like(Q)
+    LSE = torch.empty(Q.shape[:3], dtype=torch.float32, device="cuda")
+    dQ, dK, dV = torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V)
+    dims = (cfg.B, cfg.Hq, cfg.Hkv, cfg.S, cfg.D)
+    ws = lt.alloc_workspace(lt.lt_attn_bwd_workspace_bytes(*dims))
+    fws = lt.alloc_workspace(lt.lt_attn_fwd_workspace_bytes(*dims))
+    stream = torch.cuda.current_stream()
+
+    # forward (feeds the backward; timed separately, not part of the metric)
+    lt.lt_attn_fwd(Q, K, V, O, LSE, cfg.causal, cfg.scale, fws)
+    if lt.lt_attn_check_status(fws) != lt.LT_OK:
+        raise SystemExit("forward kernel reported: " + lt.last_cuda_error())
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    fwd_iters = max(3, min(10, args.steps))
+    f0.record()
+    for _ in range(fwd_iters):
+        lt.lt_attn_fwd(Q, K, V, O, LSE, cfg.causal, cfg.scale, fws)
+    f1.record()
+    torch.cuda.synchronize()
+    fwd_ms = f0.elapsed_time(f1) / fwd_iters
+    fwd_flops = cfg.flops * 2.0 / 5.0
+
+    def step(ev0=None, ev1=None):
+        lt.lt_attn_bwd_profiled(Q, K, V, O, dO, LSE, dQ, dK, dV, cfg.causal, cfg.scale, ws, stream, ev0, ev1)
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    torch.cuda.synchronize()
+    if lt.lt_attn_check_status(ws) != lt.LT_OK:
+        raise SystemExit("backward kernel reported: " + lt.last_cuda_error())
+
+    kernel_events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                     for _ in range(args.steps)]
+    for a, b in kernel_events:  # materialise the event handles
+        a.record()
+        b.record()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(torch.cuda.current_device()).uuid))
+    barrier()
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.15)
+    barrier()
+    # keep the GPU busy long enough for nvidia-smi to sample clocks under this load
+    busy_until = time.perf_counter() + 0.6
+    while time.perf_counter() < busy_until:
+        step()
+    barrier()
+    t0.record()
+    for a, b in kernel_events:
+        step(a, b)
+    t1.record()
+    barrier()
+    total_ms = t0.elapsed_time(t1)
+    busy_until = time.perf_counter() + 0.3
+    while time.perf_counter() < busy_until:
+        step()
+    torch.cuda.synchronize()
+    clocks = sampler.stop() if rank == 0 else None
+    if lt.lt_attn_check_status(ws) != lt.LT_OK:
+        raise SystemExit("backward kernel reported: " + lt.last_cuda_error())
+    main_ms = [a.elapsed_time(b) for a, b in kernel_events]
+
+    # end to end through the host-buffer entry point: pinned host inputs, host outputs
+    pin = [t.pin_memory() for t in (Qh, Kh, Vh, dOh)]
+    hO = torch.empty_like(Qh).pin_memory()
+    hL = torch.empty(Qh.shape[:3], dtype=torch.float32).pin_memory()
+    hdQ, hdK, hdV = (torch.empty_like(t).pin_memory() for t in (Qh, Kh, Vh))
+    arena = lt.alloc_workspace(lt.lt_attn_host_arena_bytes(*dims))
+
+    def e2e_step():
+        lt.lt_attn_fwd_bwd_host(*pin, None, None, hdQ, hdK, hdV, cfg.causal, cfg.scale, arena, stream)
+
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2e_iters = max(3, min(10, args.steps))
+    e0.record()
+    for _ in range(e2e_iters):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_iters
+    h2d = sum(t.numel() * t.element_size() for t in pin)
+    d2h = sum(t.numel() * t.element_size() for t in (hdQ, hdK, hdV))
+    del hO, hL
+
+    if dist is not None:
+        tt = torch.tensor([total_ms, e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms = tt.tolist()
+
+    if rank == 0:
+        ms_per_step = total_ms / args.steps
+        value = world * cfg.flops / (ms_per_step * 1e-3) / 1e12
+        peak, _hbm, peak_kind = measured_peak()
+        main_avg_ms = sum(main_ms) / len(main_ms)
+        achieved = cfg.flops / (main_avg_ms * 1e-3) / 1e12
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f16", "data": "synthetic",
+            "config": {"workload": describe(cfg),
+                       "l2": "inputs+workspace per step exceed the 126 MB L2 (no explicit flush)"
+                       if _step_bytes(cfg) > 126e6 else "working set fits L2",
+                       "multi_gpu": "replicas only" if world > 1 else "single"},
+            "pct_of_measured_peak": 100.0 * value / world / peak,
+            "pct_of_nominal_fp16_peak": 100.0 * value / world / NOMINAL_FP16_TFLOPS,
+            "peak_source": peak_kind,
+            "clocks": clocks,
+            "e2e": {"value": world * cfg.flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
+                    "includes": "H2D copies, lt_attn_fwd, lt_attn_bwd, D2H copies"},
+            "gpu_launches": args.steps * lt.lt_attn_bwd_num_launches(),
+            "roofline": {"bound": "tensor", "kernel": "bwd_main_kernel", "achieved": achieved, "peak": peak,
+                         "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                         "peak_source": peak_kind + " bf16 burst", "avg_launch_ms": main_avg_ms,
+                         "best_launch_ms": min(main_ms)},
+            "fwd": {"value": fwd_flops / (fwd_ms * 1e-3) / 1e12, "unit": UNIT, "ms": fwd_ms},
+        }
+        if not args.no_cpu_baseline and world == 1:
+            import oracle
+            n_heads = max(1, min(cfg.Hq, 2 * oracle.num_threads()))
+            sub, times, threads = time_oracle(cfg, n_heads, 1, 0)
+            line["cpu_baseline"] = {
+                "value": sub.flops / times[0] / 1e12, "unit": UNIT, "cores": threads, "kind": "oracle",
+                "sample": f"{sub.Hq} query heads ({sub.Hkv} kv groups) of batch 0, full S={cfg.S}, one pass",
+                "seconds": times[0]}
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def _step_bytes(cfg) -> float:
+    nq = cfg.B * cfg.Hq * cfg.S * cfg.D
+    nk = cfg.B * cfg.Hkv * cfg.S * cfg.D
+    return 2.0 * (4 * nq + 4 * nk) + 4.0 * nq
+
+
+def main():
+    args = parse_args()
+    cfg = workloads.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,136 @@
+/*
+ * lt_attn.h -- C ABI of the B200 (sm_100a) FP16 attention forward / backward library.
+ *
+ * The operation is the Attention Backward of a dense decoder layer as the paper's
+ * execution backend states it (Section 4.1, "Memory-resident Attention Backward",
+ * Algorithm 1):  GP = GO V^T,  GS = SoftmaxBackward(P, GP),  GV = P^T GO,
+ * GQ = GS K,  GK = GS^T Q, with the probability tile P as forward state.  Here P is
+ * not stored by the forward: it is rebuilt tile by tile from the row log-sum-exp.
+ *
+ * Conventions shared by every entry point
+ *   - Tensors are contiguous [B, H, S, D] with D innermost.  Q, O, dO, dQ have H = Hq;
+ *     K, V, dK, dV have H = Hkv.  LSE is fp32 [B, Hq, S].  fp16 is IEEE binary16.
+ *   - Grouped-query attention: query head h reads key/value head h / (Hq / Hkv);
+ *     dK and dV are summed over the Hq / Hkv query heads of a group.
+ *   - scores = scale * Q K^T; causal != 0 hides key j from query i when j > i.
+ *     LSE_i = ln sum_j exp(scores_ij) over visible keys (natural logarithm).
+ *   - Supported shapes: D in {64, 128}, S a positive multiple of 128, Hq % Hkv == 0.
+ *     Anything else returns LT_ERR_UNSUPPORTED and launches nothing.
+ *   - Unless a function says otherwise pointers are DEVICE pointers, 16-byte aligned,
+ *     owned by the caller, and must stay valid until the stream reaches the end of the
+ *     call's work.  Inputs are never written.  Outputs are fully overwritten.
+ *   - Calls only enqueue work on `stream` and return; they do not synchronise and
+ *     allocate no device memory.  Two calls may overlap on the GPU only if they use
+ *     different workspaces.
+ *   - Return value: LT_OK or an lt_status error.  Errors found on the host launch
+ *     nothing.  A device-side wait that gave up (a bounded spin on a barrier ran out)
+ *     is recorded in the workspace and read back with lt_attn_check_status.
+ *   - The library targets the current CUDA device, which must be compute capability 10.x.
+ */
+#ifndef LT_ATTN_H_
+#define LT_ATTN_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum lt_status {
+    LT_OK = 0,
+    LT_ERR_INVALID_ARG = 1,    /* NULL pointer, non-positive size, Hq % Hkv != 0, non-finite scale */
+    LT_ERR_UNSUPPORTED = 2,    /* shape, alignment or device outside the supported set */
+    LT_ERR_WORKSPACE = 3,      /* workspace NULL, misaligned (256 B) or too small */
+    LT_ERR_CUDA = 4,           /* a CUDA runtime/driver call failed; see lt_last_cuda_error */
+    LT_ERR_DEVICE_TIMEOUT = 5  /* a bounded device-side wait expired (lt_attn_check_status only) */
+} lt_status;
+
+/* ABI-compatible with cudaStream_t. */
+typedef struct CUstream_st *lt_stream_t;
+/* ABI-compatible with cudaEvent_t. */
+typedef struct CUevent_st *lt_event_t;
+/* fp16 storage type (bit pattern of an IEEE binary16). */
+typedef unsigned short lt_half;
+
+/* Bytes of caller-owned device workspace the calls below need; 0 means the shape is
+ * not supported.  The workspace must be 256-byte aligned.  Layout (backward): a
+ * 256-byte status block, delta fp32 [B,Hq,S], an fp32 dQ accumulator [B,Hq,S,D]. */
+size_t lt_attn_fwd_workspace_bytes(int B, int Hq, int Hkv, int S, int D);
+size_t lt_attn_bwd_workspace_bytes(int B, int Hq, int Hkv, int S, int D);
+
+/* Forward: O = softmax(scale Q K^T [+ causal mask]) V, and the row log-sum-exp.
+ * The forward step that produces the state Algorithm 1 requires (the paper saves P;
+ * this library saves LSE, from which the backward recomputes P).
+ *   in : Q [B,Hq,S,D], K, V [B,Hkv,S,D]  fp16
+ *   out: O [B,Hq,S,D] fp16, LSE [B,Hq,S] fp32 */
+int lt_attn_fwd(const lt_half *Q, const lt_half *K, const lt_half *V,
+                lt_half *O, float *LSE,
+                int B, int Hq, int Hkv, int S, int D, int causal, float scale,
+                void *workspace, size_t workspace_bytes, lt_stream_t stream);
+
+/* Backward (Algorithm 1): dQ, dK, dV of L with dO = dL/dO.
+ *   delta = rowsum(dO * O)                          preprocess kernel
+ *   P     = exp(scale Q K^T - LSE)  (masked)        recomputed per tile
+ *   dV   += P^T dO;  dP = dO V^T;  dS = P * (dP - delta)
+ *   dQ   += scale dS K;  dK += scale dS^T Q
+ *   in : Q, O, dO [B,Hq,S,D] fp16; K, V [B,Hkv,S,D] fp16; LSE [B,Hq,S] fp32
+ *   out: dQ [B,Hq,S,D], dK, dV [B,Hkv,S,D] fp16 (overwritten, not accumulated into)
+ * dQ is accumulated in fp32 in the workspace with atomic adds, so its last bits may
+ * differ between runs; dK and dV are bitwise reproducible. */
+int lt_attn_bwd(const lt_half *Q, const lt_half *K, const lt_half *V,
+                const lt_half *O, const lt_half *dO, const float *LSE,
+                lt_half *dQ, lt_half *dK, lt_half *dV,
+                int B, int Hq, int Hkv, int S, int D, int causal, float scale,
+                void *workspace, size_t workspace_bytes, lt_stream_t stream);
+
+/* lt_attn_bwd with two optional CUDA events recorded on `stream` immediately before and
+ * after the main (tensor-core) kernel, so a benchmark can time that kernel inside a
+ * normal call.  Either event may be NULL.  Everything else is as for lt_attn_bwd. */
+int lt_attn_bwd_profiled(const lt_half *Q, const lt_half *K, const lt_half *V,
+                         const lt_half *O, const lt_half *dO, const float *LSE,
+                         lt_half *dQ, lt_half *dK, lt_half *dV,
+                         int B, int Hq, int Hkv, int S, int D, int causal, float scale,
+                         void *workspace, size_t workspace_bytes, lt_stream_t stream,
+                         lt_event_t main_begin, lt_event_t main_end);
+
+/* Same computation as lt_attn_fwd followed by lt_attn_bwd, but every tensor pointer is
+ * a HOST pointer (pinned memory makes the copies asynchronous).  `arena` is a caller-
+ * owned DEVICE buffer of at least lt_attn_host_arena_bytes() bytes, 256-byte aligned,
+ * that holds the device copies and the workspace.  The call enqueues the host-to-device
+ * copies of Q, K, V, dO, the two kernels' work and the device-to-host copies of
+ * O, LSE, dQ, dK, dV on `stream`; the host outputs are valid once the stream is
+ * synchronised.  O and LSE may be NULL if the caller does not want them back. */
+size_t lt_attn_host_arena_bytes(int B, int Hq, int Hkv, int S, int D);
+int lt_attn_fwd_bwd_host(const lt_half *Q, const lt_half *K, const lt_half *V, const lt_half *dO,
+                         lt_half *O, float *LSE, lt_half *dQ, lt_half *dK, lt_half *dV,
+                         int B, int Hq, int Hkv, int S, int D, int causal, float scale,
+                         void *arena, size_t arena_bytes, lt_stream_t stream);
+
+/* Synchronises `stream`, reads the status block of `workspace` and returns LT_OK,
+ * LT_ERR_DEVICE_TIMEOUT (a kernel abandoned a wait; outputs are invalid) or LT_ERR_CUDA. */
+int lt_attn_check_status(const void *workspace, lt_stream_t stream);
+
+/* Static strings; never NULL. */
+const char *lt_status_string(int status);
+const char *lt_last_cuda_error(void);
+
+/* Number of kernels one call enqueues (for launch accounting by benchmarks). */
+int lt_attn_bwd_num_launches(void);
+int lt_attn_fwd_num_launches(void);
+
+/* Bring-up check of one tensor-core tile product, used by the tests to pin the
+ * shared-memory / tensor-memory operand conventions the attention kernels rely on
+ * (no counterpart in the paper; its analogue is the GEMM primitive inside Attention BP,
+ * Section 4.1).  Computes C[128,128] (fp32, row-major, device) from fp16 device
+ * matrices, each 128 x 128 row-major:
+ *   mode 0: C = A  B^T   (A rows = M, B rows = N; both contraction-contiguous)
+ *   mode 1: C = A  B     (B rows = contraction index)
+ *   mode 2: C = A^T B    (A and B rows = contraction index)
+ *   mode 3: C = A  B     (A staged through tensor memory instead of shared memory) */
+int lt_dbg_tile_gemm(const lt_half *A, const lt_half *B, float *C, int mode,
+                     void *workspace, size_t workspace_bytes, lt_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LT_ATTN_H_ */

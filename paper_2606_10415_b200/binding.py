@@ -1,0 +1,198 @@
+"""ctypes binding of the C-ABI library (``include/lt_attn.h``), same names as the C entry points.
+
+Argument marshalling only: torch is used to hold device memory and streams; every
+step of the attention path runs inside the library's kernels.  There is no CPU
+fallback -- if ``liblt_attn.so`` is missing the import fails.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import torch
+
+_PKG = Path(__file__).resolve().parent
+LIB_PATH = _PKG / "liblt_attn.so"
+
+LT_OK = 0
+LT_ERR_INVALID_ARG = 1
+LT_ERR_UNSUPPORTED = 2
+LT_ERR_WORKSPACE = 3
+LT_ERR_CUDA = 4
+LT_ERR_DEVICE_TIMEOUT = 5
+
+EXPORTS = (
+    "lt_attn_fwd_workspace_bytes", "lt_attn_bwd_workspace_bytes", "lt_attn_fwd", "lt_attn_bwd",
+    "lt_attn_bwd_profiled",
+    "lt_attn_host_arena_bytes", "lt_attn_fwd_bwd_host", "lt_attn_check_status", "lt_status_string",
+    "lt_last_cuda_error", "lt_attn_bwd_num_launches", "lt_attn_fwd_num_launches", "lt_dbg_tile_gemm",
+)
+
+
+class LtError(RuntimeError):
+    def __init__(self, fn: str, status: int):
+        self.status = status
+        super().__init__(f"{fn} failed: {status_string(status)} (status {status}); last CUDA error: "
+                         f"{last_cuda_error()}")
+
+
+def _load() -> ctypes.CDLL:
+    if not LIB_PATH.exists():
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2606_10415_b200.build` "
+            "(there is no fallback path)")
+    lib = ctypes.CDLL(str(LIB_PATH))
+    vp, i, f, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    lib.lt_attn_fwd_workspace_bytes.argtypes = [i] * 5
+    lib.lt_attn_fwd_workspace_bytes.restype = sz
+    lib.lt_attn_bwd_workspace_bytes.argtypes = [i] * 5
+    lib.lt_attn_bwd_workspace_bytes.restype = sz
+    lib.lt_attn_host_arena_bytes.argtypes = [i] * 5
+    lib.lt_attn_host_arena_bytes.restype = sz
+    lib.lt_attn_fwd.argtypes = [vp] * 5 + [i] * 6 + [f, vp, sz, vp]
+    lib.lt_attn_fwd.restype = i
+    lib.lt_attn_bwd.argtypes = [vp] * 9 + [i] * 6 + [f, vp, sz, vp]
+    lib.lt_attn_bwd.restype = i
+    lib.lt_attn_bwd_profiled.argtypes = [vp] * 9 + [i] * 6 + [f, vp, sz, vp, vp, vp]
+    lib.lt_attn_bwd_profiled.restype = i
+    lib.lt_attn_fwd_bwd_host.argtypes = [vp] * 9 + [i] * 6 + [f, vp, sz, vp]
+    lib.lt_attn_fwd_bwd_host.restype = i
+    lib.lt_attn_check_status.argtypes = [vp, vp]
+    lib.lt_attn_check_status.restype = i
+    lib.lt_status_string.argtypes = [i]
+    lib.lt_status_string.restype = ctypes.c_char_p
+    lib.lt_last_cuda_error.argtypes = []
+    lib.lt_last_cuda_error.restype = ctypes.c_char_p
+    lib.lt_attn_bwd_num_launches.restype = i
+    lib.lt_attn_fwd_num_launches.restype = i
+    lib.lt_dbg_tile_gemm.argtypes = [vp, vp, vp, i, vp, sz, vp]
+    lib.lt_dbg_tile_gemm.restype = i
+    return lib
+
+
+_lib = _load()
+
+
+def status_string(status: int) -> str:
+    return _lib.lt_status_string(int(status)).decode()
+
+
+def last_cuda_error() -> str:
+    return _lib.lt_last_cuda_error().decode()
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def _ptr(t) -> int:
+    return 0 if t is None else int(t.data_ptr())
+
+
+def _dims(Q: torch.Tensor, K: torch.Tensor):
+    B, Hq, S, D = Q.shape
+    return int(B), int(Hq), int(K.shape[1]), int(S), int(D)
+
+
+def _check_layout(*tensors):
+    for t in tensors:
+        if t is not None and not t.is_contiguous():
+            raise ValueError("tensors must be contiguous [B, H, S, D]")
+
+
+def lt_attn_fwd_workspace_bytes(B, Hq, Hkv, S, D) -> int:
+    return int(_lib.lt_attn_fwd_workspace_bytes(B, Hq, Hkv, S, D))
+
+
+def lt_attn_bwd_workspace_bytes(B, Hq, Hkv, S, D) -> int:
+    return int(_lib.lt_attn_bwd_workspace_bytes(B, Hq, Hkv, S, D))
+
+
+def lt_attn_host_arena_bytes(B, Hq, Hkv, S, D) -> int:
+    return int(_lib.lt_attn_host_arena_bytes(B, Hq, Hkv, S, D))
+
+
+def lt_attn_bwd_num_launches() -> int:
+    return int(_lib.lt_attn_bwd_num_launches())
+
+
+def lt_attn_fwd_num_launches() -> int:
+    return int(_lib.lt_attn_fwd_num_launches())
+
+
+def lt_attn_fwd_raw(*args) -> int:
+    """Direct call with integer pointers; returns the status code (for boundary tests)."""
+    return int(_lib.lt_attn_fwd(*args))
+
+
+def lt_attn_bwd_raw(*args) -> int:
+    return int(_lib.lt_attn_bwd(*args))
+
+
+def lt_attn_fwd(Q, K, V, O, LSE, causal, scale, workspace, stream=None) -> None:
+    """O (fp16) and LSE (fp32) from Q, K, V; device tensors; asynchronous on ``stream``."""
+    _check_layout(Q, K, V, O, LSE)
+    B, Hq, Hkv, S, D = _dims(Q, K)
+    rc = _lib.lt_attn_fwd(_ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(LSE), B, Hq, Hkv, S, D, int(bool(causal)),
+                          float(scale), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                          _stream_ptr(stream))
+    if rc != LT_OK:
+        raise LtError("lt_attn_fwd", rc)
+
+
+def lt_attn_bwd(Q, K, V, O, dO, LSE, dQ, dK, dV, causal, scale, workspace, stream=None) -> None:
+    """dQ, dK, dV (fp16) from Q, K, V, O, dO, LSE; device tensors; asynchronous on ``stream``."""
+    _check_layout(Q, K, V, O, dO, LSE, dQ, dK, dV)
+    B, Hq, Hkv, S, D = _dims(Q, K)
+    rc = _lib.lt_attn_bwd(_ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(dO), _ptr(LSE), _ptr(dQ), _ptr(dK), _ptr(dV),
+                          B, Hq, Hkv, S, D, int(bool(causal)), float(scale), _ptr(workspace),
+                          workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    if rc != LT_OK:
+        raise LtError("lt_attn_bwd", rc)
+
+
+def lt_attn_bwd_profiled(Q, K, V, O, dO, LSE, dQ, dK, dV, causal, scale, workspace, stream=None,
+                         main_begin=None, main_end=None) -> None:
+    """lt_attn_bwd with torch CUDA events recorded around the main kernel (events created with
+    ``enable_timing=True`` and recorded once beforehand so that their handles exist)."""
+    _check_layout(Q, K, V, O, dO, LSE, dQ, dK, dV)
+    B, Hq, Hkv, S, D = _dims(Q, K)
+    e0 = 0 if main_begin is None else int(main_begin.cuda_event)
+    e1 = 0 if main_end is None else int(main_end.cuda_event)
+    rc = _lib.lt_attn_bwd_profiled(_ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(dO), _ptr(LSE), _ptr(dQ), _ptr(dK),
+                                   _ptr(dV), B, Hq, Hkv, S, D, int(bool(causal)), float(scale), _ptr(workspace),
+                                   workspace.numel() * workspace.element_size(), _stream_ptr(stream), e0, e1)
+    if rc != LT_OK:
+        raise LtError("lt_attn_bwd_profiled", rc)
+
+
+def lt_attn_fwd_bwd_host(Q, K, V, dO, O, LSE, dQ, dK, dV, causal, scale, arena, stream=None) -> None:
+    """Host tensors in and out (pinned for asynchronous copies); ``arena`` is a device buffer."""
+    _check_layout(Q, K, V, dO, O, LSE, dQ, dK, dV)
+    for t in (Q, K, V, dO, O, LSE, dQ, dK, dV):
+        if t is not None and t.is_cuda:
+            raise ValueError("lt_attn_fwd_bwd_host takes host tensors")
+    B, Hq, Hkv, S, D = _dims(Q, K)
+    rc = _lib.lt_attn_fwd_bwd_host(_ptr(Q), _ptr(K), _ptr(V), _ptr(dO), _ptr(O), _ptr(LSE), _ptr(dQ), _ptr(dK),
+                                   _ptr(dV), B, Hq, Hkv, S, D, int(bool(causal)), float(scale), _ptr(arena),
+                                   arena.numel() * arena.element_size(), _stream_ptr(stream))
+    if rc != LT_OK:
+        raise LtError("lt_attn_fwd_bwd_host", rc)
+
+
+def lt_attn_check_status(workspace, stream=None) -> int:
+    return int(_lib.lt_attn_check_status(_ptr(workspace), _stream_ptr(stream)))
+
+
+def lt_dbg_tile_gemm(A, B, C, mode, workspace, stream=None) -> None:
+    rc = _lib.lt_dbg_tile_gemm(_ptr(A), _ptr(B), _ptr(C), int(mode), _ptr(workspace),
+                               workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    if rc != LT_OK:
+        raise LtError("lt_dbg_tile_gemm", rc)
+
+
+def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:
+    """A 256-byte aligned device byte buffer (torch's allocator aligns to 512 bytes)."""
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)

@@ -1,0 +1,141 @@
+// Bring-up check of one 128x128x128 tensor-core tile product in each operand
+// arrangement the attention kernels use (see lt_dbg_tile_gemm in lt_attn.h).
+#include "lt_common.cuh"
+#include "lt_host.h"
+
+namespace lt {
+
+constexpr int kTile = 128;
+constexpr int kBoxBytes = 128 * 128;  // one swizzled tile: 128 rows x 64 fp16
+
+struct __align__(1024) DbgSmem {
+    uint8_t a[2 * kBoxBytes];
+    uint8_t b[2 * kBoxBytes];
+    uint64_t bar_load;
+    uint64_t bar_mma;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+__global__ void __launch_bounds__(128, 1)
+dbg_tile_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                     const __half *__restrict__ a_gmem, float *__restrict__ c_gmem, int mode,
+                     unsigned int *status) {
+    extern __shared__ uint8_t smem_raw[];
+    DbgSmem &sm = *reinterpret_cast<DbgSmem *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    constexpr uint32_t kTmemCols = 256;  // accumulator: columns 0..127, A operand: 128..191
+
+    if (tid == 0) {
+        sm.abort_flag = 0;
+        mbar_init(&sm.bar_load, 1);
+        mbar_init(&sm.bar_mma, 1);
+        mbar_fence_init();
+        tma_prefetch_desc(&map_a);
+        tma_prefetch_desc(&map_b);
+    }
+    if (warp == 0) {
+        tmem_alloc(&sm.tmem_base, kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = sm.tmem_base;
+    const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
+
+    if (tid == 0) {
+        mbar_arrive_expect_tx(&sm.bar_load, 4 * kBoxBytes);
+        tma_load_2d(sm.a, &map_a, &sm.bar_load, 0, 0);
+        tma_load_2d(sm.a + kBoxBytes, &map_a, &sm.bar_load, 64, 0);
+        tma_load_2d(sm.b, &map_b, &sm.bar_load, 0, 0);
+        tma_load_2d(sm.b + kBoxBytes, &map_b, &sm.bar_load, 64, 0);
+    }
+    if (mode == 3) {
+        // thread t owns row t of A: pack pairs of fp16 into 64 tensor-memory columns
+        const uint4 *row = reinterpret_cast<const uint4 *>(a_gmem + static_cast<size_t>(tid) * kTile);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            uint32_t r[16];
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                uint4 x = row[c * 4 + v];
+                r[4 * v + 0] = x.x; r[4 * v + 1] = x.y; r[4 * v + 2] = x.z; r[4 * v + 3] = x.w;
+            }
+            tmem_st16(tmem + lane_base + 128 + c * 16, r);
+        }
+        tmem_wait_st();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+
+    bool ok = mbar_wait(&sm.bar_load, 0, &sm.abort_flag, status, 101);
+    if (ok && tid == 0) {
+        tc_fence_after_sync();
+        const uint32_t a0 = smem_u32(sm.a), b0 = smem_u32(sm.b);
+#pragma unroll 1
+        for (int kk = 0; kk < 8; ++kk) {
+            const uint32_t koff = (kk >> 2) * kBoxBytes + (kk & 3) * 32;  // contraction-contiguous operand
+            const uint32_t roff = kk * 16 * 128;                          // contraction index = row
+            const uint32_t acc = kk > 0;
+            if (mode == 0) {
+                umma_ss(tmem, desc_kmajor(a0 + koff), desc_kmajor(b0 + koff), make_idesc(128, 128, false, false), acc);
+            } else if (mode == 1) {
+                umma_ss(tmem, desc_kmajor(a0 + koff), desc_mnmajor(b0 + roff, kBoxBytes),
+                        make_idesc(128, 128, false, true), acc);
+            } else if (mode == 2) {
+                umma_ss(tmem, desc_mnmajor(a0 + roff, kBoxBytes), desc_mnmajor(b0 + roff, kBoxBytes),
+                        make_idesc(128, 128, true, true), acc);
+            } else {
+                umma_ts(tmem, tmem + 128 + kk * 8, desc_mnmajor(b0 + roff, kBoxBytes),
+                        make_idesc(128, 128, false, true), acc);
+            }
+        }
+        umma_commit(&sm.bar_mma);
+    }
+    ok = ok && mbar_wait(&sm.bar_mma, 0, &sm.abort_flag, status, 102);
+    tc_fence_after_sync();
+    if (ok) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            uint32_t r[32];
+            tmem_ld32(tmem + lane_base + c * 32, r);
+            tmem_wait_ld();
+            float4 *dst = reinterpret_cast<float4 *>(c_gmem + static_cast<size_t>(tid) * kTile + c * 32);
+#pragma unroll
+            for (int v = 0; v < 8; ++v)
+                dst[v] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                     __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+}
+
+}  // namespace lt
+
+extern "C" int lt_dbg_tile_gemm(const lt_half *A, const lt_half *B, float *C, int mode, void *workspace,
+                                size_t workspace_bytes, lt_stream_t stream) {
+    using namespace lt;
+    if (!A || !B || !C || mode < 0 || mode > 3) return LT_ERR_INVALID_ARG;
+    if (!aligned16(A) || !aligned16(B) || !aligned16(C)) return LT_ERR_UNSUPPORTED;
+    if (!workspace || !aligned256(workspace) || workspace_bytes < static_cast<size_t>(kStatusBytes))
+        return LT_ERR_WORKSPACE;
+    int rc = check_device();
+    if (rc != LT_OK) return rc;
+    CUtensorMap ma, mb;
+    if ((rc = make_tile_map(&ma, A, 128, 128, 128)) != LT_OK) return rc;
+    if ((rc = make_tile_map(&mb, B, 128, 128, 128)) != LT_OK) return rc;
+    cudaError_t e = cudaMemsetAsync(workspace, 0, kStatusBytes, stream);
+    if (e != cudaSuccess) return record_cuda_error("cudaMemsetAsync", e);
+    const size_t smem = sizeof(DbgSmem) + 1024;
+    e = cudaFuncSetAttribute(dbg_tile_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return record_cuda_error("cudaFuncSetAttribute", e);
+    dbg_tile_gemm_kernel<<<1, 128, smem, stream>>>(ma, mb, reinterpret_cast<const __half *>(A), C, mode,
+                                                   reinterpret_cast<unsigned int *>(workspace));
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return record_cuda_error("dbg_tile_gemm_kernel launch", e);
+    return LT_OK;
+}

@@ -1,0 +1,33 @@
+// Host-side helpers shared by the entry points: argument checks, the TMA tensor-map
+// encoder (fetched from the driver at run time so the library links without libcuda),
+// and the last-error string.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/lt_attn.h"
+
+namespace lt {
+
+void set_last_error(const char *what, const char *detail);
+int record_cuda_error(const char *what, cudaError_t err);
+
+// LT_OK, or the reason the current device cannot run the kernels.
+int check_device();
+
+// Validates the common (B, Hq, Hkv, S, D, scale) arguments.
+int check_shape(int B, int Hq, int Hkv, int S, int D, float scale);
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool aligned256(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
+inline size_t round256(size_t n) { return (n + 255u) & ~static_cast<size_t>(255u); }
+
+// fp16 matrix [rows, cols] row-major viewed as a 2-D tensor; tiles of box_rows x 64
+// columns are fetched with the 128-byte swizzle.  Returns LT_OK or LT_ERR_CUDA.
+int make_tile_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+
+}  // namespace lt

@@ -1,0 +1,229 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the fp64 CPU oracle
+on the same seeded inputs.  Tolerances (per gradient tensor, as the target states):
+relative Frobenius error <= 5e-3 and max abs error <= 2e-2.  Forward (not specified by
+the target): O relative Frobenius <= 2e-3, LSE max abs <= 1e-3."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2606_10415_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+
+REL_FRO_TOL = 5e-3
+MAX_ABS_TOL = 2e-2
+FWD_O_REL_FRO_TOL = 2e-3
+FWD_LSE_ABS_TOL = 1e-3
+
+
+@pytest.fixture(scope="module")
+def lt():
+    from paper_2606_10415_b200 import binding
+    return binding
+
+
+def rel_fro(a, ref):
+    a = np.asarray(a, dtype=np.float64)
+    return float(np.linalg.norm(a - ref) / max(np.linalg.norm(ref), 1e-300))
+
+
+def max_abs(a, ref):
+    return float(np.abs(np.asarray(a, dtype=np.float64) - ref).max())
+
+
+def run_fwd(lt, Q, K, V, cfg):
+    Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+    O = torch.empty_like(Qd)
+    LSE = torch.empty(Q.shape[:3], dtype=torch.float32, device="cuda")
+    ws = lt.alloc_workspace(lt.lt_attn_fwd_workspace_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.S, cfg.D))
+    lt.lt_attn_fwd(Qd, Kd, Vd, O, LSE, cfg.causal, cfg.scale, ws)
+    assert lt.lt_attn_check_status(ws) == lt.LT_OK, lt.last_cuda_error()
+    return O, LSE
+
+
+def run_bwd(lt, Q, K, V, O, dO, LSE, cfg):
+    Qd, Kd, Vd, Od, dOd, Ld = (t.cuda() for t in (Q, K, V, O, dO, LSE))
+    dQ, dK, dV = torch.empty_like(Qd), torch.empty_like(Kd), torch.empty_like(Vd)
+    # poison the outputs: the call must overwrite every element
+    for t in (dQ, dK, dV):
+        t.fill_(float("nan"))
+    ws = lt.alloc_workspace(lt.lt_attn_bwd_workspace_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.S, cfg.D))
+    ws.fill_(0xFF)
+    lt.lt_attn_bwd(Qd, Kd, Vd, Od, dOd, Ld, dQ, dK, dV, cfg.causal, cfg.scale, ws)
+    assert lt.lt_attn_check_status(ws) == lt.LT_OK, lt.last_cuda_error()
+    return dQ.cpu(), dK.cpu(), dV.cpu()
+
+
+def check_grads(got, ref, what):
+    for name, g, r in zip(("dQ", "dK", "dV"), got, ref):
+        g = g.double().numpy()
+        assert np.all(np.isfinite(g)), f"{what} {name}: non-finite output"
+        rf, ma = rel_fro(g, r), max_abs(g, r)
+        assert rf <= REL_FRO_TOL, f"{what} {name}: rel Frobenius {rf:.3e}"
+        assert ma <= MAX_ABS_TOL, f"{what} {name}: max abs {ma:.3e}"
+
+
+# ------------------------------------------------------------------ tensor-core tile conventions
+
+@pytest.mark.parametrize("mode", [0, 1, 2, 3])
+def test_tile_gemm_operand_conventions(lt, mode):
+    gen = torch.Generator().manual_seed(100 + mode)
+    A = torch.randn(128, 128, generator=gen).half()
+    B = torch.randn(128, 128, generator=gen).half()
+    ref = {0: A.double() @ B.double().T, 1: A.double() @ B.double(),
+           2: A.double().T @ B.double(), 3: A.double() @ B.double()}[mode]
+    C = torch.full((128, 128), float("nan"), dtype=torch.float32, device="cuda")
+    ws = lt.alloc_workspace(256)
+    lt.lt_dbg_tile_gemm(A.cuda(), B.cuda(), C, mode, ws)
+    assert lt.lt_attn_check_status(ws) == lt.LT_OK, lt.last_cuda_error()
+    err = (C.cpu().double() - ref).abs().max().item()
+    assert err < 1e-3, f"mode {mode}: max abs error {err}"
+
+
+# ------------------------------------------------------------------ forward
+
+FWD_SHAPES = [
+    (1, 2, 2, 128, 64, True), (1, 2, 2, 128, 128, True), (2, 4, 2, 384, 64, True),
+    (1, 5, 1, 512, 128, True), (1, 2, 2, 256, 128, False), (2, 2, 1, 384, 64, False),
+]
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,S,D,causal", FWD_SHAPES)
+def test_forward_matches_oracle(lt, oracle, B, Hq, Hkv, S, D, causal):
+    cfg = workloads.custom(B, Hq, Hkv, S, D, causal, qkv_std=1.0, do_std=1.0, seed=S + D)
+    Q, K, V, _ = workloads.make_inputs(cfg)
+    O, LSE = run_fwd(lt, Q, K, V, cfg)
+    O_ref, LSE_ref = oracle.attn_fwd(Q.double().numpy(), K.double().numpy(), V.double().numpy(), causal, cfg.scale)
+    assert rel_fro(O.cpu().double().numpy(), O_ref) <= FWD_O_REL_FRO_TOL
+    assert max_abs(LSE.cpu().double().numpy(), LSE_ref) <= FWD_LSE_ABS_TOL
+
+
+# ------------------------------------------------------------------ backward
+
+def test_delta_preprocess_matches_oracle(lt, oracle):
+    """delta is stored after the status block of the backward workspace."""
+    cfg = workloads.custom(2, 3, 3, 256, 128, True, seed=7)
+    Q, K, V, dO = workloads.make_inputs(cfg)
+    O_ref, LSE_ref = oracle.attn_fwd(Q.double().numpy(), K.double().numpy(), V.double().numpy(), True, cfg.scale)
+    O16 = torch.from_numpy(O_ref).half()
+    Qd, Kd, Vd, Od, dOd = (t.cuda() for t in (Q, K, V, O16, dO))
+    Ld = torch.from_numpy(LSE_ref).float().cuda()
+    dQ, dK, dV = torch.empty_like(Qd), torch.empty_like(Kd), torch.empty_like(Vd)
+    ws = lt.alloc_workspace(lt.lt_attn_bwd_workspace_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.S, cfg.D))
+    lt.lt_attn_bwd(Qd, Kd, Vd, Od, dOd, Ld, dQ, dK, dV, True, cfg.scale, ws)
+    assert lt.lt_attn_check_status(ws) == lt.LT_OK
+    n = cfg.B * cfg.Hq * cfg.S
+    delta = ws[256:256 + 4 * n].view(torch.float32).cpu().double().numpy().reshape(cfg.B, cfg.Hq, cfg.S)
+    ref = oracle.delta(dO.double().numpy(), O16.double().numpy())
+    np.testing.assert_allclose(delta, ref, rtol=1e-5, atol=1e-6 * np.abs(ref).max())
+
+
+BWD_SHAPES = [
+    # B, Hq, Hkv, S, D, causal
+    (1, 2, 2, 128, 64, True), (1, 2, 2, 128, 128, True), (1, 1, 1, 256, 128, True),
+    (2, 4, 2, 384, 64, True), (1, 5, 1, 512, 128, True), (2, 8, 1, 256, 128, True),
+    (1, 2, 2, 256, 128, False), (2, 4, 2, 384, 64, False), (1, 1, 1, 128, 128, False),
+]
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,S,D,causal", BWD_SHAPES)
+@pytest.mark.parametrize("stds", [(1.0, 1.0), (None, 1e-2)])
+def test_backward_matches_oracle_small(lt, oracle, B, Hq, Hkv, S, D, causal, stds):
+    """Several tiles, GQA groups, both head dims; forward state taken from the oracle
+    (O rounded to fp16, LSE to fp32) so the backward is judged on its own."""
+    cfg = workloads.custom(B, Hq, Hkv, S, D, causal, qkv_std=stds[0], do_std=stds[1], seed=B * 1000 + S + D)
+    Q, K, V, dO = workloads.make_inputs(cfg)
+    Qn, Kn, Vn, dOn = (t.double().numpy() for t in (Q, K, V, dO))
+    O_ref, LSE_ref = oracle.attn_fwd(Qn, Kn, Vn, causal, cfg.scale)
+    ref = oracle.attn_bwd(Qn, Kn, Vn, dOn, causal, cfg.scale)
+    got = run_bwd(lt, Q, K, V, torch.from_numpy(O_ref).half(), dO, torch.from_numpy(LSE_ref).float(), cfg)
+    check_grads(got, ref, f"{cfg}")
+
+
+def test_tiny_config_end_to_end(lt, oracle):
+    """The tiny benchmark configuration with the library's own forward feeding its backward."""
+    cfg = workloads.CONFIGS["tiny"]
+    Q, K, V, dO = workloads.make_inputs(cfg)
+    O, LSE = run_fwd(lt, Q, K, V, cfg)
+    got = run_bwd(lt, Q, K, V, O.cpu(), dO, LSE.cpu(), cfg)
+    ref = oracle.attn_bwd(*(t.double().numpy() for t in (Q, K, V, dO)), cfg.causal, cfg.scale)
+    check_grads(got, ref, "tiny")
+
+
+def test_backward_is_linear_in_dO_and_repeatable(lt, oracle):
+    cfg = workloads.custom(1, 4, 2, 256, 128, True, seed=11)
+    Q, K, V, dO = workloads.make_inputs(cfg)
+    O, LSE = run_fwd(lt, Q, K, V, cfg)
+    a = run_bwd(lt, Q, K, V, O.cpu(), dO, LSE.cpu(), cfg)
+    b = run_bwd(lt, Q, K, V, O.cpu(), dO, LSE.cpu(), cfg)
+    # dK and dV have a fixed summation order; dQ is reduced with atomics
+    assert torch.equal(a[1], b[1]) and torch.equal(a[2], b[2])
+    assert rel_fro(a[0].double().numpy(), b[0].double().numpy()) < 1e-3
+    c = run_bwd(lt, Q, K, V, O.cpu(), (dO.float() * 4).half(), LSE.cpu(), cfg)
+    for x, y in zip(a, c):
+        assert rel_fro(y.double().numpy() / 4, x.double().numpy()) < 2e-3
+
+
+def test_zero_dO_gives_zero_gradients(lt):
+    cfg = workloads.custom(1, 2, 1, 256, 64, True, seed=12)
+    Q, K, V, dO = workloads.make_inputs(cfg)
+    O, LSE = run_fwd(lt, Q, K, V, cfg)
+    got = run_bwd(lt, Q, K, V, O.cpu(), torch.zeros_like(dO), LSE.cpu(), cfg)
+    for g in got:
+        assert torch.count_nonzero(g) == 0
+
+
+def test_host_buffer_entry_point(lt, oracle):
+    cfg = workloads.custom(1, 4, 2, 256, 128, True, seed=13)
+    Q, K, V, dO = (t.pin_memory() for t in workloads.make_inputs(cfg))
+    O = torch.empty_like(Q).pin_memory()
+    LSE = torch.empty(Q.shape[:3], dtype=torch.float32).pin_memory()
+    dQ, dK, dV = torch.empty_like(Q).pin_memory(), torch.empty_like(K).pin_memory(), torch.empty_like(V).pin_memory()
+    arena = lt.alloc_workspace(lt.lt_attn_host_arena_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.S, cfg.D))
+    lt.lt_attn_fwd_bwd_host(Q, K, V, dO, O, LSE, dQ, dK, dV, cfg.causal, cfg.scale, arena)
+    torch.cuda.synchronize()
+    ref = oracle.attn_bwd(*(t.double().numpy() for t in (Q, K, V, dO)), cfg.causal, cfg.scale)
+    check_grads((dQ, dK, dV), ref, "host entry")
+
+
+# ------------------------------------------------------------------ benchmark configurations, full size
+
+def _full_size_check(lt, oracle, name, units):
+    """Run the whole configuration on the GPU (the launch the benchmark times); compare the
+    (batch, kv head) units in `units` -- all query heads of the group -- against the oracle."""
+    cfg = workloads.CONFIGS[name]
+    Q, K, V, dO = workloads.make_inputs(cfg)
+    O, LSE = run_fwd(lt, Q, K, V, cfg)
+    got = run_bwd(lt, Q, K, V, O.cpu(), dO, LSE.cpu(), cfg)
+    G = cfg.Hq // cfg.Hkv
+    for (b, g) in units:
+        hs = slice(g * G, (g + 1) * G)
+        sub = [Q[b:b + 1, hs], K[b:b + 1, g:g + 1], V[b:b + 1, g:g + 1], dO[b:b + 1, hs]]
+        sub_n = [t.double().numpy() for t in sub]
+        O_ref, LSE_ref = oracle.attn_fwd(*sub_n[:3], cfg.causal, cfg.scale)
+        assert rel_fro(O[b:b + 1, hs].cpu().double().numpy(), O_ref) <= FWD_O_REL_FRO_TOL
+        assert max_abs(LSE[b:b + 1, hs].cpu().double().numpy(), LSE_ref) <= FWD_LSE_ABS_TOL
+        ref = oracle.attn_bwd(*sub_n, cfg.causal, cfg.scale)
+        sub_got = (got[0][b:b + 1, hs], got[1][b:b + 1, g:g + 1], got[2][b:b + 1, g:g + 1])
+        check_grads(sub_got, ref, f"{name} unit {(b, g)}")
+    # properties that hold at any size: finite everywhere, first query row has zero dQ
+    for t in got:
+        assert torch.isfinite(t.float()).all()
+    assert torch.count_nonzero(got[0][:, :, 0]) == 0
+
+
+def test_llama2_7b_config_all_heads(lt, oracle):
+    cfg = workloads.CONFIGS["llama2_7b"]
+    _full_size_check(lt, oracle, "llama2_7b", [(0, g) for g in range(cfg.Hkv)])
+
+
+def test_baichuan2_13b_config_sampled_heads(lt, oracle):
+    _full_size_check(lt, oracle, "baichuan2_13b", [(0, 0), (0, 17), (0, 39)])
+
+
+def test_qwen25_32b_gqa_config_sampled_groups(lt, oracle):
+    _full_size_check(lt, oracle, "qwen25_32b_gqa", [(0, 0), (0, 7)])
+
+
+def test_llama2_70b_gqa_config_sampled_groups(lt, oracle):
+    _full_size_check(lt, oracle, "llama2_70b_gqa", [(0, 3), (1, 7)])
