@@ -44,7 +44,10 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", default="llama2_7b", choices=sorted(workloads.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the timed oracle leg (debugging)")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the timed oracle leg (profiling runs)")
+    ap.add_argument("--clock-sample-ms", type=int, default=600,
+                    help="untimed busy period before the timed steps so nvidia-smi samples clocks under load "
+                         "(0 for profiler runs)")
     return ap.parse_args()
 
 
@@ -240,7 +243,7 @@ def run_ours(args, cfg):
         time.sleep(0.15)
     barrier()
     # keep the GPU busy long enough for nvidia-smi to sample clocks under this load
-    busy_until = time.perf_counter() + 0.6
+    busy_until = time.perf_counter() + args.clock_sample_ms * 1e-3
     while time.perf_counter() < busy_until:
         step()
     barrier()
@@ -250,7 +253,7 @@ def run_ours(args, cfg):
     t1.record()
     barrier()
     total_ms = t0.elapsed_time(t1)
-    busy_until = time.perf_counter() + 0.3
+    busy_until = time.perf_counter() + args.clock_sample_ms * 0.5e-3
     while time.perf_counter() < busy_until:
         step()
     torch.cuda.synchronize()
