@@ -54,7 +54,8 @@ typedef unsigned short lt_half;
 
 /* Bytes of caller-owned device workspace the calls below need; 0 means the shape is
  * not supported.  The workspace must be 256-byte aligned.  Layout (backward): a
- * 256-byte status block, delta fp32 [B,Hq,S], an fp32 dQ accumulator [B,Hq,S,D]. */
+ * 256-byte status block, delta fp32 [B,Hq,S], -LSE*log2(e) fp32 [B,Hq,S], an fp32 dQ
+ * accumulator [B,Hq,S,D]. */
 size_t lt_attn_fwd_workspace_bytes(int B, int Hq, int Hkv, int S, int D);
 size_t lt_attn_bwd_workspace_bytes(int B, int Hq, int Hkv, int S, int D);
 
@@ -126,7 +127,9 @@ int lt_attn_fwd_num_launches(void);
  *   mode 0: C = A  B^T   (A rows = M, B rows = N; both contraction-contiguous)
  *   mode 1: C = A  B     (B rows = contraction index)
  *   mode 2: C = A^T B    (A and B rows = contraction index)
- *   mode 3: C = A  B     (A staged through tensor memory instead of shared memory) */
+ *   mode 3: C = A  B     (A staged through tensor memory instead of shared memory)
+ *   mode 4: as mode 0, with the accumulator read back in the 16-lane x 256-bit
+ *           arrangement that the dQ reduction uses */
 int lt_dbg_tile_gemm(const lt_half *A, const lt_half *B, float *C, int mode,
                      void *workspace, size_t workspace_bytes, lt_stream_t stream);
 

@@ -79,7 +79,7 @@ dbg_tile_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             const uint32_t koff = (kk >> 2) * kBoxBytes + (kk & 3) * 32;  // contraction-contiguous operand
             const uint32_t roff = kk * 16 * 128;                          // contraction index = row
             const uint32_t acc = kk > 0;
-            if (mode == 0) {
+            if (mode == 0 || mode == 4) {
                 umma_ss(tmem, desc_kmajor(a0 + koff), desc_kmajor(b0 + koff), make_idesc(128, 128, false, false), acc);
             } else if (mode == 1) {
                 umma_ss(tmem, desc_kmajor(a0 + koff), desc_mnmajor(b0 + roff, kBoxBytes),
@@ -96,7 +96,28 @@ dbg_tile_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     }
     ok = ok && mbar_wait(&sm.bar_mma, 0, &sm.abort_flag, status, 102);
     tc_fence_after_sync();
-    if (ok) {
+    if (ok && mode == 4) {
+        // read the accumulator back in the 16-lane x 256-bit arrangement the dQ reduction uses
+        const int lane = tid & 31;
+#pragma unroll
+        for (int ch = 0; ch < 2; ++ch) {
+#pragma unroll
+            for (int lh = 0; lh < 2; ++lh) {
+                uint32_t r[32];
+                tmem_ld_16x256b_x8(tmem + (static_cast<uint32_t>(warp * 32 + lh * 16) << 16) + ch * 64, r);
+                tmem_wait_ld();
+                float *base = c_gmem + static_cast<size_t>(warp * 32 + lh * 16 + (lane >> 2)) * kTile + ch * 64 +
+                              2 * (lane & 3);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    *reinterpret_cast<float2 *>(base + 8 * k) =
+                        make_float2(__uint_as_float(r[4 * k]), __uint_as_float(r[4 * k + 1]));
+                    *reinterpret_cast<float2 *>(base + 8 * kTile + 8 * k) =
+                        make_float2(__uint_as_float(r[4 * k + 2]), __uint_as_float(r[4 * k + 3]));
+                }
+            }
+        }
+    } else if (ok) {
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
             uint32_t r[32];
@@ -119,7 +140,7 @@ dbg_tile_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
 extern "C" int lt_dbg_tile_gemm(const lt_half *A, const lt_half *B, float *C, int mode, void *workspace,
                                 size_t workspace_bytes, lt_stream_t stream) {
     using namespace lt;
-    if (!A || !B || !C || mode < 0 || mode > 3) return LT_ERR_INVALID_ARG;
+    if (!A || !B || !C || mode < 0 || mode > 4) return LT_ERR_INVALID_ARG;
     if (!aligned16(A) || !aligned16(B) || !aligned16(C)) return LT_ERR_UNSUPPORTED;
     if (!workspace || !aligned256(workspace) || workspace_bytes < static_cast<size_t>(kStatusBytes))
         return LT_ERR_WORKSPACE;

@@ -38,9 +38,9 @@ def test_library_exports_every_declared_symbol(binding):
 
 
 def test_workspace_sizes(binding):
-    # 256-byte status block + delta fp32 [B,Hq,S] + dQ accumulator fp32 [B,Hq,S,D]
-    assert binding.lt_attn_bwd_workspace_bytes(1, 2, 2, 128, 64) == 256 + 1024 + 65536
-    assert binding.lt_attn_bwd_workspace_bytes(1, 32, 32, 4096, 128) == 256 + 524288 + 67108864
+    # 256-byte status block + delta and -LSE*log2e fp32 [B,Hq,S] each + dQ accumulator fp32 [B,Hq,S,D]
+    assert binding.lt_attn_bwd_workspace_bytes(1, 2, 2, 128, 64) == 256 + 2 * 1024 + 65536
+    assert binding.lt_attn_bwd_workspace_bytes(1, 32, 32, 4096, 128) == 256 + 2 * 524288 + 67108864
     assert binding.lt_attn_fwd_workspace_bytes(1, 2, 2, 128, 64) == 256
     # unsupported shapes report 0
     assert binding.lt_attn_bwd_workspace_bytes(1, 2, 2, 100, 64) == 0

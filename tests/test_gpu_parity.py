@@ -65,13 +65,13 @@ def check_grads(got, ref, what):
 
 # ------------------------------------------------------------------ tensor-core tile conventions
 
-@pytest.mark.parametrize("mode", [0, 1, 2, 3])
+@pytest.mark.parametrize("mode", [0, 1, 2, 3, 4])
 def test_tile_gemm_operand_conventions(lt, mode):
     gen = torch.Generator().manual_seed(100 + mode)
     A = torch.randn(128, 128, generator=gen).half()
     B = torch.randn(128, 128, generator=gen).half()
     ref = {0: A.double() @ B.double().T, 1: A.double() @ B.double(),
-           2: A.double().T @ B.double(), 3: A.double() @ B.double()}[mode]
+           2: A.double().T @ B.double(), 3: A.double() @ B.double(), 4: A.double() @ B.double().T}[mode]
     C = torch.full((128, 128), float("nan"), dtype=torch.float32, device="cuda")
     ws = lt.alloc_workspace(256)
     lt.lt_dbg_tile_gemm(A.cuda(), B.cuda(), C, mode, ws)
