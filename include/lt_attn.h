@@ -12,7 +12,7 @@
  *     K, V, dK, dV have H = Hkv.  LSE is fp32 [B, Hq, S].  fp16 is IEEE binary16.
  *   - Grouped-query attention: query head h reads key/value head h / (Hq / Hkv);
  *     dK and dV are summed over the Hq / Hkv query heads of a group.
- *   - scores = scale * Q K^T; causal != 0 hides key j from query i when j > i.
+ *   - scores = scale * Q K^T with a finite, non-zero scale; causal != 0 hides key j from query i when j > i.
  *     LSE_i = ln sum_j exp(scores_ij) over visible keys (natural logarithm).
  *   - Supported shapes: D in {64, 128}, S a positive multiple of 128, Hq % Hkv == 0.
  *     Anything else returns LT_ERR_UNSUPPORTED and launches nothing.
@@ -38,7 +38,7 @@ extern "C" {
 
 typedef enum lt_status {
     LT_OK = 0,
-    LT_ERR_INVALID_ARG = 1,    /* NULL pointer, non-positive size, Hq % Hkv != 0, non-finite scale */
+    LT_ERR_INVALID_ARG = 1,    /* NULL pointer, non-positive size, Hq % Hkv != 0, zero or non-finite scale */
     LT_ERR_UNSUPPORTED = 2,    /* shape, alignment or device outside the supported set */
     LT_ERR_WORKSPACE = 3,      /* workspace NULL, misaligned (256 B) or too small */
     LT_ERR_CUDA = 4,           /* a CUDA runtime/driver call failed; see lt_last_cuda_error */
@@ -54,8 +54,8 @@ typedef unsigned short lt_half;
 
 /* Bytes of caller-owned device workspace the calls below need; 0 means the shape is
  * not supported.  The workspace must be 256-byte aligned.  Layout (backward): a
- * 256-byte status block, delta fp32 [B,Hq,S], -LSE*log2(e) fp32 [B,Hq,S], an fp32 dQ
- * accumulator [B,Hq,S,D]. */
+ * 256-byte status block, -delta and -LSE/scale as 16-byte rows of fp16 (hi, lo, 0 x 6)
+ * with 256*hi + lo = value, [B,Hq,S] rows each, then an fp32 dQ accumulator [B,Hq,S,D]. */
 size_t lt_attn_fwd_workspace_bytes(int B, int Hq, int Hkv, int S, int D);
 size_t lt_attn_bwd_workspace_bytes(int B, int Hq, int Hkv, int S, int D);
 
@@ -129,7 +129,9 @@ int lt_attn_fwd_num_launches(void);
  *   mode 2: C = A^T B    (A and B rows = contraction index)
  *   mode 3: C = A  B     (A staged through tensor memory instead of shared memory)
  *   mode 4: as mode 0, with the accumulator read back in the 16-lane x 256-bit
- *           arrangement that the dQ reduction uses */
+ *           arrangement that the dQ reduction uses
+ *   mode 5: C = A B^T + 1000 * B[n][0] added to column n through one extra, unswizzled
+ *           contraction step (the way the kernels subtract LSE and delta) */
 int lt_dbg_tile_gemm(const lt_half *A, const lt_half *B, float *C, int mode,
                      void *workspace, size_t workspace_bytes, lt_stream_t stream);
 

@@ -23,6 +23,11 @@ NVCC_FLAGS = [
 ]
 
 
+def _extra_flags() -> list[str]:
+    """Extra nvcc flags from LT_NVCC_FLAGS (development builds, e.g. -DLT_BWD_TRACE)."""
+    return os.environ.get("LT_NVCC_FLAGS", "").split()
+
+
 def _nvcc() -> str:
     cand = os.environ.get("NVCC") or "/usr/local/cuda/bin/nvcc"
     return cand if Path(cand).exists() else "nvcc"
@@ -42,7 +47,7 @@ def build(force: bool = False, verbose: bool = False) -> Path:
 
     def compile_one(job):
         src, obj = job
-        cmd = [_nvcc(), *NVCC_FLAGS, "-c", str(src), "-o", str(obj)]
+        cmd = [_nvcc(), *NVCC_FLAGS, *_extra_flags(), "-c", str(src), "-o", str(obj)]
         res = subprocess.run(cmd, capture_output=True, text=True)
         (OBJ / (src.stem + ".ptxas.log")).write_text(res.stderr)
         if res.returncode != 0:

@@ -1,9 +1,9 @@
 // Attention backward (Algorithm 1 of the paper, Section 4.1) for sm_100a.
 //
 // Three kernels per call:
-//   bwd_preprocess_kernel : delta = rowsum(dO * O), -LSE*log2(e), zero the fp32 dQ
-//                           accumulator, record max |delta| and max ||dO_row||^2
-//                           (together with the V tile they bound |dS|)
+//   bwd_preprocess_kernel : delta = rowsum(dO * O); writes -delta and -LSE/scale as fp16
+//                           (hi, lo) pairs, zeroes the fp32 dQ accumulator, records
+//                           max |delta| and max ||dO_row||^2 (with the V tile they bound |dS|)
 //   bwd_main_kernel       : per (batch, kv head, key tile j): loop over the group's
 //                           query heads and the visible query tiles i, recompute
 //                           P^T from LSE, and run the five tile contractions on
@@ -14,17 +14,20 @@
 // across workers): here a CTA owns one key/value tile, keeps dK_j and dV_j resident in
 // tensor memory for the whole loop, and the cross-CTA reduction falls on dQ instead.
 //
-// The main kernel is warp specialised (16 warps):
-//   warp 0       TMA producer: K_j, V_j once; then a two-stage ring of {Q_i, dO_i, -LSE*log2e, delta}
+// The main kernel is warp specialised (14 warps, 144 registers per thread):
+//   warp 0       TMA producer (one thread): K_j, V_j once; then a two-stage ring of Q_i and a
+//                single-buffered dO_i; the warp also owns the tensor-memory allocation
 //   warp 1       tensor-core issuer (one thread)
-//   warp 2       owns the tensor-memory allocation
-//   warps 4-11   softmax / dS warps: warps 4-7 take query columns 0-63 of a tile pair,
-//                warps 8-11 columns 64-127; each thread owns one key row
-//   warps 12-15  dQ reduction: tensor memory -> fp32 red.global into the accumulator
+//   warps 2-9    softmax / dS warps: warps 2-5 take query columns 0-63 of a tile pair,
+//                warps 6-9 columns 64-127; each thread owns one key row
+//   warps 10-13  dQ reduction: tensor memory -> fp32 red.global into the accumulator
 // Transposed scores are used (S^T = K Q^T, dP^T = V dO^T) so that P^T, written back to
 // tensor memory as fp16, is directly the A operand of dV += P^T dO; dS^T goes through
 // shared memory once and serves both dK += dS^T Q (contraction-contiguous A) and
-// dQ = dS K (row-contracted A).
+// dQ = dS K (row-contracted A).  The row terms -LSE_i/scale and -delta_i are added inside
+// the S^T and dP^T products by one extra 16-element contraction step whose operands are
+// (256, 1, 0...) and the (hi, lo, 0...) split of the term, so the softmax warps never
+// touch LSE or delta.
 #include "lt_common.cuh"
 #include "lt_host.h"
 
@@ -38,7 +41,7 @@ constexpr float kLog2e = 1.4426950408889634f;
 enum {
     kWaitKV = 201, kWaitStageEmpty = 202, kWaitStageFull = 203, kWaitSFull = 204, kWaitPReady = 205,
     kWaitDpFull = 206, kWaitDsReady = 207, kWaitDsFree = 208, kWaitDqFull = 209, kWaitDqEmpty = 210,
-    kWaitDkvFull = 211, kBadSmemAlign = 220
+    kWaitDkvFull = 211, kWaitDoFull = 212, kWaitDoEmpty = 213, kBadSmemAlign = 220
 };
 
 // ----------------------------------------------------------------------------- preprocess
@@ -46,8 +49,8 @@ enum {
 template <int D>
 __global__ void __launch_bounds__(256)
 bwd_preprocess_kernel(const __half *__restrict__ dO, const __half *__restrict__ O, const float *__restrict__ lse,
-                      float *__restrict__ delta, float *__restrict__ neg_lse_log2, float *__restrict__ dq_acc,
-                      long long n_rows, unsigned int *status) {
+                      uint4 *__restrict__ delta_ext, uint4 *__restrict__ lse_ext, float *__restrict__ dq_acc,
+                      long long n_rows, float inv_scale, unsigned int *status) {
     constexpr int kLanesPerRow = D / 8;
     constexpr int kRowsPerWarp = 32 / kLanesPerRow;
     const int lane = threadIdx.x & 31;
@@ -83,8 +86,9 @@ bwd_preprocess_kernel(const __half *__restrict__ dO, const __half *__restrict__ 
         }
         if (row < n_rows) {
             if (sub == 0) {
-                delta[row] = acc;
-                neg_lse_log2[row] = -lse[row] * kLog2e;
+                // operand rows of the main kernel's extra contraction step: 256*hi + lo = value
+                delta_ext[row] = make_uint4(split_hi_lo(-acc), 0u, 0u, 0u);
+                lse_ext[row] = make_uint4(split_hi_lo(-lse[row] * inv_scale), 0u, 0u, 0u);
             }
             max_abs_delta = fmaxf(max_abs_delta, fabsf(acc));
             max_norm2 = fmaxf(max_norm2, n2);
@@ -118,11 +122,56 @@ bwd_finalize_kernel(const float *__restrict__ dq_acc, __half *__restrict__ dQ, l
     }
 }
 
+// ----------------------------------------------------------------------------- optional cycle trace
+// Built only with -DLT_BWD_TRACE (development aid): per-role cycle totals, summed over all CTAs.
+// Slot = 16 * role + (wait code - 200); slot 16 * role + 15 = the role's whole loop.
+enum { kRoleProducer = 0, kRoleMma = 1, kRoleCompute = 2, kRoleReduce = 3 };
+#ifdef LT_BWD_TRACE
+__device__ unsigned long long g_bwd_trace[80];
+struct Trace {
+    unsigned int acc[16];
+    unsigned int t0;
+    __device__ __forceinline__ void start() {
+        t0 = static_cast<unsigned int>(clock());
+#pragma unroll
+        for (int i = 0; i < 16; ++i) acc[i] = 0;
+    }
+    __device__ __forceinline__ void flush(int role) {
+        acc[15] = static_cast<unsigned int>(clock()) - t0;
+        if ((threadIdx.x & 31) == 0) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+                if (acc[i]) atomicAdd(&g_bwd_trace[16 * role + i], static_cast<unsigned long long>(acc[i]));
+        }
+    }
+};
+#define LT_TRACE_BEGIN() Trace trace_; trace_.start()
+#define LT_TRACE_MARK(var) const unsigned int var = static_cast<unsigned int>(clock())
+#define LT_TRACE_SINCE(slot, var) trace_.acc[slot] += static_cast<unsigned int>(clock()) - var
+#define LT_TRACE_END(role) trace_.flush(role)
+#define LT_WAIT(bar, parity, code) traced_wait(trace_, bar, parity, abort_flag, p.status, code)
+__device__ __forceinline__ bool traced_wait(Trace &tr, uint64_t *bar, uint32_t parity, volatile int *abort_flag,
+                                            unsigned int *status, int code) {
+    const unsigned int t0 = static_cast<unsigned int>(clock());
+    const bool r = mbar_wait(bar, parity, abort_flag, status, code);
+    tr.acc[code - 200] += static_cast<unsigned int>(clock()) - t0;
+    return r;
+}
+#else
+#define LT_TRACE_BEGIN()
+#define LT_TRACE_MARK(var)
+#define LT_TRACE_SINCE(slot, var)
+#define LT_TRACE_END(role)
+#define LT_WAIT(bar, parity, code) mbar_wait(bar, parity, abort_flag, p.status, code)
+#endif
+
 // ----------------------------------------------------------------------------- main kernel
-constexpr int kStages = 2;
-constexpr int kBwdThreads = 512;
-constexpr int kComputeWarp0 = 4, kNumComputeWarps = 8;
-constexpr int kReduceWarp0 = 12, kNumReduceWarps = 4;
+constexpr int kQStages = 2;   // Q_i ring; dO_i is single-buffered (it is dead once dV has been issued)
+constexpr int kBwdThreads = 448;  // 14 warps: 65536 / 448 leaves 144 registers per thread
+constexpr int kComputeWarp0 = 2, kNumComputeWarps = 8;
+constexpr int kReduceWarp0 = 10, kNumReduceWarps = 4;
+constexpr int kExtBytes = 2048;            // 128 rows x 16 bytes: one operand of the extra contraction step
+constexpr float kPScaleLog2Max = 14.f;     // P is kept as P * 2^c with c <= 14 so that fp16(P') <= 16384
 
 template <int D>
 struct BwdSmem {
@@ -130,13 +179,16 @@ struct BwdSmem {
     static constexpr int kTile = kBoxes * kBoxBytesBwd;
     uint8_t k[kTile];
     uint8_t v[kTile];
-    uint8_t q[kStages][kTile];
-    uint8_t d_o[kStages][kTile];
-    uint8_t ds[2 * kBoxBytesBwd];           // dS^T: rows = key index, 128 query columns in two swizzled tiles
-    float neg_lse_log2[kStages][kTileRows]; // -LSE * log2(e) of the stage's query tile
-    float delta[kStages][kTileRows];
+    uint8_t q[kQStages][kTile];
+    uint8_t d_o[kTile];
+    uint8_t ds[2 * kBoxBytesBwd];      // dS^T: rows = key index, 128 query columns in two swizzled tiles
+    // operands of the extra contraction step that subtracts LSE/scale from S and delta from dP
+    uint8_t ext_ones[kExtBytes];       // rows (256, 1, 0...): goes with K_j and with V_j
+    uint8_t ext_q[kQStages][kExtBytes];// rows (hi, lo, 0...) of -LSE/scale for the stage's query tile
+    uint8_t ext_do[kExtBytes];         // rows (hi, lo, 0...) of -delta
+    uint8_t ext_zero[kExtBytes];       // contraction elements 8-15 of all of the above
     uint64_t bar_kv;
-    uint64_t bar_stage_full[kStages], bar_stage_empty[kStages];
+    uint64_t bar_q_full[kQStages], bar_q_empty[kQStages], bar_do_full, bar_do_empty;
     uint64_t bar_s_full, bar_p_ready, bar_dp_full, bar_ds_ready, bar_ds_free, bar_dq_full, bar_dq_empty, bar_dkv_full;
     float red[4];
     float ds_mult;
@@ -145,8 +197,8 @@ struct BwdSmem {
 };
 
 struct BwdParams {
-    const float *neg_lse_log2;
-    const float *delta;
+    const uint4 *lse_ext;    // per query row: fp16 (hi, lo, 0 x 6) with 256*hi + lo = -LSE / scale
+    const uint4 *delta_ext;  // per query row: fp16 (hi, lo, 0 x 6) with 256*hi + lo = -delta
     float *dq_acc;
     __half *dK;
     __half *dV;
@@ -163,12 +215,14 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     using Smem = BwdSmem<D>;
     constexpr int kBoxes = D / 64;
     constexpr uint32_t kTileBytes = kBoxes * kBoxBytesBwd;
-    constexpr uint32_t kStageBytes = 2 * kTileBytes + 2 * kTileRows * sizeof(float);
     constexpr uint32_t kTmemCols = 512;
     constexpr uint32_t kColS = 0, kColdP = 128, kColdV = 256, kColdK = 384;
 
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     Smem &sm = *reinterpret_cast<Smem *>(smem_raw);
+#ifdef LT_BWD_TRACE
+    const long long trace_cta_t0 = clock64();
+#endif
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
     const int lane = tid & 31;
@@ -192,10 +246,12 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         sm.abort_flag = smem_ok ? 0 : 1;
         if (!smem_ok) atomicCAS(p.status + kStatusWordTimeout, 0u, static_cast<unsigned int>(kBadSmemAlign));
         mbar_init(&sm.bar_kv, 1);
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(&sm.bar_stage_full[s], 1);
-            mbar_init(&sm.bar_stage_empty[s], 1);
+        for (int s = 0; s < kQStages; ++s) {
+            mbar_init(&sm.bar_q_full[s], 1);
+            mbar_init(&sm.bar_q_empty[s], 1);
         }
+        mbar_init(&sm.bar_do_full, 1);
+        mbar_init(&sm.bar_do_empty, 1);
         mbar_init(&sm.bar_s_full, 1);
         mbar_init(&sm.bar_p_ready, kNumComputeWarps);
         mbar_init(&sm.bar_dp_full, 1);
@@ -210,9 +266,18 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         tma_prefetch_desc(&map_v);
         tma_prefetch_desc(&map_do);
     }
-    if (warp == 2) {
+    if (warp == 0) {
         tmem_alloc(&sm.tmem_base, kTmemCols);
         tmem_relinquish();
+    }
+    if (warp == 1) {
+        // constant operands of the extra contraction step
+        const __half2 ones = __halves2half2(__float2half_rn(256.f), __float2half_rn(1.f));
+        for (int r = lane; r < kTileRows; r += 32) {
+            reinterpret_cast<uint4 *>(sm.ext_ones)[r] = make_uint4(*reinterpret_cast<const uint32_t *>(&ones), 0u, 0u, 0u);
+            reinterpret_cast<uint4 *>(sm.ext_zero)[r] = make_uint4(0u, 0u, 0u, 0u);
+        }
+        fence_proxy_async_smem();
     }
     tc_fence_before_sync();
     __syncthreads();
@@ -237,9 +302,10 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
     }
 
-    // Power-of-two factor applied to dS before it is rounded to fp16, chosen from a bound
+    // Power-of-two factor 2^c carried by dS before it is rounded to fp16, chosen from a bound
     // on |dS| <= |dP| + |delta| <= max||dO_row|| * max||V_row|| + max|delta| so that the scaled
-    // values use fp16's normal range without overflow.  Undone exactly in the dQ/dK epilogues.
+    // values use fp16's normal range without overflow.  The factor rides on P (P' = P * 2^c,
+    // c <= 14), so dV and dQ/dK undo it exactly in their epilogues.
     if (warp >= kComputeWarp0 && warp < kComputeWarp0 + 4) {
         const int row = tid - kComputeWarp0 * 32;
         float n2 = 0.f;
@@ -270,116 +336,142 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const float do2 = __uint_as_float(p.status[kStatusWordMaxDoNorm2]);
         const float dmax = __uint_as_float(p.status[kStatusWordMaxAbsDelta]);
         const float bound = sqrtf(do2) * sqrtf(vmax2) + dmax;
-        int e = 24;                                  // all-zero dO: any factor works
+        int e = static_cast<int>(kPScaleLog2Max);    // all-zero dO: any factor works
         if (!(bound < 3.0e38f)) e = -14;             // inf/NaN inputs: outputs are non-finite anyway
-        else if (bound > 1e-30f) e = min(24, max(-14, ilogbf(32768.f / bound)));
-        sm.ds_mult = ldexpf(1.f, e);
+        else if (bound > 1e-30f) e = min(static_cast<int>(kPScaleLog2Max), max(-14, ilogbf(32768.f / bound)));
+        sm.ds_mult = static_cast<float>(e);
     }
     __syncthreads();
-    const float ds_mult = sm.ds_mult;
-    const float dq_mult = p.scale / ds_mult;
+    const float p_scale_log2 = sm.ds_mult;              // c
+    const float inv_p_scale = exp2f(-p_scale_log2);     // 2^-c, exact
+    const float dq_mult = p.scale * inv_p_scale;
+#ifdef LT_BWD_TRACE
+    const long long trace_prologue_end = clock64();
+#endif
 
-    if (warp == 0) {
-        // ================================================================= TMA producer
-        if (lane == 0 && smem_ok) {
-            int issued = 0;
-            for (int n = 0; n < n_iter; ++n) {
-                const int s = n & 1, k = n >> 1;
-                if (k >= 1 && !mbar_wait(&sm.bar_stage_empty[s], (k - 1) & 1, abort_flag, p.status, kWaitStageEmpty))
-                    break;
-                const long long q_row0 = q_row_of(n);
-                mbar_arrive_expect_tx(&sm.bar_stage_full[s], kStageBytes);
+    if (warp < kComputeWarp0) {
+        if (warp == 0) {
+            // ================================================================= TMA producer
+            if (lane == 0 && smem_ok) {
+                LT_TRACE_BEGIN();
+                int q_issued = 0, do_issued = 0;
+                for (int n = 0; n < n_iter; ++n) {
+                    const int s = n & 1, k = n >> 1;
+                    const long long q_row0 = q_row_of(n);
+                    if (k >= 1 && !LT_WAIT(&sm.bar_q_empty[s], (k - 1) & 1, kWaitStageEmpty)) break;
+                    mbar_arrive_expect_tx(&sm.bar_q_full[s], kTileBytes + kExtBytes);
 #pragma unroll
-                for (int x = 0; x < kBoxes; ++x) {
-                    tma_load_2d(sm.q[s] + x * kBoxBytesBwd, &map_q, &sm.bar_stage_full[s], x * 64,
-                                static_cast<int>(q_row0));
-                    tma_load_2d(sm.d_o[s] + x * kBoxBytesBwd, &map_do, &sm.bar_stage_full[s], x * 64,
-                                static_cast<int>(q_row0));
+                    for (int x = 0; x < kBoxes; ++x)
+                        tma_load_2d(sm.q[s] + x * kBoxBytesBwd, &map_q, &sm.bar_q_full[s], x * 64,
+                                    static_cast<int>(q_row0));
+                    bulk_load_1d(sm.ext_q[s], p.lse_ext + q_row0, kExtBytes, &sm.bar_q_full[s]);
+                    q_issued = n + 1;
+                    if (n >= 1 && !LT_WAIT(&sm.bar_do_empty, (n - 1) & 1, kWaitDoEmpty)) break;
+                    mbar_arrive_expect_tx(&sm.bar_do_full, kTileBytes + kExtBytes);
+#pragma unroll
+                    for (int x = 0; x < kBoxes; ++x)
+                        tma_load_2d(sm.d_o + x * kBoxBytesBwd, &map_do, &sm.bar_do_full, x * 64,
+                                    static_cast<int>(q_row0));
+                    bulk_load_1d(sm.ext_do, p.delta_ext + q_row0, kExtBytes, &sm.bar_do_full);
+                    do_issued = n + 1;
                 }
-                bulk_load_1d(sm.neg_lse_log2[s], p.neg_lse_log2 + q_row0, kTileRows * sizeof(float),
-                             &sm.bar_stage_full[s]);
-                bulk_load_1d(sm.delta[s], p.delta + q_row0, kTileRows * sizeof(float), &sm.bar_stage_full[s]);
-                issued = n + 1;
+                LT_TRACE_END(kRoleProducer);
+                if (*abort_flag) {
+                    // abandoned: give this CTA's own copies a bounded time to land before shared memory is released
+                    for (int t = 0; t < (1 << 16) && !mbar_try_wait(&sm.bar_kv, 0); ++t) {}
+                    for (int n = max(0, q_issued - kQStages); n < q_issued; ++n)
+                        for (int t = 0; t < (1 << 16) && !mbar_try_wait(&sm.bar_q_full[n & 1], (n >> 1) & 1); ++t) {}
+                    if (do_issued > 0)
+                        for (int t = 0; t < (1 << 16) && !mbar_try_wait(&sm.bar_do_full, (do_issued - 1) & 1); ++t) {}
+                }
             }
-            if (*abort_flag) {
-                // abandoned: give this CTA's own copies a bounded time to land before shared memory is released
-                for (int t = 0; t < (1 << 16) && !mbar_try_wait(&sm.bar_kv, 0); ++t) {}
-                for (int n = max(0, issued - kStages); n < issued; ++n)
-                    for (int t = 0; t < (1 << 16) && !mbar_try_wait(&sm.bar_stage_full[n & 1], (n >> 1) & 1); ++t) {}
+            __syncwarp();
+        } else if (warp == 1) {
+            // ================================================================= tensor-core issuer
+            if (lane == 0 && smem_ok) {
+                LT_TRACE_BEGIN();
+                const uint32_t sK = smem_u32(sm.k), sV = smem_u32(sm.v), sdS = smem_u32(sm.ds), sdO = smem_u32(sm.d_o);
+                const uint32_t s_ones = smem_u32(sm.ext_ones), s_zero = smem_u32(sm.ext_zero);
+                const uint64_t desc_ones = desc_kmajor_noswz(s_ones, s_zero - s_ones, 128);
+                const uint64_t desc_ext_do = desc_kmajor_noswz(smem_u32(sm.ext_do), s_zero - smem_u32(sm.ext_do), 128);
+                constexpr uint32_t idesc_s = make_idesc(128, 128, false, false);
+                constexpr uint32_t idesc_dv = make_idesc(128, D, false, true);
+                constexpr uint32_t idesc_dq = make_idesc(128, D == 128 ? 128 : D, true, true);
+                auto issue_s = [&](int n) {  // S^T = K_j Q_i^T - LSE_i / scale
+                    const uint32_t sQn = smem_u32(sm.q[n & 1]), s_ext = smem_u32(sm.ext_q[n & 1]);
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint32_t koff = (kk >> 2) * kBoxBytesBwd + (kk & 3) * 32;
+                        umma_ss(tmem + kColS, desc_kmajor(sK + koff), desc_kmajor(sQn + koff), idesc_s, kk > 0);
+                    }
+                    umma_ss(tmem + kColS, desc_ones, desc_kmajor_noswz(s_ext, s_zero - s_ext, 128), idesc_s, 1);
+                    umma_commit(&sm.bar_s_full);
+                };
+                bool ok = LT_WAIT(&sm.bar_kv, 0, kWaitKV) && LT_WAIT(&sm.bar_q_full[0], 0, kWaitStageFull);
+                if (ok) {
+                    tc_fence_after_sync();
+                    issue_s(0);
+                }
+                for (int n = 0; n < n_iter && ok; ++n) {
+                    const int s = n & 1;
+                    const uint32_t sQ = smem_u32(sm.q[s]);
+                    // dP^T = V_j dO_i^T - delta_i   (its columns held the previous dQ partial until the
+                    //                                reduce warps drained it)
+                    if (!(ok = LT_WAIT(&sm.bar_do_full, n & 1, kWaitDoFull))) break;
+                    if (n > 0 && !(ok = LT_WAIT(&sm.bar_dq_empty, (n - 1) & 1, kWaitDqEmpty))) break;
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint32_t koff = (kk >> 2) * kBoxBytesBwd + (kk & 3) * 32;
+                        umma_ss(tmem + kColdP, desc_kmajor(sV + koff), desc_kmajor(sdO + koff), idesc_s, kk > 0);
+                    }
+                    umma_ss(tmem + kColdP, desc_ones, desc_ext_do, idesc_s, 1);
+                    umma_commit(&sm.bar_dp_full);
+                    // dV_j += P'^T dO_i   (A = P'^T from tensor memory; query columns 0-63 sit at columns
+                    //                      0-31, query columns 64-127 at columns 64-95 of the S region)
+                    if (!(ok = LT_WAIT(&sm.bar_p_ready, n & 1, kWaitPReady))) break;
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk)
+                        umma_ts(tmem + kColdV, tmem + kColS + (kk >> 2) * 64 + (kk & 3) * 8,
+                                desc_mnmajor(sdO + kk * 2048, kBoxBytesBwd), idesc_dv, (n > 0) | (kk > 0));
+                    umma_commit(&sm.bar_do_empty);
+                    // the next S^T overwrites P'^T; the tensor pipe executes in issue order
+                    if (n + 1 < n_iter) {
+                        if (!(ok = LT_WAIT(&sm.bar_q_full[(n + 1) & 1], ((n + 1) >> 1) & 1, kWaitStageFull))) break;
+                        issue_s(n + 1);
+                    }
+                    if (!(ok = LT_WAIT(&sm.bar_ds_ready, n & 1, kWaitDsReady))) break;
+                    tc_fence_after_sync();
+                    // dQ_i partial (contraction over key rows; lands on the dP columns).  For D = 128 it is
+                    // produced transposed, dQ^T = K_j^T dS^T (lanes = head dim, columns = query rows), so
+                    // that a warp of the reduction adds 128 contiguous bytes; for D = 64 as dQ = dS K_j.
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {
+                        if constexpr (D == 128)
+                            umma_ss(tmem + kColdP, desc_mnmajor(sK + kk * 2048, kBoxBytesBwd),
+                                    desc_mnmajor(sdS + kk * 2048, kBoxBytesBwd), idesc_dq, kk > 0);
+                        else
+                            umma_ss(tmem + kColdP, desc_mnmajor(sdS + kk * 2048, kBoxBytesBwd),
+                                    desc_mnmajor(sK + kk * 2048, kBoxBytesBwd), idesc_dq, kk > 0);
+                    }
+                    umma_commit(&sm.bar_dq_full);
+                    // dK_j += dS^T Q_i
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {
+                        const uint32_t koff = (kk >> 2) * kBoxBytesBwd + (kk & 3) * 32;
+                        umma_ss(tmem + kColdK, desc_kmajor(sdS + koff), desc_mnmajor(sQ + kk * 2048, kBoxBytesBwd),
+                                idesc_dv, (n > 0) | (kk > 0));
+                    }
+                    umma_commit(&sm.bar_q_empty[s]);
+                    umma_commit(&sm.bar_ds_free);
+                }
+                if (ok) umma_commit(&sm.bar_dkv_full);
+                LT_TRACE_END(kRoleMma);
             }
+            __syncwarp();
         }
-        __syncwarp();
-    } else if (warp == 1) {
-        // ================================================================= tensor-core issuer
-        if (lane == 0 && smem_ok) {
-            const uint32_t sK = smem_u32(sm.k), sV = smem_u32(sm.v), sdS = smem_u32(sm.ds);
-            constexpr uint32_t idesc_s = make_idesc(128, 128, false, false);
-            constexpr uint32_t idesc_dv = make_idesc(128, D, false, true);
-            constexpr uint32_t idesc_dq = make_idesc(128, D, true, true);
-            auto issue_s = [&](int n) {  // S^T = K_j Q_i^T
-                const uint32_t sQn = smem_u32(sm.q[n & 1]);
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t koff = (kk >> 2) * kBoxBytesBwd + (kk & 3) * 32;
-                    umma_ss(tmem + kColS, desc_kmajor(sK + koff), desc_kmajor(sQn + koff), idesc_s, kk > 0);
-                }
-                umma_commit(&sm.bar_s_full);
-            };
-            bool ok = mbar_wait(&sm.bar_kv, 0, abort_flag, p.status, kWaitKV) &&
-                      mbar_wait(&sm.bar_stage_full[0], 0, abort_flag, p.status, kWaitStageFull);
-            if (ok) {
-                tc_fence_after_sync();
-                issue_s(0);
-            }
-            for (int n = 0; n < n_iter && ok; ++n) {
-                const int s = n & 1;
-                const uint32_t sQ = smem_u32(sm.q[s]), sdO = smem_u32(sm.d_o[s]);
-                // dP^T = V_j dO_i^T   (its columns held the previous dQ partial until the reduce warps drained it)
-                if (n > 0 && !(ok = mbar_wait(&sm.bar_dq_empty, (n - 1) & 1, abort_flag, p.status, kWaitDqEmpty))) break;
-                tc_fence_after_sync();
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t koff = (kk >> 2) * kBoxBytesBwd + (kk & 3) * 32;
-                    umma_ss(tmem + kColdP, desc_kmajor(sV + koff), desc_kmajor(sdO + koff), idesc_s, kk > 0);
-                }
-                umma_commit(&sm.bar_dp_full);
-                // dV_j += P^T dO_i   (A = P^T from tensor memory; query columns 0-63 sit at columns 0-31,
-                //                     query columns 64-127 at columns 64-95 of the S region)
-                if (!(ok = mbar_wait(&sm.bar_p_ready, n & 1, abort_flag, p.status, kWaitPReady))) break;
-                tc_fence_after_sync();
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
-                    umma_ts(tmem + kColdV, tmem + kColS + (kk >> 2) * 64 + (kk & 3) * 8,
-                            desc_mnmajor(sdO + kk * 2048, kBoxBytesBwd), idesc_dv, (n > 0) | (kk > 0));
-                // the next S^T overwrites P^T; the tensor pipe executes in issue order
-                if (n + 1 < n_iter) {
-                    if (!(ok = mbar_wait(&sm.bar_stage_full[(n + 1) & 1], ((n + 1) >> 1) & 1, abort_flag, p.status,
-                                         kWaitStageFull)))
-                        break;
-                    issue_s(n + 1);
-                }
-                if (!(ok = mbar_wait(&sm.bar_ds_ready, n & 1, abort_flag, p.status, kWaitDsReady))) break;
-                tc_fence_after_sync();
-                // dQ_i partial = dS K_j   (contraction over key rows; lands on the dP columns)
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
-                    umma_ss(tmem + kColdP, desc_mnmajor(sdS + kk * 2048, kBoxBytesBwd),
-                            desc_mnmajor(sK + kk * 2048, kBoxBytesBwd), idesc_dq, kk > 0);
-                umma_commit(&sm.bar_dq_full);
-                // dK_j += dS^T Q_i
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t koff = (kk >> 2) * kBoxBytesBwd + (kk & 3) * 32;
-                    umma_ss(tmem + kColdK, desc_kmajor(sdS + koff), desc_mnmajor(sQ + kk * 2048, kBoxBytesBwd),
-                            idesc_dv, (n > 0) | (kk > 0));
-                }
-                umma_commit(&sm.bar_stage_empty[s]);
-                umma_commit(&sm.bar_ds_free);
-            }
-            if (ok) umma_commit(&sm.bar_dkv_full);
-        }
-        __syncwarp();
-    } else if (warp >= kComputeWarp0 && warp < kComputeWarp0 + kNumComputeWarps) {
+    } else if (warp < kReduceWarp0) {
         // ================================================================= softmax / dS warps
         const int quad = warp & 3;                           // tensor-memory lane quadrant
         const int half_sel = (warp - kComputeWarp0) >> 2;    // 0: query columns 0-63, 1: 64-127
@@ -388,14 +480,14 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const uint32_t cbase = half_sel * 64;
         const float scale_log2 = p.scale * kLog2e;
         uint8_t *ds_tile = sm.ds + half_sel * kBoxBytesBwd;
-        uint32_t pp[32];  // this thread's 64 P^T values of the current tile pair, packed fp16 pairs
+        uint32_t pv[64];  // bits of this thread's 64 fp32 values of P' = P * 2^c for the current tile pair
         bool ok = smem_ok;
+        LT_TRACE_BEGIN();
 
         auto compute_p = [&](int n) -> bool {
-            const int s = n & 1;
-            if (!mbar_wait(&sm.bar_stage_full[s], (n >> 1) & 1, abort_flag, p.status, kWaitStageFull)) return false;
-            if (!mbar_wait(&sm.bar_s_full, n & 1, abort_flag, p.status, kWaitSFull)) return false;
+            if (!LT_WAIT(&sm.bar_s_full, n & 1, kWaitSFull)) return false;
             tc_fence_after_sync();
+            LT_TRACE_MARK(tp0);
             const int hh = n / tiles_per_head;
             const bool diag = p.causal && (i_first + (n - hh * tiles_per_head) == j);
 #pragma unroll
@@ -403,79 +495,72 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 uint32_t sv[32];
                 tmem_ld32(tmem + lane_base + kColS + cbase + c * 32, sv);
                 tmem_wait_ld();
+                // P' = exp2(scale*log2e * (K.Q - LSE/scale) + c)
 #pragma unroll
-                for (int e = 0; e < 32; e += 4) {
-                    const int q0 = cbase + c * 32 + e;
-                    const float4 nl = *reinterpret_cast<const float4 *>(&sm.neg_lse_log2[s][q0]);
-                    float p0 = fast_exp2(fmaf(__uint_as_float(sv[e]), scale_log2, nl.x));
-                    float p1 = fast_exp2(fmaf(__uint_as_float(sv[e + 1]), scale_log2, nl.y));
-                    float p2 = fast_exp2(fmaf(__uint_as_float(sv[e + 2]), scale_log2, nl.z));
-                    float p3 = fast_exp2(fmaf(__uint_as_float(sv[e + 3]), scale_log2, nl.w));
-                    if (diag) {  // key row is hidden from query column q when row > q
-                        if (row > q0) p0 = 0.f;
-                        if (row > q0 + 1) p1 = 0.f;
-                        if (row > q0 + 2) p2 = 0.f;
-                        if (row > q0 + 3) p3 = 0.f;
-                    }
-                    pp[c * 16 + e / 2] = pack_half2(p0, p1);
-                    pp[c * 16 + e / 2 + 1] = pack_half2(p2, p3);
-                }
+                for (int e = 0; e < 32; ++e)
+                    pv[c * 32 + e] = __float_as_uint(fast_exp2(fmaf(__uint_as_float(sv[e]), scale_log2, p_scale_log2)));
+            }
+            if (diag) {  // key row is hidden from query column q when row > q
+#pragma unroll
+                for (int e = 0; e < 64; ++e)
+                    if (row > static_cast<int>(cbase) + e) pv[e] = 0u;
+            }
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
                 uint32_t out[16];
 #pragma unroll
-                for (int e = 0; e < 16; ++e) out[e] = pp[c * 16 + e];
-                // in place: these 16 columns were read by this thread in this or the previous chunk
+                for (int e = 0; e < 16; ++e)
+                    out[e] = pack_half2(__uint_as_float(pv[c * 32 + 2 * e]), __uint_as_float(pv[c * 32 + 2 * e + 1]));
+                // in place: these columns lie inside the 64 columns this thread has just read
                 tmem_st16(tmem + lane_base + kColS + cbase + c * 16, out);
             }
             tmem_wait_st();
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.bar_p_ready);
+            LT_TRACE_SINCE(12, tp0);
             return true;
         };
 
         ok = ok && compute_p(0);
         for (int n = 0; n < n_iter && ok; ++n) {
-            const int s = n & 1;
-            if (!(ok = mbar_wait(&sm.bar_dp_full, n & 1, abort_flag, p.status, kWaitDpFull))) break;
+            if (!(ok = LT_WAIT(&sm.bar_dp_full, n & 1, kWaitDpFull))) break;
             tc_fence_after_sync();
-            uint32_t o[32];
+            // the previous dS^T tile must have been consumed by dQ and dK before it is overwritten
+            if (n > 0 && !(ok = LT_WAIT(&sm.bar_ds_free, (n - 1) & 1, kWaitDsFree))) break;
+            LT_TRACE_MARK(td0);
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
                 uint32_t dp[32];
                 tmem_ld32(tmem + lane_base + kColdP + cbase + c * 32, dp);
                 tmem_wait_ld();
+                // dS' = P' * (dP - delta); the subtraction happened inside the tensor-core product.
+                // 32 query columns = four 16-byte chunks of row `row` in this half's tile.
 #pragma unroll
-                for (int e = 0; e < 32; e += 4) {
-                    const int q0 = cbase + c * 32 + e;
-                    const float4 dl = *reinterpret_cast<const float4 *>(&sm.delta[s][q0]);
-                    const float2 pa = __half22float2(*reinterpret_cast<const __half2 *>(&pp[c * 16 + e / 2]));
-                    const float2 pb = __half22float2(*reinterpret_cast<const __half2 *>(&pp[c * 16 + e / 2 + 1]));
-                    const float d0 = pa.x * ds_mult * (__uint_as_float(dp[e]) - dl.x);
-                    const float d1 = pa.y * ds_mult * (__uint_as_float(dp[e + 1]) - dl.y);
-                    const float d2 = pb.x * ds_mult * (__uint_as_float(dp[e + 2]) - dl.z);
-                    const float d3 = pb.y * ds_mult * (__uint_as_float(dp[e + 3]) - dl.w);
-                    o[c * 16 + e / 2] = pack_half2(d0, d1);
-                    o[c * 16 + e / 2 + 1] = pack_half2(d2, d3);
+                for (int v4 = 0; v4 < 4; ++v4) {
+                    uint4 w;
+                    const int e = c * 32 + v4 * 8;
+                    w.x = pack_half2(__uint_as_float(pv[e + 0]) * __uint_as_float(dp[v4 * 8 + 0]), __uint_as_float(pv[e + 1]) * __uint_as_float(dp[v4 * 8 + 1]));
+                    w.y = pack_half2(__uint_as_float(pv[e + 2]) * __uint_as_float(dp[v4 * 8 + 2]), __uint_as_float(pv[e + 3]) * __uint_as_float(dp[v4 * 8 + 3]));
+                    w.z = pack_half2(__uint_as_float(pv[e + 4]) * __uint_as_float(dp[v4 * 8 + 4]), __uint_as_float(pv[e + 5]) * __uint_as_float(dp[v4 * 8 + 5]));
+                    w.w = pack_half2(__uint_as_float(pv[e + 6]) * __uint_as_float(dp[v4 * 8 + 6]), __uint_as_float(pv[e + 7]) * __uint_as_float(dp[v4 * 8 + 7]));
+                    *reinterpret_cast<uint4 *>(ds_tile + swz128_offset(row, c * 32 + v4 * 8)) = w;
                 }
             }
-            // the previous dS^T tile must have been consumed by dQ and dK before it is overwritten
-            if (n > 0 && !(ok = mbar_wait(&sm.bar_ds_free, (n - 1) & 1, abort_flag, p.status, kWaitDsFree))) break;
-            // 64 query columns = eight 16-byte chunks of row `row` in this half's tile
-#pragma unroll
-            for (int v4 = 0; v4 < 8; ++v4)
-                *reinterpret_cast<uint4 *>(ds_tile + swz128_offset(row, v4 * 8)) =
-                    make_uint4(o[4 * v4], o[4 * v4 + 1], o[4 * v4 + 2], o[4 * v4 + 3]);
+            LT_TRACE_SINCE(13, td0);
             fence_proxy_async_smem();
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.bar_ds_ready);
+            LT_TRACE_SINCE(14, td0);
             if (n + 1 < n_iter) ok = compute_p(n + 1);
         }
+        LT_TRACE_END(kRoleCompute);
 
-        // epilogue: warps 4-7 write dK_j, warps 8-11 write dV_j; thread = key row
+        // epilogue: the first four softmax warps write dK_j, the other four dV_j; thread = key row
         if (ok && mbar_wait(&sm.bar_dkv_full, 0, abort_flag, p.status, kWaitDkvFull)) {
             tc_fence_after_sync();
-            const float mult = half_sel == 0 ? dq_mult : 1.f;
+            const float mult = half_sel == 0 ? dq_mult : inv_p_scale;
             const uint32_t col0 = half_sel == 0 ? kColdK : kColdV;
             __half *dst = (half_sel == 0 ? p.dK : p.dV) + (static_cast<long long>(kv_row0) + row) * D;
 #pragma unroll
@@ -494,49 +579,99 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 }
             }
         }
-    } else if (warp >= kReduceWarp0) {
+    } else {
         // ================================================================= dQ reduction warps
         const int quad = warp & 3;
         bool ok = smem_ok;
+        LT_TRACE_BEGIN();
         for (int n = 0; n < n_iter && ok; ++n) {
-            if (!(ok = mbar_wait(&sm.bar_dq_full, n & 1, abort_flag, p.status, kWaitDqFull))) break;
+            if (!(ok = LT_WAIT(&sm.bar_dq_full, n & 1, kWaitDqFull))) break;
             tc_fence_after_sync();
+            LT_TRACE_MARK(tr0);
             float *dq_tile = p.dq_acc + q_row_of(n) * D;
+            if constexpr (D == 128) {
+                // dQ^T: this thread holds head-dim element d = 32*quad + lane of all 128 query rows;
+                // one warp instruction adds 32 consecutive floats of one accumulator row
+                float *col = dq_tile + quad * 32 + lane;
 #pragma unroll
-            for (int ch = 0; ch < D / 64; ++ch) {
-                uint32_t r[2][32];
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(tmem + (static_cast<uint32_t>(quad * 32) << 16) + kColdP + c * 32, r);
+                    tmem_wait_ld();
+                    if (c == 3) {
+                        // the whole partial has been read: the dP columns may be overwritten
+                        tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&sm.bar_dq_empty);
+                        LT_TRACE_SINCE(12, tr0);
+                    }
 #pragma unroll
-                for (int lh = 0; lh < 2; ++lh)
-                    tmem_ld_16x256b_x8(tmem + (static_cast<uint32_t>(quad * 32 + lh * 16) << 16) + kColdP + ch * 64,
-                                       r[lh]);
-                tmem_wait_ld();
-                if (ch == D / 64 - 1) {
-                    // the whole partial is in registers: the dP columns may be overwritten
-                    tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&sm.bar_dq_empty);
+                    for (int e = 0; e < 32; ++e)
+                        atomicAdd(col + static_cast<long long>(c * 32 + e) * D, __uint_as_float(r[e]) * dq_mult);
                 }
-                // four neighbouring threads add 32 contiguous bytes of one query row
+            } else {
 #pragma unroll
-                for (int lh = 0; lh < 2; ++lh) {
-                    float *base = dq_tile + static_cast<long long>(quad * 32 + lh * 16 + (lane >> 2)) * D + ch * 64 +
-                                  2 * (lane & 3);
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        red_add_v2(base + 8 * k, __uint_as_float(r[lh][4 * k]) * dq_mult,
-                                   __uint_as_float(r[lh][4 * k + 1]) * dq_mult);
-                        red_add_v2(base + 8 * D + 8 * k, __uint_as_float(r[lh][4 * k + 2]) * dq_mult,
-                                   __uint_as_float(r[lh][4 * k + 3]) * dq_mult);
+                for (int ch = 0; ch < D / 64; ++ch) {
+                    uint32_t r[2][32];
+    #pragma unroll
+                    for (int lh = 0; lh < 2; ++lh)
+                        tmem_ld_16x256b_x8(tmem + (static_cast<uint32_t>(quad * 32 + lh * 16) << 16) + kColdP + ch * 64,
+                                           r[lh]);
+                    tmem_wait_ld();
+                    if (ch == D / 64 - 1) {
+                        // the whole partial is in registers: the dP columns may be overwritten
+                        tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&sm.bar_dq_empty);
+                        LT_TRACE_SINCE(12, tr0);
+                    }
+                    // four neighbouring threads add 32 contiguous bytes of one query row
+    #pragma unroll
+                    for (int lh = 0; lh < 2; ++lh) {
+                        float *base = dq_tile + static_cast<long long>(quad * 32 + lh * 16 + (lane >> 2)) * D + ch * 64 +
+                                      2 * (lane & 3);
+    #pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            red_add_v2(base + 8 * k, __uint_as_float(r[lh][4 * k]) * dq_mult,
+                                       __uint_as_float(r[lh][4 * k + 1]) * dq_mult);
+                            red_add_v2(base + 8 * D + 8 * k, __uint_as_float(r[lh][4 * k + 2]) * dq_mult,
+                                       __uint_as_float(r[lh][4 * k + 3]) * dq_mult);
+                        }
                     }
                 }
             }
+            LT_TRACE_SINCE(13, tr0);
         }
+        LT_TRACE_END(kRoleReduce);
     }
 
+#ifdef LT_BWD_TRACE
+    const long long trace_teardown_begin = clock64();
+#endif
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 2) tmem_dealloc(tmem, kTmemCols);
+    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+#ifdef LT_BWD_TRACE
+    if (tid == 0) {
+        atomicAdd(&g_bwd_trace[64 + 3], static_cast<unsigned long long>(clock64() - trace_cta_t0));
+        atomicAdd(&g_bwd_trace[64 + 2], static_cast<unsigned long long>(n_iter));
+        atomicAdd(&g_bwd_trace[64 + 1], 1ull);
+        atomicAdd(&g_bwd_trace[64 + 0], static_cast<unsigned long long>(trace_prologue_end - trace_cta_t0));
+        atomicAdd(&g_bwd_trace[64 + 4], static_cast<unsigned long long>(trace_teardown_begin - trace_prologue_end));
+    }
+#endif
 }
+
+#ifdef LT_BWD_TRACE
+extern "C" int lt_dbg_bwd_trace(unsigned long long *out, int reset) {
+    if (out && cudaMemcpyFromSymbol(out, g_bwd_trace, sizeof(g_bwd_trace)) != cudaSuccess) return LT_ERR_CUDA;
+    if (reset) {
+        static unsigned long long zeros[80];
+        if (cudaMemcpyToSymbol(g_bwd_trace, zeros, sizeof(zeros)) != cudaSuccess) return LT_ERR_CUDA;
+    }
+    return LT_OK;
+}
+#endif
 
 template <int D>
 static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, const lt_half *O, const lt_half *dO,
@@ -546,10 +681,10 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
     const long long n_rows = static_cast<long long>(B) * Hq * S;
     uint8_t *ws = static_cast<uint8_t *>(workspace);
     unsigned int *status = reinterpret_cast<unsigned int *>(ws);
-    const size_t row_bytes = round256(static_cast<size_t>(n_rows) * 4);
-    float *delta = reinterpret_cast<float *>(ws + kStatusBytes);
-    float *neg_lse_log2 = reinterpret_cast<float *>(ws + kStatusBytes + row_bytes);
-    float *dq_acc = reinterpret_cast<float *>(ws + kStatusBytes + 2 * row_bytes);
+    const size_t ext_bytes = round256(static_cast<size_t>(n_rows) * 16);
+    uint4 *delta_ext = reinterpret_cast<uint4 *>(ws + kStatusBytes);
+    uint4 *lse_ext = reinterpret_cast<uint4 *>(ws + kStatusBytes + ext_bytes);
+    float *dq_acc = reinterpret_cast<float *>(ws + kStatusBytes + 2 * ext_bytes);
 
     CUtensorMap mq, mk, mv, mdo;
     int rc;
@@ -571,14 +706,14 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
     const long long want = (n_rows + kRowsPerBlock - 1) / kRowsPerBlock;
     const int pre_blocks = static_cast<int>(want < static_cast<long long>(sms) * 16 ? want : sms * 16);
     bwd_preprocess_kernel<D><<<pre_blocks, 256, 0, stream>>>(reinterpret_cast<const __half *>(dO),
-                                                             reinterpret_cast<const __half *>(O), LSE, delta,
-                                                             neg_lse_log2, dq_acc, n_rows, status);
+                                                             reinterpret_cast<const __half *>(O), LSE, delta_ext,
+                                                             lse_ext, dq_acc, n_rows, 1.f / scale, status);
     e = cudaGetLastError();
     if (e != cudaSuccess) return record_cuda_error("bwd_preprocess_kernel launch", e);
 
     BwdParams prm;
-    prm.neg_lse_log2 = neg_lse_log2;
-    prm.delta = delta;
+    prm.lse_ext = lse_ext;
+    prm.delta_ext = delta_ext;
     prm.dq_acc = dq_acc;
     prm.dK = reinterpret_cast<__half *>(dK);
     prm.dV = reinterpret_cast<__half *>(dV);
@@ -613,7 +748,7 @@ extern "C" {
 size_t lt_attn_bwd_workspace_bytes(int B, int Hq, int Hkv, int S, int D) {
     if (lt::check_shape(B, Hq, Hkv, S, D, 1.0f) != LT_OK) return 0;
     const size_t n_rows = static_cast<size_t>(B) * Hq * S;
-    return lt::kStatusBytes + 2 * lt::round256(n_rows * 4) + lt::round256(n_rows * D * 4);
+    return lt::kStatusBytes + 2 * lt::round256(n_rows * 16) + lt::round256(n_rows * D * 4);
 }
 
 int lt_attn_bwd_num_launches(void) { return 3; }

@@ -154,6 +154,23 @@ __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t smem_addr, uint32_t mn
            (static_cast<uint64_t>(1024 >> 4) << 32) | static_cast<uint64_t>((smem_addr & 0x3FFFF) >> 4);
 }
 
+// Unswizzled contraction-contiguous operand for one 16-element contraction step: rows of
+// 16 bytes (8 fp16) grouped in blocks of 8 rows (128 contiguous bytes); `sbo` bytes between
+// 8-row blocks, `lbo` bytes from the block holding elements 0-7 to the one holding 8-15.
+__device__ __forceinline__ uint64_t desc_kmajor_noswz(uint32_t smem_addr, uint32_t lbo, uint32_t sbo) {
+    return (1ull << 46) | (static_cast<uint64_t>((lbo >> 4) & 0x3FFF) << 16) |
+           (static_cast<uint64_t>((sbo >> 4) & 0x3FFF) << 32) | static_cast<uint64_t>((smem_addr & 0x3FFFF) >> 4);
+}
+
+// x = 256 * hi + lo with both parts fp16: about 22 significant bits and a range of 1.6e7.
+// Used to add a per-row fp32 value inside a tensor-core product: one extra contraction step
+// whose other operand holds (256, 1, 0, ..., 0).
+__device__ __forceinline__ uint32_t split_hi_lo(float x) {
+    const __half hi = __float2half_rn(x * (1.f / 256.f));
+    const __half lo = __float2half_rn(x - 256.f * __half2float(hi));
+    return static_cast<uint32_t>(__half_as_ushort(hi)) | (static_cast<uint32_t>(__half_as_ushort(lo)) << 16);
+}
+
 // Instruction descriptor, kind::f16: fp16 A and B, fp32 accumulator, dense.
 constexpr uint32_t make_idesc(int M, int N, bool a_mn_major, bool b_mn_major) {
     return (1u << 4)                                   // accumulator format: f32
@@ -261,6 +278,10 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 __device__ __forceinline__ void red_add_v2(float *addr, float a, float b) {
+#ifdef LT_EXP_NO_RED
+    if (a == 1234.5f) asm volatile("red.global.add.v2.f32 [%0], {%1, %2};" ::"l"(addr), "f"(a), "f"(b) : "memory");
+    return;
+#endif
     asm volatile("red.global.add.v2.f32 [%0], {%1, %2};" ::"l"(addr), "f"(a), "f"(b) : "memory");
 }
 __device__ __forceinline__ void red_add_v4(float *addr, float a, float b, float c, float d) {

@@ -11,6 +11,9 @@ constexpr int kBoxBytes = 128 * 128;  // one swizzled tile: 128 rows x 64 fp16
 struct __align__(1024) DbgSmem {
     uint8_t a[2 * kBoxBytes];
     uint8_t b[2 * kBoxBytes];
+    uint8_t ext_a[2048];     // rows of (256, 1, 0, ..., 0)
+    uint8_t ext_b[2048];     // rows of (hi, lo, 0, ..., 0)
+    uint8_t ext_zero[2048];  // elements 8-15 of both
     uint64_t bar_load;
     uint64_t bar_mma;
     uint32_t tmem_base;
@@ -19,7 +22,8 @@ struct __align__(1024) DbgSmem {
 
 __global__ void __launch_bounds__(128, 1)
 dbg_tile_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                     const __half *__restrict__ a_gmem, float *__restrict__ c_gmem, int mode,
+                     const __half *__restrict__ a_gmem, const __half *__restrict__ b_gmem,
+                     float *__restrict__ c_gmem, int mode,
                      unsigned int *status) {
     extern __shared__ uint8_t smem_raw[];
     DbgSmem &sm = *reinterpret_cast<DbgSmem *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -67,6 +71,15 @@ dbg_tile_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         }
         tmem_wait_st();
     }
+    if (mode == 5) {
+        // thread n owns row n of the two extra-step operands: adds x_n = 1000 * B[n][0] to column n
+        const float x = 1000.f * __half2float(reinterpret_cast<const __half *>(b_gmem)[static_cast<size_t>(tid) * kTile]);
+        const __half2 ones = __halves2half2(__float2half_rn(256.f), __float2half_rn(1.f));
+        reinterpret_cast<uint4 *>(sm.ext_a)[tid] = make_uint4(*reinterpret_cast<const uint32_t *>(&ones), 0u, 0u, 0u);
+        reinterpret_cast<uint4 *>(sm.ext_b)[tid] = make_uint4(split_hi_lo(x), 0u, 0u, 0u);
+        reinterpret_cast<uint4 *>(sm.ext_zero)[tid] = make_uint4(0u, 0u, 0u, 0u);
+        fence_proxy_async_smem();
+    }
     tc_fence_before_sync();
     __syncthreads();
 
@@ -79,7 +92,7 @@ dbg_tile_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             const uint32_t koff = (kk >> 2) * kBoxBytes + (kk & 3) * 32;  // contraction-contiguous operand
             const uint32_t roff = kk * 16 * 128;                          // contraction index = row
             const uint32_t acc = kk > 0;
-            if (mode == 0 || mode == 4) {
+            if (mode == 0 || mode == 4 || mode == 5) {
                 umma_ss(tmem, desc_kmajor(a0 + koff), desc_kmajor(b0 + koff), make_idesc(128, 128, false, false), acc);
             } else if (mode == 1) {
                 umma_ss(tmem, desc_kmajor(a0 + koff), desc_mnmajor(b0 + roff, kBoxBytes),
@@ -92,10 +105,34 @@ dbg_tile_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                         make_idesc(128, 128, false, true), acc);
             }
         }
+        if (mode == 5) {
+            const uint32_t ea = smem_u32(sm.ext_a), eb = smem_u32(sm.ext_b), ez = smem_u32(sm.ext_zero);
+            umma_ss(tmem, desc_kmajor_noswz(ea, ez - ea, 128), desc_kmajor_noswz(eb, ez - eb, 128),
+                    make_idesc(128, 128, false, false), 1);
+        }
         umma_commit(&sm.bar_mma);
     }
     ok = ok && mbar_wait(&sm.bar_mma, 0, &sm.abort_flag, status, 102);
     tc_fence_after_sync();
+    // development aid: cycles for this thread to pull the 128 accumulator columns into registers
+    if (ok) {
+        const long long t0 = clock64();
+        float acc = 0.f;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            uint32_t r[32];
+            if (mode == 4) tmem_ld_16x256b_x8(tmem + (static_cast<uint32_t>(warp * 32 + (c & 1) * 16) << 16) + (c >> 1) * 64, r);
+            else tmem_ld32(tmem + lane_base + c * 32, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) acc += __uint_as_float(r[e]);
+        }
+        const long long t1 = clock64();
+        if (tid == 0) {
+            status[8] = static_cast<unsigned int>(t1 - t0);
+            status[9] = __float_as_uint(acc);
+        }
+    }
     if (ok && mode == 4) {
         // read the accumulator back in the 16-lane x 256-bit arrangement the dQ reduction uses
         const int lane = tid & 31;
@@ -140,7 +177,7 @@ dbg_tile_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
 extern "C" int lt_dbg_tile_gemm(const lt_half *A, const lt_half *B, float *C, int mode, void *workspace,
                                 size_t workspace_bytes, lt_stream_t stream) {
     using namespace lt;
-    if (!A || !B || !C || mode < 0 || mode > 4) return LT_ERR_INVALID_ARG;
+    if (!A || !B || !C || mode < 0 || mode > 5) return LT_ERR_INVALID_ARG;
     if (!aligned16(A) || !aligned16(B) || !aligned16(C)) return LT_ERR_UNSUPPORTED;
     if (!workspace || !aligned256(workspace) || workspace_bytes < static_cast<size_t>(kStatusBytes))
         return LT_ERR_WORKSPACE;
@@ -154,7 +191,8 @@ extern "C" int lt_dbg_tile_gemm(const lt_half *A, const lt_half *B, float *C, in
     const size_t smem = sizeof(DbgSmem) + 1024;
     e = cudaFuncSetAttribute(dbg_tile_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return record_cuda_error("cudaFuncSetAttribute", e);
-    dbg_tile_gemm_kernel<<<1, 128, smem, stream>>>(ma, mb, reinterpret_cast<const __half *>(A), C, mode,
+    dbg_tile_gemm_kernel<<<1, 128, smem, stream>>>(ma, mb, reinterpret_cast<const __half *>(A),
+                                                   reinterpret_cast<const __half *>(B), C, mode,
                                                    reinterpret_cast<unsigned int *>(workspace));
     e = cudaGetLastError();
     if (e != cudaSuccess) return record_cuda_error("dbg_tile_gemm_kernel launch", e);

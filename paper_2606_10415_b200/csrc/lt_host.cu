@@ -36,7 +36,7 @@ int check_device() {
 int check_shape(int B, int Hq, int Hkv, int S, int D, float scale) {
     if (B <= 0 || Hq <= 0 || Hkv <= 0 || S <= 0 || D <= 0) return LT_ERR_INVALID_ARG;
     if (Hq % Hkv != 0) return LT_ERR_INVALID_ARG;
-    if (!isfinite(scale)) return LT_ERR_INVALID_ARG;
+    if (!isfinite(scale) || scale == 0.f) return LT_ERR_INVALID_ARG;
     if (D != 64 && D != 128) return LT_ERR_UNSUPPORTED;
     if (S % 128 != 0) return LT_ERR_UNSUPPORTED;
     // row indices of the [B*H*S, D] tensor views must fit a 32-bit TMA coordinate

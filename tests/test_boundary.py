@@ -38,9 +38,9 @@ def test_library_exports_every_declared_symbol(binding):
 
 
 def test_workspace_sizes(binding):
-    # 256-byte status block + delta and -LSE*log2e fp32 [B,Hq,S] each + dQ accumulator fp32 [B,Hq,S,D]
-    assert binding.lt_attn_bwd_workspace_bytes(1, 2, 2, 128, 64) == 256 + 2 * 1024 + 65536
-    assert binding.lt_attn_bwd_workspace_bytes(1, 32, 32, 4096, 128) == 256 + 2 * 524288 + 67108864
+    # 256-byte status block + two [B,Hq,S] arrays of 16-byte rows + dQ accumulator fp32 [B,Hq,S,D]
+    assert binding.lt_attn_bwd_workspace_bytes(1, 2, 2, 128, 64) == 256 + 2 * 4096 + 65536
+    assert binding.lt_attn_bwd_workspace_bytes(1, 32, 32, 4096, 128) == 256 + 2 * 2097152 + 67108864
     assert binding.lt_attn_fwd_workspace_bytes(1, 2, 2, 128, 64) == 256
     # unsupported shapes report 0
     assert binding.lt_attn_bwd_workspace_bytes(1, 2, 2, 100, 64) == 0
@@ -67,6 +67,7 @@ def test_bwd_rejects_bad_arguments_without_launching(binding):
     assert b.lt_attn_bwd_raw(*_bwd_args(B=0)) == b.LT_ERR_INVALID_ARG
     assert b.lt_attn_bwd_raw(*_bwd_args(Hq=3, Hkv=2)) == b.LT_ERR_INVALID_ARG
     assert b.lt_attn_bwd_raw(*_bwd_args(scale=float("nan"))) == b.LT_ERR_INVALID_ARG
+    assert b.lt_attn_bwd_raw(*_bwd_args(scale=0.0)) == b.LT_ERR_INVALID_ARG
     assert b.lt_attn_bwd_raw(*_bwd_args(S=100)) == b.LT_ERR_UNSUPPORTED
     assert b.lt_attn_bwd_raw(*_bwd_args(D=96)) == b.LT_ERR_UNSUPPORTED
     assert b.lt_attn_bwd_raw(*_bwd_args(ptr=0x1004)) == b.LT_ERR_UNSUPPORTED  # misaligned
