@@ -170,6 +170,7 @@ constexpr int kQStages = 2;   // Q_i ring; dO_i is single-buffered (it is dead o
 constexpr int kBwdThreads = 448;  // 14 warps: 65536 / 448 leaves 144 registers per thread
 constexpr int kComputeWarp0 = 2, kNumComputeWarps = 8;
 constexpr int kReduceWarp0 = 10, kNumReduceWarps = 4;
+constexpr int kDqStageBufs = 3, kDqStageRows = 16;
 constexpr int kExtBytes = 2048;            // 128 rows x 16 bytes: one operand of the extra contraction step
 constexpr float kPScaleLog2Max = 14.f;     // P is kept as P * 2^c with c <= 14 so that fp16(P') <= 16384
 
@@ -187,6 +188,9 @@ struct BwdSmem {
     uint8_t ext_q[kQStages][kExtBytes];// rows (hi, lo, 0...) of -LSE/scale for the stage's query tile
     uint8_t ext_do[kExtBytes];         // rows (hi, lo, 0...) of -delta
     uint8_t ext_zero[kExtBytes];       // contraction elements 8-15 of all of the above
+    // staging of the dQ partial for bulk reduction into global memory (D = 128 only):
+    // each buffer holds 16 accumulator rows (16 query rows x 128 floats)
+    float dq_stage[D == 128 ? kDqStageBufs : 1][D == 128 ? kDqStageRows * 128 : 4];
     uint64_t bar_kv;
     uint64_t bar_q_full[kQStages], bar_q_empty[kQStages], bar_do_full, bar_do_empty;
     uint64_t bar_s_full, bar_p_ready, bar_dp_full, bar_ds_ready, bar_ds_free, bar_dq_full, bar_dq_empty, bar_dkv_full;
@@ -195,6 +199,8 @@ struct BwdSmem {
     uint32_t tmem_base;
     int abort_flag;
 };
+
+static_assert(sizeof(BwdSmem<128>) <= 232448, "main kernel shared memory exceeds the 227 KB per-block limit");
 
 struct BwdParams {
     const uint4 *lse_ext;    // per query row: fp16 (hi, lo, 0 x 6) with 256*hi + lo = -LSE / scale
@@ -585,35 +591,62 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         bool ok = smem_ok;
         LT_TRACE_BEGIN();
         for (int n = 0; n < n_iter && ok; ++n) {
-            if (!(ok = LT_WAIT(&sm.bar_dq_full, n & 1, kWaitDqFull))) break;
+            ok = LT_WAIT(&sm.bar_dq_full, n & 1, kWaitDqFull);
+            // the four reduction warps share named barriers below, so they leave the loop together
+            if constexpr (D == 128) ok = named_barrier_and(1, kNumReduceWarps * 32, ok);
+            if (!ok) break;
             tc_fence_after_sync();
             LT_TRACE_MARK(tr0);
             float *dq_tile = p.dq_acc + q_row_of(n) * D;
             if constexpr (D == 128) {
                 // dQ^T: this thread holds head-dim element d = 32*quad + lane of all 128 query rows;
                 // one warp instruction adds 32 consecutive floats of one accumulator row
-                float *col = dq_tile + quad * 32 + lane;
+                // dQ^T: this thread holds head-dim element d = 32*quad + lane of all 128 query rows.
+                // Sixteen query rows at a time are scaled, staged in shared memory exactly as they lie
+                // in the accumulator (16 rows x 128 floats, contiguous) and added to it by one bulk
+                // reduction; three staging buffers keep the copies in flight.
+                const int d_idx = quad * 32 + lane;
+                const uint32_t taddr = tmem + (static_cast<uint32_t>(quad * 32) << 16) + kColdP;
+                const bool elected = (warp == kReduceWarp0) && (lane == 0);
+                auto stage_rows = [&](int k, const uint32_t *r) {  // r: 16 values, query rows 16k .. 16k+15
+                    float *buf = sm.dq_stage[(n * 8 + k) % kDqStageBufs];
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t r[32];
-                    tmem_ld32(tmem + (static_cast<uint32_t>(quad * 32) << 16) + kColdP + c * 32, r);
-                    tmem_wait_ld();
-                    if (c == 3) {
-                        // the whole partial has been read: the dP columns may be overwritten
-                        tc_fence_before_sync();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&sm.bar_dq_empty);
-                        LT_TRACE_SINCE(12, tr0);
+                    for (int e = 0; e < kDqStageRows; ++e) buf[e * 128 + d_idx] = __uint_as_float(r[e]) * dq_mult;
+                    fence_proxy_async_smem();
+                    // the buffer of the next group of rows was last read two bulk operations ago
+                    if (elected) bulk_wait_group_read<1>();
+                    named_barrier_sync(1, kNumReduceWarps * 32);
+                    if (elected) {
+                        bulk_reduce_add_f32(dq_tile + k * kDqStageRows * 128, buf, kDqStageRows * 128 * sizeof(float));
+                        bulk_commit_group();
                     }
-#pragma unroll
-                    for (int e = 0; e < 32; ++e)
-                        atomicAdd(col + static_cast<long long>(c * 32 + e) * D, __uint_as_float(r[e]) * dq_mult);
-                }
+                };
+                // three quarters of the partial are read before anything is staged, so that the dP
+                // columns are released early
+                uint32_t r0[32], r1[32], r2[32];
+                tmem_ld32(taddr, r0);
+                tmem_ld32(taddr + 32, r1);
+                tmem_ld32(taddr + 64, r2);
+                tmem_wait_ld();
+                stage_rows(0, r0);
+                stage_rows(1, r0 + 16);
+                tmem_ld32(taddr + 96, r0);
+                tmem_wait_ld();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.bar_dq_empty);
+                LT_TRACE_SINCE(12, tr0);
+                stage_rows(2, r1);
+                stage_rows(3, r1 + 16);
+                stage_rows(4, r2);
+                stage_rows(5, r2 + 16);
+                stage_rows(6, r0);
+                stage_rows(7, r0 + 16);
             } else {
 #pragma unroll
                 for (int ch = 0; ch < D / 64; ++ch) {
                     uint32_t r[2][32];
-    #pragma unroll
+#pragma unroll
                     for (int lh = 0; lh < 2; ++lh)
                         tmem_ld_16x256b_x8(tmem + (static_cast<uint32_t>(quad * 32 + lh * 16) << 16) + kColdP + ch * 64,
                                            r[lh]);
@@ -626,11 +659,11 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         LT_TRACE_SINCE(12, tr0);
                     }
                     // four neighbouring threads add 32 contiguous bytes of one query row
-    #pragma unroll
+#pragma unroll
                     for (int lh = 0; lh < 2; ++lh) {
                         float *base = dq_tile + static_cast<long long>(quad * 32 + lh * 16 + (lane >> 2)) * D + ch * 64 +
                                       2 * (lane & 3);
-    #pragma unroll
+#pragma unroll
                         for (int k = 0; k < 8; ++k) {
                             red_add_v2(base + 8 * k, __uint_as_float(r[lh][4 * k]) * dq_mult,
                                        __uint_as_float(r[lh][4 * k + 1]) * dq_mult);
@@ -642,6 +675,8 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             }
             LT_TRACE_SINCE(13, tr0);
         }
+        // shared memory must stay valid until the bulk reductions have read it
+        if constexpr (D == 128) bulk_wait_group_all();
         LT_TRACE_END(kRoleReduce);
     }
 
