@@ -22,9 +22,8 @@
 //                warps 6-9 columns 64-127; each thread owns one key row
 //   warps 10-13  dQ reduction: tensor memory -> fp32 red.global into the accumulator
 // Transposed scores are used (S^T = K Q^T, dP^T = V dO^T) so that P^T, written back to
-// tensor memory as fp16, is directly the A operand of dV += P^T dO; dS^T goes through
-// shared memory once and serves both dK += dS^T Q (contraction-contiguous A) and
-// dQ = dS K (row-contracted A).  The row terms -LSE_i/scale and -delta_i are added inside
+// tensor memory as fp16, is directly the A operand of dV += P^T dO; dS^T is written both to
+// tensor memory (A operand of dK += dS^T Q) and to shared memory (operand of the dQ product).  The row terms -LSE_i/scale and -delta_i are added inside
 // the S^T and dP^T products by one extra 16-element contraction step whose operands are
 // (256, 1, 0...) and the (hi, lo, 0...) split of the term, so the softmax warps never
 // touch LSE or delta.
@@ -449,9 +448,17 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     }
                     if (!(ok = LT_WAIT(&sm.bar_ds_ready, n & 1, kWaitDsReady))) break;
                     tc_fence_after_sync();
-                    // dQ_i partial (contraction over key rows; lands on the dP columns).  For D = 128 it is
+                    // dK_j += dS'^T Q_i   (A = dS'^T from tensor memory, stored like P'^T: query columns
+                    //                       0-63 at columns 0-31 and 64-127 at columns 64-95 of the dP region)
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk)
+                        umma_ts(tmem + kColdK, tmem + kColdP + (kk >> 2) * 64 + (kk & 3) * 8,
+                                desc_mnmajor(sQ + kk * 2048, kBoxBytesBwd), idesc_dv, (n > 0) | (kk > 0));
+                    umma_commit(&sm.bar_q_empty[s]);
+                    // dQ_i partial (contraction over key rows); it overwrites the dP columns, which is safe
+                    // after dK because the tensor pipe executes in issue order.  For D = 128 it is
                     // produced transposed, dQ^T = K_j^T dS^T (lanes = head dim, columns = query rows), so
-                    // that a warp of the reduction adds 128 contiguous bytes; for D = 64 as dQ = dS K_j.
+                    // that the reduction moves whole accumulator rows; for D = 64 as dQ = dS K_j.
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk) {
                         if constexpr (D == 128)
@@ -462,14 +469,6 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                                     desc_mnmajor(sK + kk * 2048, kBoxBytesBwd), idesc_dq, kk > 0);
                     }
                     umma_commit(&sm.bar_dq_full);
-                    // dK_j += dS^T Q_i
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {
-                        const uint32_t koff = (kk >> 2) * kBoxBytesBwd + (kk & 3) * 32;
-                        umma_ss(tmem + kColdK, desc_kmajor(sdS + koff), desc_mnmajor(sQ + kk * 2048, kBoxBytesBwd),
-                                idesc_dv, (n > 0) | (kk > 0));
-                    }
-                    umma_commit(&sm.bar_q_empty[s]);
                     umma_commit(&sm.bar_ds_free);
                 }
                 if (ok) umma_commit(&sm.bar_dkv_full);
@@ -541,18 +540,22 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 tmem_ld32(tmem + lane_base + kColdP + cbase + c * 32, dp);
                 tmem_wait_ld();
                 // dS' = P' * (dP - delta); the subtraction happened inside the tensor-core product.
-                // 32 query columns = four 16-byte chunks of row `row` in this half's tile.
+                // The fp16 result goes to shared memory (32 query columns = four 16-byte chunks of row
+                // `row` in this half's tile; operand of dQ^T) and, in place, to tensor memory (operand
+                // of dK).
+                uint32_t o[16];
 #pragma unroll
-                for (int v4 = 0; v4 < 4; ++v4) {
-                    uint4 w;
-                    const int e = c * 32 + v4 * 8;
-                    w.x = pack_half2(__uint_as_float(pv[e + 0]) * __uint_as_float(dp[v4 * 8 + 0]), __uint_as_float(pv[e + 1]) * __uint_as_float(dp[v4 * 8 + 1]));
-                    w.y = pack_half2(__uint_as_float(pv[e + 2]) * __uint_as_float(dp[v4 * 8 + 2]), __uint_as_float(pv[e + 3]) * __uint_as_float(dp[v4 * 8 + 3]));
-                    w.z = pack_half2(__uint_as_float(pv[e + 4]) * __uint_as_float(dp[v4 * 8 + 4]), __uint_as_float(pv[e + 5]) * __uint_as_float(dp[v4 * 8 + 5]));
-                    w.w = pack_half2(__uint_as_float(pv[e + 6]) * __uint_as_float(dp[v4 * 8 + 6]), __uint_as_float(pv[e + 7]) * __uint_as_float(dp[v4 * 8 + 7]));
-                    *reinterpret_cast<uint4 *>(ds_tile + swz128_offset(row, c * 32 + v4 * 8)) = w;
-                }
+                for (int e = 0; e < 16; ++e)
+                    o[e] = pack_half2(__uint_as_float(pv[c * 32 + 2 * e]) * __uint_as_float(dp[2 * e]),
+                                      __uint_as_float(pv[c * 32 + 2 * e + 1]) * __uint_as_float(dp[2 * e + 1]));
+#pragma unroll
+                for (int v4 = 0; v4 < 4; ++v4)
+                    *reinterpret_cast<uint4 *>(ds_tile + swz128_offset(row, c * 32 + v4 * 8)) =
+                        make_uint4(o[4 * v4], o[4 * v4 + 1], o[4 * v4 + 2], o[4 * v4 + 3]);
+                // these 16 columns lie inside the columns this thread has already read
+                tmem_st16(tmem + lane_base + kColdP + cbase + c * 16, o);
             }
+            tmem_wait_st();
             LT_TRACE_SINCE(13, td0);
             fence_proxy_async_smem();
             tc_fence_before_sync();
@@ -592,7 +595,8 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         LT_TRACE_BEGIN();
         for (int n = 0; n < n_iter && ok; ++n) {
             ok = LT_WAIT(&sm.bar_dq_full, n & 1, kWaitDqFull);
-            // the four reduction warps share named barriers below, so they leave the loop together
+            // the four reduction warps share named barriers below, so they leave the loop together;
+            // the vote also tells them that the staging buffers of the previous tile are free
             if constexpr (D == 128) ok = named_barrier_and(1, kNumReduceWarps * 32, ok);
             if (!ok) break;
             tc_fence_after_sync();
@@ -608,40 +612,55 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 const int d_idx = quad * 32 + lane;
                 const uint32_t taddr = tmem + (static_cast<uint32_t>(quad * 32) << 16) + kColdP;
                 const bool elected = (warp == kReduceWarp0) && (lane == 0);
-                auto stage_rows = [&](int k, const uint32_t *r) {  // r: 16 values, query rows 16k .. 16k+15
-                    float *buf = sm.dq_stage[(n * 8 + k) % kDqStageBufs];
+                auto store_rows = [&](int k, const uint32_t *r) {  // r: 16 values, query rows 16k .. 16k+15
+                    float *buf = sm.dq_stage[k % kDqStageBufs];
 #pragma unroll
                     for (int e = 0; e < kDqStageRows; ++e) buf[e * 128 + d_idx] = __uint_as_float(r[e]) * dq_mult;
-                    fence_proxy_async_smem();
-                    // the buffer of the next group of rows was last read two bulk operations ago
-                    if (elected) bulk_wait_group_read<1>();
-                    named_barrier_sync(1, kNumReduceWarps * 32);
-                    if (elected) {
-                        bulk_reduce_add_f32(dq_tile + k * kDqStageRows * 128, buf, kDqStageRows * 128 * sizeof(float));
-                        bulk_commit_group();
-                    }
                 };
-                // three quarters of the partial are read before anything is staged, so that the dP
-                // columns are released early
+                auto add_rows = [&](int k) {
+                    bulk_reduce_add_f32(dq_tile + k * kDqStageRows * 128, sm.dq_stage[k % kDqStageBufs],
+                                        kDqStageRows * 128 * sizeof(float));
+                    bulk_commit_group();
+                };
+                // All staging buffers are free here (the elected thread waited for its bulk reductions
+                // before the vote above).  Three quarters of the partial are read, two groups of rows
+                // are parked in shared memory to make room for the last quarter, and the dP columns
+                // are released before any reduction is issued.
                 uint32_t r0[32], r1[32], r2[32];
                 tmem_ld32(taddr, r0);
                 tmem_ld32(taddr + 32, r1);
                 tmem_ld32(taddr + 64, r2);
                 tmem_wait_ld();
-                stage_rows(0, r0);
-                stage_rows(1, r0 + 16);
+                store_rows(0, r0);
+                store_rows(1, r0 + 16);
                 tmem_ld32(taddr + 96, r0);
                 tmem_wait_ld();
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sm.bar_dq_empty);
                 LT_TRACE_SINCE(12, tr0);
+                fence_proxy_async_smem();
+                named_barrier_sync(1, kNumReduceWarps * 32);
+                if (elected) {
+                    add_rows(0);
+                    add_rows(1);
+                }
+                // groups 2..7 rotate through the three buffers: before group k is issued, the bulk
+                // reduction of group k-2 has finished reading, which frees the buffer of group k+1
+                auto stage_rows = [&](int k, const uint32_t *r) {
+                    store_rows(k, r);
+                    fence_proxy_async_smem();
+                    if (elected) bulk_wait_group_read<1>();
+                    named_barrier_sync(1, kNumReduceWarps * 32);
+                    if (elected) add_rows(k);
+                };
                 stage_rows(2, r1);
                 stage_rows(3, r1 + 16);
                 stage_rows(4, r2);
                 stage_rows(5, r2 + 16);
                 stage_rows(6, r0);
                 stage_rows(7, r0 + 16);
+                if (elected) bulk_wait_group_read<0>();
             } else {
 #pragma unroll
                 for (int ch = 0; ch < D / 64; ++ch) {
