@@ -14,7 +14,8 @@
 // across workers): here a CTA owns one key/value tile, keeps dK_j and dV_j resident in
 // tensor memory for the whole loop, and the cross-CTA reduction falls on dQ instead.
 //
-// The main kernel is warp specialised (14 warps, 144 registers per thread):
+// The main kernel is persistent (one CTA per SM walks a list of work items, heavy ones first)
+// and warp specialised (14 warps):
 //   warp 0       TMA producer (one thread): K_j, V_j once; then a two-stage ring of Q_i and a
 //                single-buffered dO_i; the warp also owns the tensor-memory allocation
 //   warp 1       tensor-core issuer (one thread)
@@ -40,7 +41,8 @@ constexpr float kLog2e = 1.4426950408889634f;
 enum {
     kWaitKV = 201, kWaitStageEmpty = 202, kWaitStageFull = 203, kWaitSFull = 204, kWaitPReady = 205,
     kWaitDpFull = 206, kWaitDsReady = 207, kWaitDsFree = 208, kWaitDqFull = 209, kWaitDqEmpty = 210,
-    kWaitDkvFull = 211, kWaitDoFull = 212, kWaitDoEmpty = 213, kBadSmemAlign = 220
+    kWaitDkvFull = 211, kWaitDoFull = 212, kWaitDoEmpty = 213, kWaitAccFree = 214, kWaitScale = 215,
+    kBadSmemAlign = 220
 };
 
 // ----------------------------------------------------------------------------- preprocess
@@ -166,12 +168,13 @@ __device__ __forceinline__ bool traced_wait(Trace &tr, uint64_t *bar, uint32_t p
 
 // ----------------------------------------------------------------------------- main kernel
 constexpr int kQStages = 2;   // Q_i ring; dO_i is single-buffered (it is dead once dV has been issued)
-constexpr int kBwdThreads = 448;  // 14 warps: 65536 / 448 leaves 144 registers per thread
+constexpr int kBwdThreads = 448;  // 14 warps; 128 registers per thread
 constexpr int kComputeWarp0 = 2, kNumComputeWarps = 8;
 constexpr int kReduceWarp0 = 10, kNumReduceWarps = 4;
 constexpr int kDqStageBufs = 3, kDqStageRows = 16;
 constexpr int kExtBytes = 2048;            // 128 rows x 16 bytes: one operand of the extra contraction step
 constexpr float kPScaleLog2Max = 14.f;     // P is kept as P * 2^c with c <= 14 so that fp16(P') <= 16384
+constexpr int kBarComputeWarps = 2, kBarReduceWarps = 1;  // named barrier ids
 
 template <int D>
 struct BwdSmem {
@@ -190,11 +193,13 @@ struct BwdSmem {
     // staging of the dQ partial for bulk reduction into global memory (D = 128 only):
     // each buffer holds 16 accumulator rows (16 query rows x 128 floats)
     float dq_stage[D == 128 ? kDqStageBufs : 1][D == 128 ? kDqStageRows * 128 : 4];
-    uint64_t bar_kv;
+    // per work item: K/V landed; dK/dV accumulators complete; accumulators read out; scale published
+    uint64_t bar_kv, bar_dkv_full, bar_acc_free, bar_scale_ready;
+    // per (query head, query tile) iteration
     uint64_t bar_q_full[kQStages], bar_q_empty[kQStages], bar_do_full, bar_do_empty;
-    uint64_t bar_s_full, bar_p_ready, bar_dp_full, bar_ds_ready, bar_ds_free, bar_dq_full, bar_dq_empty, bar_dkv_full;
-    float red[4];
-    float ds_mult;
+    uint64_t bar_s_full, bar_p_ready, bar_dp_full, bar_ds_ready, bar_ds_free, bar_dq_full, bar_dq_empty;
+    float red[2][4];       // per item parity: max squared row norm of V_j seen by each of four warps
+    float p_scale[2];      // per item parity: the exponent c of P' = P * 2^c
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -211,6 +216,33 @@ struct BwdParams {
     int B, Hq, Hkv, S, causal;
     float scale;
 };
+
+// One work item = key tile j of (batch b, kv head g).  Items are numbered so that the heavy
+// ones (small j under a causal mask) come first; CTA c takes items c, c + gridDim.x, ...
+struct BwdItem {
+    int j, b, g, i_first, tiles_per_head, n_iter, kv_row0;
+};
+__device__ __forceinline__ BwdItem bwd_item(const BwdParams &p, int item) {
+    BwdItem w;
+    const int n_tiles = p.S / kTileRows;
+    const int n_bg = p.B * p.Hkv;
+    w.j = item / n_bg;
+    const int bg = item - w.j * n_bg;
+    w.b = bg / p.Hkv;
+    w.g = bg - w.b * p.Hkv;
+    w.i_first = p.causal ? w.j : 0;
+    w.tiles_per_head = n_tiles - w.i_first;
+    w.n_iter = (p.Hq / p.Hkv) * w.tiles_per_head;  // flattened (query head of the group, query tile) loop
+    w.kv_row0 = (w.b * p.Hkv + w.g) * p.S + w.j * kTileRows;
+    return w;
+}
+// iteration n of an item -> first row of its query tile in the [B*Hq*S, D] view
+__device__ __forceinline__ long long bwd_q_row(const BwdParams &p, const BwdItem &w, int n) {
+    const int hh = n / w.tiles_per_head;
+    const int i = w.i_first + (n - hh * w.tiles_per_head);
+    return (static_cast<long long>(w.b) * p.Hq + w.g * (p.Hq / p.Hkv) + hh) * p.S +
+           static_cast<long long>(i) * kTileRows;
+}
 
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1)
@@ -231,19 +263,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
     const int lane = tid & 31;
-
-    // work item: key tile j of (batch b, kv head g); heavy (small j) items get the low block ids
-    const int n_tiles = p.S / kTileRows;
-    const int G = p.Hq / p.Hkv;
-    const int n_bg = p.B * p.Hkv;
-    const int j = blockIdx.x / n_bg;
-    const int bg = blockIdx.x % n_bg;
-    const int b = bg / p.Hkv;
-    const int g = bg % p.Hkv;
-    const int i_first = p.causal ? j : 0;
-    const int tiles_per_head = n_tiles - i_first;
-    const int n_iter = G * tiles_per_head;  // flattened (query head of the group, query tile) loop
-    const int kv_row0 = (b * p.Hkv + g) * p.S + j * kTileRows;
+    const int n_items = (p.S / kTileRows) * p.B * p.Hkv;
 
     // the swizzled tiles need 1024-byte alignment; the shared window is expected to give it
     const bool smem_ok = (smem_u32(smem_raw) & 1023u) == 0u;
@@ -251,6 +271,9 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         sm.abort_flag = smem_ok ? 0 : 1;
         if (!smem_ok) atomicCAS(p.status + kStatusWordTimeout, 0u, static_cast<unsigned int>(kBadSmemAlign));
         mbar_init(&sm.bar_kv, 1);
+        mbar_init(&sm.bar_dkv_full, 1);
+        mbar_init(&sm.bar_acc_free, kNumComputeWarps);
+        mbar_init(&sm.bar_scale_ready, 1);
         for (int s = 0; s < kQStages; ++s) {
             mbar_init(&sm.bar_q_full[s], 1);
             mbar_init(&sm.bar_q_empty[s], 1);
@@ -264,7 +287,6 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         mbar_init(&sm.bar_ds_free, 1);
         mbar_init(&sm.bar_dq_full, 1);
         mbar_init(&sm.bar_dq_empty, kNumReduceWarps);
-        mbar_init(&sm.bar_dkv_full, 1);
         mbar_fence_init();
         tma_prefetch_desc(&map_q);
         tma_prefetch_desc(&map_k);
@@ -289,141 +311,105 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     tc_fence_after_sync();
     const uint32_t tmem = sm.tmem_base;
     volatile int *abort_flag = &sm.abort_flag;
-
-    // iteration n -> first row of its query tile in the [B*Hq*S, D] view
-    auto q_row_of = [&](int n) -> long long {
-        const int hh = n / tiles_per_head;
-        const int i = i_first + (n - hh * tiles_per_head);
-        return (static_cast<long long>(b) * p.Hq + g * G + hh) * p.S + static_cast<long long>(i) * kTileRows;
-    };
-
-    // ---- K_j and V_j are requested before anything else
-    if (warp == 0 && lane == 0 && smem_ok) {
-        mbar_arrive_expect_tx(&sm.bar_kv, 2 * kTileBytes);
-#pragma unroll
-        for (int x = 0; x < kBoxes; ++x) {
-            tma_load_2d(sm.k + x * kBoxBytesBwd, &map_k, &sm.bar_kv, x * 64, kv_row0);
-            tma_load_2d(sm.v + x * kBoxBytesBwd, &map_v, &sm.bar_kv, x * 64, kv_row0);
-        }
-    }
-
-    // Power-of-two factor 2^c carried by dS before it is rounded to fp16, chosen from a bound
-    // on |dS| <= |dP| + |delta| <= max||dO_row|| * max||V_row|| + max|delta| so that the scaled
-    // values use fp16's normal range without overflow.  The factor rides on P (P' = P * 2^c,
-    // c <= 14), so dV and dQ/dK undo it exactly in their epilogues.
-    if (warp >= kComputeWarp0 && warp < kComputeWarp0 + 4) {
-        const int row = tid - kComputeWarp0 * 32;
-        float n2 = 0.f;
-        if (mbar_wait(&sm.bar_kv, 0, abort_flag, p.status, kWaitKV)) {
-#pragma unroll
-            for (int x = 0; x < kBoxes; ++x) {
-                const uint4 *src = reinterpret_cast<const uint4 *>(sm.v + x * kBoxBytesBwd + row * 128);
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const uint4 u = src[c];
-                    const __half2 *h = reinterpret_cast<const __half2 *>(&u);
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float2 f = __half22float2(h[e]);
-                        n2 = fmaf(f.x, f.x, n2);
-                        n2 = fmaf(f.y, f.y, n2);
-                    }
-                }
-            }
-        }
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) n2 = fmaxf(n2, __shfl_xor_sync(0xffffffffu, n2, off));
-        if (lane == 0) sm.red[warp - kComputeWarp0] = n2;
-    }
-    __syncthreads();
-    if (tid == 0) {
-        const float vmax2 = fmaxf(fmaxf(sm.red[0], sm.red[1]), fmaxf(sm.red[2], sm.red[3]));
-        const float do2 = __uint_as_float(p.status[kStatusWordMaxDoNorm2]);
-        const float dmax = __uint_as_float(p.status[kStatusWordMaxAbsDelta]);
-        const float bound = sqrtf(do2) * sqrtf(vmax2) + dmax;
-        int e = static_cast<int>(kPScaleLog2Max);    // all-zero dO: any factor works
-        if (!(bound < 3.0e38f)) e = -14;             // inf/NaN inputs: outputs are non-finite anyway
-        else if (bound > 1e-30f) e = min(static_cast<int>(kPScaleLog2Max), max(-14, ilogbf(32768.f / bound)));
-        sm.ds_mult = static_cast<float>(e);
-    }
-    __syncthreads();
-    const float p_scale_log2 = sm.ds_mult;              // c
-    const float inv_p_scale = exp2f(-p_scale_log2);     // 2^-c, exact
-    const float dq_mult = p.scale * inv_p_scale;
 #ifdef LT_BWD_TRACE
     const long long trace_prologue_end = clock64();
+    int trace_iters = 0;
 #endif
 
-    if (warp < kComputeWarp0) {
-        if (warp == 0) {
-            // ================================================================= TMA producer
-            if (lane == 0 && smem_ok) {
-                LT_TRACE_BEGIN();
-                int q_issued = 0, do_issued = 0;
-                for (int n = 0; n < n_iter; ++n) {
-                    const int s = n & 1, k = n >> 1;
-                    const long long q_row0 = q_row_of(n);
-                    if (k >= 1 && !LT_WAIT(&sm.bar_q_empty[s], (k - 1) & 1, kWaitStageEmpty)) break;
+    // Every role walks the same list of work items and keeps its own running iteration count
+    // `it` (over all items): each per-iteration barrier completes once per iteration, so its
+    // phase parity is a function of `it`; the per-item barriers use the item count `ic`.
+    if (warp == 0) {
+        // ================================================================= TMA producer
+        if (lane == 0 && smem_ok) {
+            LT_TRACE_BEGIN();
+            bool ok = true;
+            int it = 0, ic = 0;
+            int last_q = -1, last_do = -1, kv_loads = 0;  // for the cleanup after an abandoned wait
+            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++ic) {
+                const BwdItem w = bwd_item(p, item);
+                for (int n = 0; n < w.n_iter && ok; ++n, ++it) {
+                    const int s = it & 1, k = it >> 1;
+                    const long long q_row0 = bwd_q_row(p, w, n);
+                    if (k >= 1 && !(ok = LT_WAIT(&sm.bar_q_empty[s], (k - 1) & 1, kWaitStageEmpty))) break;
                     mbar_arrive_expect_tx(&sm.bar_q_full[s], kTileBytes + kExtBytes);
 #pragma unroll
                     for (int x = 0; x < kBoxes; ++x)
                         tma_load_2d(sm.q[s] + x * kBoxBytesBwd, &map_q, &sm.bar_q_full[s], x * 64,
                                     static_cast<int>(q_row0));
                     bulk_load_1d(sm.ext_q[s], p.lse_ext + q_row0, kExtBytes, &sm.bar_q_full[s]);
-                    q_issued = n + 1;
-                    if (n >= 1 && !LT_WAIT(&sm.bar_do_empty, (n - 1) & 1, kWaitDoEmpty)) break;
+                    last_q = it;
+                    if (it >= 1 && !(ok = LT_WAIT(&sm.bar_do_empty, (it - 1) & 1, kWaitDoEmpty))) break;
                     mbar_arrive_expect_tx(&sm.bar_do_full, kTileBytes + kExtBytes);
 #pragma unroll
                     for (int x = 0; x < kBoxes; ++x)
                         tma_load_2d(sm.d_o + x * kBoxBytesBwd, &map_do, &sm.bar_do_full, x * 64,
                                     static_cast<int>(q_row0));
                     bulk_load_1d(sm.ext_do, p.delta_ext + q_row0, kExtBytes, &sm.bar_do_full);
-                    do_issued = n + 1;
-                }
-                LT_TRACE_END(kRoleProducer);
-                if (*abort_flag) {
-                    // abandoned: give this CTA's own copies a bounded time to land before shared memory is released
-                    for (int t = 0; t < (1 << 16) && !mbar_try_wait(&sm.bar_kv, 0); ++t) {}
-                    for (int n = max(0, q_issued - kQStages); n < q_issued; ++n)
-                        for (int t = 0; t < (1 << 16) && !mbar_try_wait(&sm.bar_q_full[n & 1], (n >> 1) & 1); ++t) {}
-                    if (do_issued > 0)
-                        for (int t = 0; t < (1 << 16) && !mbar_try_wait(&sm.bar_do_full, (do_issued - 1) & 1); ++t) {}
+                    last_do = it;
+                    if (n == 0) {
+                        // K_j and V_j follow the first query tile: they may only be overwritten once every
+                        // product of the previous item has completed
+                        if (ic >= 1 && !(ok = LT_WAIT(&sm.bar_dkv_full, (ic - 1) & 1, kWaitDkvFull))) break;
+                        mbar_arrive_expect_tx(&sm.bar_kv, 2 * kTileBytes);
+#pragma unroll
+                        for (int x = 0; x < kBoxes; ++x) {
+                            tma_load_2d(sm.k + x * kBoxBytesBwd, &map_k, &sm.bar_kv, x * 64, w.kv_row0);
+                            tma_load_2d(sm.v + x * kBoxBytesBwd, &map_v, &sm.bar_kv, x * 64, w.kv_row0);
+                        }
+                        ++kv_loads;
+                    }
                 }
             }
-            __syncwarp();
-        } else if (warp == 1) {
-            // ================================================================= tensor-core issuer
-            if (lane == 0 && smem_ok) {
-                LT_TRACE_BEGIN();
-                const uint32_t sK = smem_u32(sm.k), sV = smem_u32(sm.v), sdS = smem_u32(sm.ds), sdO = smem_u32(sm.d_o);
-                const uint32_t s_ones = smem_u32(sm.ext_ones), s_zero = smem_u32(sm.ext_zero);
-                const uint64_t desc_ones = desc_kmajor_noswz(s_ones, s_zero - s_ones, 128);
-                const uint64_t desc_ext_do = desc_kmajor_noswz(smem_u32(sm.ext_do), s_zero - smem_u32(sm.ext_do), 128);
-                constexpr uint32_t idesc_s = make_idesc(128, 128, false, false);
-                constexpr uint32_t idesc_dv = make_idesc(128, D, false, true);
-                constexpr uint32_t idesc_dq = make_idesc(128, D == 128 ? 128 : D, true, true);
-                auto issue_s = [&](int n) {  // S^T = K_j Q_i^T - LSE_i / scale
-                    const uint32_t sQn = smem_u32(sm.q[n & 1]), s_ext = smem_u32(sm.ext_q[n & 1]);
+            LT_TRACE_END(kRoleProducer);
+            if (*abort_flag) {
+                // abandoned: give this CTA's own copies a bounded time to land before shared memory is released
+                if (kv_loads > 0)
+                    for (int t = 0; t < (1 << 16) && !mbar_try_wait(&sm.bar_kv, (kv_loads - 1) & 1); ++t) {}
+                for (int n = max(0, last_q - 1); n <= last_q; ++n)
+                    for (int t = 0; t < (1 << 16) && !mbar_try_wait(&sm.bar_q_full[n & 1], (n >> 1) & 1); ++t) {}
+                if (last_do >= 0)
+                    for (int t = 0; t < (1 << 16) && !mbar_try_wait(&sm.bar_do_full, last_do & 1); ++t) {}
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ================================================================= tensor-core issuer
+        if (lane == 0 && smem_ok) {
+            LT_TRACE_BEGIN();
+            const uint32_t sK = smem_u32(sm.k), sV = smem_u32(sm.v), sdS = smem_u32(sm.ds), sdO = smem_u32(sm.d_o);
+            const uint32_t s_ones = smem_u32(sm.ext_ones), s_zero = smem_u32(sm.ext_zero);
+            const uint64_t desc_ones = desc_kmajor_noswz(s_ones, s_zero - s_ones, 128);
+            const uint64_t desc_ext_do = desc_kmajor_noswz(smem_u32(sm.ext_do), s_zero - smem_u32(sm.ext_do), 128);
+            constexpr uint32_t idesc_s = make_idesc(128, 128, false, false);
+            constexpr uint32_t idesc_dv = make_idesc(128, D, false, true);
+            constexpr uint32_t idesc_dq = make_idesc(128, D == 128 ? 128 : D, true, true);
+            auto issue_s = [&](int t) {  // S^T = K_j Q_i^T - LSE_i / scale, for running iteration t
+                const uint32_t sQn = smem_u32(sm.q[t & 1]), s_ext = smem_u32(sm.ext_q[t & 1]);
 #pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk) {
-                        const uint32_t koff = (kk >> 2) * kBoxBytesBwd + (kk & 3) * 32;
-                        umma_ss(tmem + kColS, desc_kmajor(sK + koff), desc_kmajor(sQn + koff), idesc_s, kk > 0);
-                    }
-                    umma_ss(tmem + kColS, desc_ones, desc_kmajor_noswz(s_ext, s_zero - s_ext, 128), idesc_s, 1);
-                    umma_commit(&sm.bar_s_full);
-                };
-                bool ok = LT_WAIT(&sm.bar_kv, 0, kWaitKV) && LT_WAIT(&sm.bar_q_full[0], 0, kWaitStageFull);
-                if (ok) {
-                    tc_fence_after_sync();
-                    issue_s(0);
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t koff = (kk >> 2) * kBoxBytesBwd + (kk & 3) * 32;
+                    umma_ss(tmem + kColS, desc_kmajor(sK + koff), desc_kmajor(sQn + koff), idesc_s, kk > 0);
                 }
-                for (int n = 0; n < n_iter && ok; ++n) {
-                    const int s = n & 1;
+                umma_ss(tmem + kColS, desc_ones, desc_kmajor_noswz(s_ext, s_zero - s_ext, 128), idesc_s, 1);
+                umma_commit(&sm.bar_s_full);
+            };
+            bool ok = true;
+            int it = 0, ic = 0;
+            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++ic) {
+                const BwdItem w = bwd_item(p, item);
+                ok = LT_WAIT(&sm.bar_kv, ic & 1, kWaitKV) &&
+                     LT_WAIT(&sm.bar_q_full[it & 1], (it >> 1) & 1, kWaitStageFull);
+                if (!ok) break;
+                tc_fence_after_sync();
+                issue_s(it);
+                for (int n = 0; n < w.n_iter && ok; ++n, ++it) {
+                    const int s = it & 1;
                     const uint32_t sQ = smem_u32(sm.q[s]);
                     // dP^T = V_j dO_i^T - delta_i   (its columns held the previous dQ partial until the
                     //                                reduce warps drained it)
-                    if (!(ok = LT_WAIT(&sm.bar_do_full, n & 1, kWaitDoFull))) break;
-                    if (n > 0 && !(ok = LT_WAIT(&sm.bar_dq_empty, (n - 1) & 1, kWaitDqEmpty))) break;
+                    if (!(ok = LT_WAIT(&sm.bar_do_full, it & 1, kWaitDoFull))) break;
+                    if (it > 0 && !(ok = LT_WAIT(&sm.bar_dq_empty, (it - 1) & 1, kWaitDqEmpty))) break;
                     tc_fence_after_sync();
 #pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk) {
@@ -434,7 +420,9 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     umma_commit(&sm.bar_dp_full);
                     // dV_j += P'^T dO_i   (A = P'^T from tensor memory; query columns 0-63 sit at columns
                     //                      0-31, query columns 64-127 at columns 64-95 of the S region)
-                    if (!(ok = LT_WAIT(&sm.bar_p_ready, n & 1, kWaitPReady))) break;
+                    if (!(ok = LT_WAIT(&sm.bar_p_ready, it & 1, kWaitPReady))) break;
+                    // the first product of an item overwrites accumulators the previous item's epilogue reads
+                    if (n == 0 && ic > 0 && !(ok = LT_WAIT(&sm.bar_acc_free, (ic - 1) & 1, kWaitAccFree))) break;
                     tc_fence_after_sync();
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk)
@@ -442,11 +430,11 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                                 desc_mnmajor(sdO + kk * 2048, kBoxBytesBwd), idesc_dv, (n > 0) | (kk > 0));
                     umma_commit(&sm.bar_do_empty);
                     // the next S^T overwrites P'^T; the tensor pipe executes in issue order
-                    if (n + 1 < n_iter) {
-                        if (!(ok = LT_WAIT(&sm.bar_q_full[(n + 1) & 1], ((n + 1) >> 1) & 1, kWaitStageFull))) break;
-                        issue_s(n + 1);
+                    if (n + 1 < w.n_iter) {
+                        if (!(ok = LT_WAIT(&sm.bar_q_full[(it + 1) & 1], ((it + 1) >> 1) & 1, kWaitStageFull))) break;
+                        issue_s(it + 1);
                     }
-                    if (!(ok = LT_WAIT(&sm.bar_ds_ready, n & 1, kWaitDsReady))) break;
+                    if (!(ok = LT_WAIT(&sm.bar_ds_ready, it & 1, kWaitDsReady))) break;
                     tc_fence_after_sync();
                     // dK_j += dS'^T Q_i   (A = dS'^T from tensor memory, stored like P'^T: query columns
                     //                       0-63 at columns 0-31 and 64-127 at columns 64-95 of the dP region)
@@ -472,10 +460,10 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     umma_commit(&sm.bar_ds_free);
                 }
                 if (ok) umma_commit(&sm.bar_dkv_full);
-                LT_TRACE_END(kRoleMma);
             }
-            __syncwarp();
+            LT_TRACE_END(kRoleMma);
         }
+        __syncwarp();
     } else if (warp < kReduceWarp0) {
         // ================================================================= softmax / dS warps
         const int quad = warp & 3;                           // tensor-memory lane quadrant
@@ -486,15 +474,17 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const float scale_log2 = p.scale * kLog2e;
         uint8_t *ds_tile = sm.ds + half_sel * kBoxBytesBwd;
         uint32_t pv[64];  // bits of this thread's 64 fp32 values of P' = P * 2^c for the current tile pair
+        float p_scale_log2 = 0.f;
         bool ok = smem_ok;
+        int it = 0, ic = 0;
         LT_TRACE_BEGIN();
 
-        auto compute_p = [&](int n) -> bool {
-            if (!LT_WAIT(&sm.bar_s_full, n & 1, kWaitSFull)) return false;
+        auto compute_p = [&](const BwdItem &w, int n, int t) -> bool {
+            if (!LT_WAIT(&sm.bar_s_full, t & 1, kWaitSFull)) return false;
             tc_fence_after_sync();
             LT_TRACE_MARK(tp0);
-            const int hh = n / tiles_per_head;
-            const bool diag = p.causal && (i_first + (n - hh * tiles_per_head) == j);
+            const int hh = n / w.tiles_per_head;
+            const bool diag = p.causal && (w.i_first + (n - hh * w.tiles_per_head) == w.j);
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
                 uint32_t sv[32];
@@ -527,176 +517,242 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             return true;
         };
 
-        ok = ok && compute_p(0);
-        for (int n = 0; n < n_iter && ok; ++n) {
-            if (!(ok = LT_WAIT(&sm.bar_dp_full, n & 1, kWaitDpFull))) break;
-            tc_fence_after_sync();
-            // the previous dS^T tile must have been consumed by dQ and dK before it is overwritten
-            if (n > 0 && !(ok = LT_WAIT(&sm.bar_ds_free, (n - 1) & 1, kWaitDsFree))) break;
-            LT_TRACE_MARK(td0);
+        for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++ic) {
+            const BwdItem w = bwd_item(p, item);
+            // ---- per item: a power-of-two factor 2^c carried by dS before it is rounded to fp16, chosen
+            // from a bound on |dS| <= |dP| + |delta| <= max||dO_row|| * max||V_row|| + max|delta| so that
+            // the scaled values use fp16's normal range without overflow.  The factor rides on P
+            // (P' = P * 2^c, c <= 14); dV and dQ/dK undo it exactly in their epilogues.
+            ok = ok && LT_WAIT(&sm.bar_kv, ic & 1, kWaitKV);
+            if (ok && half_sel == 0) {
+                float n2 = 0.f;
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                uint32_t dp[32];
-                tmem_ld32(tmem + lane_base + kColdP + cbase + c * 32, dp);
-                tmem_wait_ld();
-                // dS' = P' * (dP - delta); the subtraction happened inside the tensor-core product.
-                // The fp16 result goes to shared memory (32 query columns = four 16-byte chunks of row
-                // `row` in this half's tile; operand of dQ^T) and, in place, to tensor memory (operand
-                // of dK).
-                uint32_t o[16];
+                for (int x = 0; x < kBoxes; ++x) {
+                    const uint4 *src = reinterpret_cast<const uint4 *>(sm.v + x * kBoxBytesBwd + row * 128);
 #pragma unroll
-                for (int e = 0; e < 16; ++e)
-                    o[e] = pack_half2(__uint_as_float(pv[c * 32 + 2 * e]) * __uint_as_float(dp[2 * e]),
-                                      __uint_as_float(pv[c * 32 + 2 * e + 1]) * __uint_as_float(dp[2 * e + 1]));
+                    for (int c = 0; c < 8; ++c) {
+                        const uint4 u = src[(c + row) & 7];  // rotated start: conflict-free across the warp
+                        const __half2 *h = reinterpret_cast<const __half2 *>(&u);
 #pragma unroll
-                for (int v4 = 0; v4 < 4; ++v4)
-                    *reinterpret_cast<uint4 *>(ds_tile + swz128_offset(row, c * 32 + v4 * 8)) =
-                        make_uint4(o[4 * v4], o[4 * v4 + 1], o[4 * v4 + 2], o[4 * v4 + 3]);
-                // these 16 columns lie inside the columns this thread has already read
-                tmem_st16(tmem + lane_base + kColdP + cbase + c * 16, o);
+                        for (int e = 0; e < 4; ++e) {
+                            const float2 f = __half22float2(h[e]);
+                            n2 = fmaf(f.x, f.x, n2);
+                            n2 = fmaf(f.y, f.y, n2);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) n2 = fmaxf(n2, __shfl_xor_sync(0xffffffffu, n2, off));
+                if (lane == 0) sm.red[ic & 1][quad] = n2;
             }
-            tmem_wait_st();
-            LT_TRACE_SINCE(13, td0);
-            fence_proxy_async_smem();
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.bar_ds_ready);
-            LT_TRACE_SINCE(14, td0);
-            if (n + 1 < n_iter) ok = compute_p(n + 1);
-        }
-        LT_TRACE_END(kRoleCompute);
+            // all eight warps vote here, also when leaving after an abandoned wait, so nobody is left behind
+            ok = named_barrier_and(kBarComputeWarps, kNumComputeWarps * 32, ok);
+            if (!ok) break;
+            {
+                const float *rd = sm.red[ic & 1];
+                const float vmax2 = fmaxf(fmaxf(rd[0], rd[1]), fmaxf(rd[2], rd[3]));
+                const float do2 = __uint_as_float(p.status[kStatusWordMaxDoNorm2]);
+                const float dmax = __uint_as_float(p.status[kStatusWordMaxAbsDelta]);
+                const float bound = sqrtf(do2) * sqrtf(vmax2) + dmax;
+                int e = static_cast<int>(kPScaleLog2Max);    // all-zero dO: any factor works
+                if (!(bound < 3.0e38f)) e = -14;             // inf/NaN inputs: outputs are non-finite anyway
+                else if (bound > 1e-30f) e = min(static_cast<int>(kPScaleLog2Max), max(-14, ilogbf(32768.f / bound)));
+                p_scale_log2 = static_cast<float>(e);
+                if (warp == kComputeWarp0 && lane == 0) {
+                    sm.p_scale[ic & 1] = p_scale_log2;
+                    mbar_arrive(&sm.bar_scale_ready);  // the reduction warps read it
+                }
+            }
+            const float inv_p_scale = exp2f(-p_scale_log2);  // 2^-c, exact
 
-        // epilogue: the first four softmax warps write dK_j, the other four dV_j; thread = key row
-        if (ok && mbar_wait(&sm.bar_dkv_full, 0, abort_flag, p.status, kWaitDkvFull)) {
-            tc_fence_after_sync();
-            const float mult = half_sel == 0 ? dq_mult : inv_p_scale;
-            const uint32_t col0 = half_sel == 0 ? kColdK : kColdV;
-            __half *dst = (half_sel == 0 ? p.dK : p.dV) + (static_cast<long long>(kv_row0) + row) * D;
+            ok = compute_p(w, 0, it);
+            for (int n = 0; n < w.n_iter && ok; ++n, ++it) {
+                if (!(ok = LT_WAIT(&sm.bar_dp_full, it & 1, kWaitDpFull))) break;
+                tc_fence_after_sync();
+                // the previous dS^T tile must have been consumed by the dQ product before it is overwritten
+                if (it > 0 && !(ok = LT_WAIT(&sm.bar_ds_free, (it - 1) & 1, kWaitDsFree))) break;
+                LT_TRACE_MARK(td0);
 #pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
-                uint32_t r[32];
-                tmem_ld32(tmem + lane_base + col0 + c * 32, r);
-                tmem_wait_ld();
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t dp[32];
+                    tmem_ld32(tmem + lane_base + kColdP + cbase + c * 32, dp);
+                    tmem_wait_ld();
+                    // dS' = P' * (dP - delta); the subtraction happened inside the tensor-core product.
+                    // The fp16 result goes to shared memory (32 query columns = four 16-byte chunks of row
+                    // `row` in this half's tile; operand of the dQ product) and, in place, to tensor
+                    // memory (operand of dK).
+                    uint32_t o[16];
 #pragma unroll
-                for (int v8 = 0; v8 < 4; ++v8) {
-                    uint4 w;
-                    w.x = pack_half2(__uint_as_float(r[8 * v8 + 0]) * mult, __uint_as_float(r[8 * v8 + 1]) * mult);
-                    w.y = pack_half2(__uint_as_float(r[8 * v8 + 2]) * mult, __uint_as_float(r[8 * v8 + 3]) * mult);
-                    w.z = pack_half2(__uint_as_float(r[8 * v8 + 4]) * mult, __uint_as_float(r[8 * v8 + 5]) * mult);
-                    w.w = pack_half2(__uint_as_float(r[8 * v8 + 6]) * mult, __uint_as_float(r[8 * v8 + 7]) * mult);
-                    reinterpret_cast<uint4 *>(dst + c * 32)[v8] = w;
+                    for (int e = 0; e < 16; ++e)
+                        o[e] = pack_half2(__uint_as_float(pv[c * 32 + 2 * e]) * __uint_as_float(dp[2 * e]),
+                                          __uint_as_float(pv[c * 32 + 2 * e + 1]) * __uint_as_float(dp[2 * e + 1]));
+#pragma unroll
+                    for (int v4 = 0; v4 < 4; ++v4)
+                        *reinterpret_cast<uint4 *>(ds_tile + swz128_offset(row, c * 32 + v4 * 8)) =
+                            make_uint4(o[4 * v4], o[4 * v4 + 1], o[4 * v4 + 2], o[4 * v4 + 3]);
+                    // these 16 columns lie inside the columns this thread has already read
+                    tmem_st16(tmem + lane_base + kColdP + cbase + c * 16, o);
+                }
+                tmem_wait_st();
+                LT_TRACE_SINCE(13, td0);
+                fence_proxy_async_smem();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.bar_ds_ready);
+                LT_TRACE_SINCE(14, td0);
+                if (n + 1 < w.n_iter) ok = compute_p(w, n + 1, it + 1);
+            }
+
+            // epilogue: the first four softmax warps write dK_j, the other four dV_j; thread = key row
+            if (ok && (ok = LT_WAIT(&sm.bar_dkv_full, ic & 1, kWaitDkvFull))) {
+                tc_fence_after_sync();
+                const float mult = half_sel == 0 ? p.scale * inv_p_scale : inv_p_scale;
+                const uint32_t col0 = half_sel == 0 ? kColdK : kColdV;
+                __half *dst = (half_sel == 0 ? p.dK : p.dV) + (static_cast<long long>(w.kv_row0) + row) * D;
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(tmem + lane_base + col0 + c * 32, r);
+                    tmem_wait_ld();
+                    if (c == D / 32 - 1) {
+                        // the accumulators are in registers: the next item may overwrite them
+                        tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&sm.bar_acc_free);
+                    }
+#pragma unroll
+                    for (int v8 = 0; v8 < 4; ++v8) {
+                        uint4 o;
+                        o.x = pack_half2(__uint_as_float(r[8 * v8 + 0]) * mult, __uint_as_float(r[8 * v8 + 1]) * mult);
+                        o.y = pack_half2(__uint_as_float(r[8 * v8 + 2]) * mult, __uint_as_float(r[8 * v8 + 3]) * mult);
+                        o.z = pack_half2(__uint_as_float(r[8 * v8 + 4]) * mult, __uint_as_float(r[8 * v8 + 5]) * mult);
+                        o.w = pack_half2(__uint_as_float(r[8 * v8 + 6]) * mult, __uint_as_float(r[8 * v8 + 7]) * mult);
+                        reinterpret_cast<uint4 *>(dst + c * 32)[v8] = o;
+                    }
                 }
             }
         }
+        LT_TRACE_END(kRoleCompute);
     } else {
         // ================================================================= dQ reduction warps
         const int quad = warp & 3;
         bool ok = smem_ok;
+        int it = 0, ic = 0;
         LT_TRACE_BEGIN();
-        for (int n = 0; n < n_iter && ok; ++n) {
-            ok = LT_WAIT(&sm.bar_dq_full, n & 1, kWaitDqFull);
-            // the four reduction warps share named barriers below, so they leave the loop together;
-            // the vote also tells them that the staging buffers of the previous tile are free
-            if constexpr (D == 128) ok = named_barrier_and(1, kNumReduceWarps * 32, ok);
-            if (!ok) break;
-            tc_fence_after_sync();
-            LT_TRACE_MARK(tr0);
-            float *dq_tile = p.dq_acc + q_row_of(n) * D;
-            if constexpr (D == 128) {
-                // dQ^T: this thread holds head-dim element d = 32*quad + lane of all 128 query rows;
-                // one warp instruction adds 32 consecutive floats of one accumulator row
-                // dQ^T: this thread holds head-dim element d = 32*quad + lane of all 128 query rows.
-                // Sixteen query rows at a time are scaled, staged in shared memory exactly as they lie
-                // in the accumulator (16 rows x 128 floats, contiguous) and added to it by one bulk
-                // reduction; three staging buffers keep the copies in flight.
-                const int d_idx = quad * 32 + lane;
-                const uint32_t taddr = tmem + (static_cast<uint32_t>(quad * 32) << 16) + kColdP;
-                const bool elected = (warp == kReduceWarp0) && (lane == 0);
-                auto store_rows = [&](int k, const uint32_t *r) {  // r: 16 values, query rows 16k .. 16k+15
-                    float *buf = sm.dq_stage[k % kDqStageBufs];
-#pragma unroll
-                    for (int e = 0; e < kDqStageRows; ++e) buf[e * 128 + d_idx] = __uint_as_float(r[e]) * dq_mult;
-                };
-                auto add_rows = [&](int k) {
-                    bulk_reduce_add_f32(dq_tile + k * kDqStageRows * 128, sm.dq_stage[k % kDqStageBufs],
-                                        kDqStageRows * 128 * sizeof(float));
-                    bulk_commit_group();
-                };
-                // All staging buffers are free here (the elected thread waited for its bulk reductions
-                // before the vote above).  Three quarters of the partial are read, two groups of rows
-                // are parked in shared memory to make room for the last quarter, and the dP columns
-                // are released before any reduction is issued.
-                uint32_t r0[32], r1[32], r2[32];
-                tmem_ld32(taddr, r0);
-                tmem_ld32(taddr + 32, r1);
-                tmem_ld32(taddr + 64, r2);
-                tmem_wait_ld();
-                store_rows(0, r0);
-                store_rows(1, r0 + 16);
-                tmem_ld32(taddr + 96, r0);
-                tmem_wait_ld();
-                tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&sm.bar_dq_empty);
-                LT_TRACE_SINCE(12, tr0);
-                fence_proxy_async_smem();
-                named_barrier_sync(1, kNumReduceWarps * 32);
-                if (elected) {
-                    add_rows(0);
-                    add_rows(1);
+        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++ic) {
+            const BwdItem w = bwd_item(p, item);
+            float dq_mult = 0.f;
+            for (int n = 0; n < w.n_iter; ++n, ++it) {
+                ok = LT_WAIT(&sm.bar_dq_full, it & 1, kWaitDqFull);
+                if (ok && n == 0) {
+                    ok = LT_WAIT(&sm.bar_scale_ready, ic & 1, kWaitScale);
+                    dq_mult = p.scale * exp2f(-sm.p_scale[ic & 1]);
                 }
-                // groups 2..7 rotate through the three buffers: before group k is issued, the bulk
-                // reduction of group k-2 has finished reading, which frees the buffer of group k+1
-                auto stage_rows = [&](int k, const uint32_t *r) {
-                    store_rows(k, r);
-                    fence_proxy_async_smem();
-                    if (elected) bulk_wait_group_read<1>();
-                    named_barrier_sync(1, kNumReduceWarps * 32);
-                    if (elected) add_rows(k);
-                };
-                stage_rows(2, r1);
-                stage_rows(3, r1 + 16);
-                stage_rows(4, r2);
-                stage_rows(5, r2 + 16);
-                stage_rows(6, r0);
-                stage_rows(7, r0 + 16);
-                if (elected) bulk_wait_group_read<0>();
-            } else {
+                // the four reduction warps share named barriers below, so they leave the loop together;
+                // the vote also tells them that the staging buffers of the previous tile are free
+                if constexpr (D == 128) ok = named_barrier_and(kBarReduceWarps, kNumReduceWarps * 32, ok);
+                if (!ok) break;
+                tc_fence_after_sync();
+                LT_TRACE_MARK(tr0);
+                float *dq_tile = p.dq_acc + bwd_q_row(p, w, n) * D;
+                if constexpr (D == 128) {
+                    // dQ^T: this thread holds head-dim element d = 32*quad + lane of all 128 query rows.
+                    // Sixteen query rows at a time are scaled, staged in shared memory exactly as they lie
+                    // in the accumulator (16 rows x 128 floats, contiguous) and added to it by one bulk
+                    // reduction; three staging buffers keep the copies in flight.
+                    const int d_idx = quad * 32 + lane;
+                    const uint32_t taddr = tmem + (static_cast<uint32_t>(quad * 32) << 16) + kColdP;
+                    const bool elected = (warp == kReduceWarp0) && (lane == 0);
+                    auto store_rows = [&](int k, const uint32_t *r) {  // r: 16 values, query rows 16k .. 16k+15
+                        float *buf = sm.dq_stage[k % kDqStageBufs];
 #pragma unroll
-                for (int ch = 0; ch < D / 64; ++ch) {
-                    uint32_t r[2][32];
-#pragma unroll
-                    for (int lh = 0; lh < 2; ++lh)
-                        tmem_ld_16x256b_x8(tmem + (static_cast<uint32_t>(quad * 32 + lh * 16) << 16) + kColdP + ch * 64,
-                                           r[lh]);
+                        for (int e = 0; e < kDqStageRows; ++e) buf[e * 128 + d_idx] = __uint_as_float(r[e]) * dq_mult;
+                    };
+                    auto add_rows = [&](int k) {
+                        bulk_reduce_add_f32(dq_tile + k * kDqStageRows * 128, sm.dq_stage[k % kDqStageBufs],
+                                            kDqStageRows * 128 * sizeof(float));
+                        bulk_commit_group();
+                    };
+                    // All staging buffers are free here (the elected thread waited for its bulk reductions
+                    // before the vote above).  Three quarters of the partial are read, two groups of rows
+                    // are parked in shared memory to make room for the last quarter, and the dP columns
+                    // are released before any reduction is issued.
+                    uint32_t r0[32], r1[32], r2[32];
+                    tmem_ld32(taddr, r0);
+                    tmem_ld32(taddr + 32, r1);
+                    tmem_ld32(taddr + 64, r2);
                     tmem_wait_ld();
-                    if (ch == D / 64 - 1) {
-                        // the whole partial is in registers: the dP columns may be overwritten
-                        tc_fence_before_sync();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&sm.bar_dq_empty);
-                        LT_TRACE_SINCE(12, tr0);
+                    store_rows(0, r0);
+                    store_rows(1, r0 + 16);
+                    tmem_ld32(taddr + 96, r0);
+                    tmem_wait_ld();
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm.bar_dq_empty);
+                    LT_TRACE_SINCE(12, tr0);
+                    fence_proxy_async_smem();
+                    named_barrier_sync(kBarReduceWarps, kNumReduceWarps * 32);
+                    if (elected) {
+                        add_rows(0);
+                        add_rows(1);
                     }
-                    // four neighbouring threads add 32 contiguous bytes of one query row
+                    // groups 2..7 rotate through the three buffers: before group k is issued, the bulk
+                    // reduction of group k-2 has finished reading, which frees the buffer of group k+1
+                    auto stage_rows = [&](int k, const uint32_t *r) {
+                        store_rows(k, r);
+                        fence_proxy_async_smem();
+                        if (elected) bulk_wait_group_read<1>();
+                        named_barrier_sync(kBarReduceWarps, kNumReduceWarps * 32);
+                        if (elected) add_rows(k);
+                    };
+                    stage_rows(2, r1);
+                    stage_rows(3, r1 + 16);
+                    stage_rows(4, r2);
+                    stage_rows(5, r2 + 16);
+                    stage_rows(6, r0);
+                    stage_rows(7, r0 + 16);
+                    if (elected) bulk_wait_group_read<0>();
+                } else {
+                    // D = 64: dQ partial with lanes = query rows; four neighbouring threads add 32
+                    // contiguous bytes of one query row
 #pragma unroll
-                    for (int lh = 0; lh < 2; ++lh) {
-                        float *base = dq_tile + static_cast<long long>(quad * 32 + lh * 16 + (lane >> 2)) * D + ch * 64 +
-                                      2 * (lane & 3);
+                    for (int ch = 0; ch < D / 64; ++ch) {
+                        uint32_t r[2][32];
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) {
-                            red_add_v2(base + 8 * k, __uint_as_float(r[lh][4 * k]) * dq_mult,
-                                       __uint_as_float(r[lh][4 * k + 1]) * dq_mult);
-                            red_add_v2(base + 8 * D + 8 * k, __uint_as_float(r[lh][4 * k + 2]) * dq_mult,
-                                       __uint_as_float(r[lh][4 * k + 3]) * dq_mult);
+                        for (int lh = 0; lh < 2; ++lh)
+                            tmem_ld_16x256b_x8(tmem + (static_cast<uint32_t>(quad * 32 + lh * 16) << 16) + kColdP + ch * 64,
+                                               r[lh]);
+                        tmem_wait_ld();
+                        if (ch == D / 64 - 1) {
+                            // the whole partial is in registers: the dP columns may be overwritten
+                            tc_fence_before_sync();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&sm.bar_dq_empty);
+                            LT_TRACE_SINCE(12, tr0);
+                        }
+#pragma unroll
+                        for (int lh = 0; lh < 2; ++lh) {
+                            float *base = dq_tile + static_cast<long long>(quad * 32 + lh * 16 + (lane >> 2)) * D +
+                                          ch * 64 + 2 * (lane & 3);
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) {
+                                red_add_v2(base + 8 * k, __uint_as_float(r[lh][4 * k]) * dq_mult,
+                                           __uint_as_float(r[lh][4 * k + 1]) * dq_mult);
+                                red_add_v2(base + 8 * D + 8 * k, __uint_as_float(r[lh][4 * k + 2]) * dq_mult,
+                                           __uint_as_float(r[lh][4 * k + 3]) * dq_mult);
+                            }
                         }
                     }
                 }
+                LT_TRACE_SINCE(13, tr0);
             }
-            LT_TRACE_SINCE(13, tr0);
         }
         // shared memory must stay valid until the bulk reductions have read it
         if constexpr (D == 128) bulk_wait_group_all();
         LT_TRACE_END(kRoleReduce);
+#ifdef LT_BWD_TRACE
+        trace_iters = it;
+#endif
     }
 
 #ifdef LT_BWD_TRACE
@@ -708,11 +764,11 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #ifdef LT_BWD_TRACE
     if (tid == 0) {
         atomicAdd(&g_bwd_trace[64 + 3], static_cast<unsigned long long>(clock64() - trace_cta_t0));
-        atomicAdd(&g_bwd_trace[64 + 2], static_cast<unsigned long long>(n_iter));
         atomicAdd(&g_bwd_trace[64 + 1], 1ull);
         atomicAdd(&g_bwd_trace[64 + 0], static_cast<unsigned long long>(trace_prologue_end - trace_cta_t0));
         atomicAdd(&g_bwd_trace[64 + 4], static_cast<unsigned long long>(trace_teardown_begin - trace_prologue_end));
     }
+    if (tid == kReduceWarp0 * 32) atomicAdd(&g_bwd_trace[64 + 2], static_cast<unsigned long long>(trace_iters));
 #endif
 }
 
@@ -777,7 +833,8 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
     const size_t smem = sizeof(BwdSmem<D>);
     e = cudaFuncSetAttribute(bwd_main_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return record_cuda_error("cudaFuncSetAttribute(bwd_main)", e);
-    const int grid = B * Hkv * (S / kTileRows);
+    const int n_items = B * Hkv * (S / kTileRows);
+    const int grid = n_items < sms ? n_items : sms;  // persistent: one CTA per SM walks the item list
     if (ev_main_begin && (e = cudaEventRecord(ev_main_begin, stream)) != cudaSuccess)
         return record_cuda_error("cudaEventRecord", e);
     bwd_main_kernel<D><<<grid, kBwdThreads, smem, stream>>>(mq, mk, mv, mdo, prm);
