@@ -94,6 +94,32 @@ int lt_attn_bwd_profiled(const lt_half *Q, const lt_half *K, const lt_half *V,
                          void *workspace, size_t workspace_bytes, lt_stream_t stream,
                          lt_event_t main_begin, lt_event_t main_end);
 
+/* lt_attn_bwd for callers that cannot allocate device memory (the paper has no counterpart
+ * to this entry point).  Some hosts of this library may not call cudaMalloc at the point
+ * where they need the backward: code running inside a memory pool that must not grow, a
+ * plugin that is handed tensors but no allocator, a step that has to stay allocation-free
+ * after start-up.  For them the scratch that lt_attn_bwd takes as `workspace` comes from a
+ * fixed array of LT_ATTN_BWD_NOALLOC_MAX_SCRATCH_BYTES inside the library itself, which every
+ * GPU that loads the library holds until the process ends.  Inputs and outputs are still the
+ * caller's device tensors, with the meaning and layout of lt_attn_bwd.
+ *   - Shapes whose lt_attn_bwd_workspace_bytes() exceeds the built-in scratch (roughly
+ *     B*Hq*S*D above four million elements) return LT_ERR_WORKSPACE; lt_last_cuda_error()
+ *     then names both sizes.  Nothing is launched in that case.
+ *   - The call allocates nothing: no cudaMalloc/cudaFree and no allocating library routine.
+ *   - The first call on each device looks up the array's device address (one runtime query,
+ *     under a lock); make that first call before any CUDA stream capture begins.
+ *   - All calls on a device share the one scratch array.  Each call clears what it needs at
+ *     zero itself, so an earlier call's leftovers are harmless, but two calls that overlap
+ *     on the GPU (different streams) race on it: serialise them.
+ *   - A device-side wait that gave up cannot be read back through this entry point, since
+ *     the caller has no pointer to the scratch for lt_attn_check_status. */
+#define LT_ATTN_BWD_NOALLOC_MAX_SCRATCH_BYTES (18u * 1024u * 1024u)
+int lt_attn_bwd_noalloc(const lt_half *Q, const lt_half *K, const lt_half *V,
+                        const lt_half *O, const lt_half *dO, const float *LSE,
+                        lt_half *dQ, lt_half *dK, lt_half *dV,
+                        int B, int Hq, int Hkv, int S, int D, int causal, float scale,
+                        lt_stream_t stream);
+
 /* Same computation as lt_attn_fwd followed by lt_attn_bwd, but every tensor pointer is
  * a HOST pointer (pinned memory makes the copies asynchronous).  `arena` is a caller-
  * owned DEVICE buffer of at least lt_attn_host_arena_bytes() bytes, 256-byte aligned,

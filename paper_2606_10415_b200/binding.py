@@ -23,7 +23,7 @@ LT_ERR_DEVICE_TIMEOUT = 5
 
 EXPORTS = (
     "lt_attn_fwd_workspace_bytes", "lt_attn_bwd_workspace_bytes", "lt_attn_fwd", "lt_attn_bwd",
-    "lt_attn_bwd_profiled",
+    "lt_attn_bwd_profiled", "lt_attn_bwd_noalloc",
     "lt_attn_host_arena_bytes", "lt_attn_fwd_bwd_host", "lt_attn_check_status", "lt_status_string",
     "lt_last_cuda_error", "lt_attn_bwd_num_launches", "lt_attn_fwd_num_launches", "lt_dbg_tile_gemm",
 )
@@ -55,6 +55,8 @@ def _load() -> ctypes.CDLL:
     lib.lt_attn_bwd.restype = i
     lib.lt_attn_bwd_profiled.argtypes = [vp] * 9 + [i] * 6 + [f, vp, sz, vp, vp, vp]
     lib.lt_attn_bwd_profiled.restype = i
+    lib.lt_attn_bwd_noalloc.argtypes = [vp] * 9 + [i] * 6 + [f, vp]
+    lib.lt_attn_bwd_noalloc.restype = i
     lib.lt_attn_fwd_bwd_host.argtypes = [vp] * 9 + [i] * 6 + [f, vp, sz, vp]
     lib.lt_attn_fwd_bwd_host.restype = i
     lib.lt_attn_check_status.argtypes = [vp, vp]
@@ -166,6 +168,22 @@ def lt_attn_bwd_profiled(Q, K, V, O, dO, LSE, dQ, dK, dV, causal, scale, workspa
                                    workspace.numel() * workspace.element_size(), _stream_ptr(stream), e0, e1)
     if rc != LT_OK:
         raise LtError("lt_attn_bwd_profiled", rc)
+
+
+NOALLOC_MAX_SCRATCH_BYTES = 18 * 1024 * 1024
+
+
+def lt_attn_bwd_noalloc(Q, K, V, O, dO, LSE, dQ, dK, dV, causal, scale, stream=None) -> None:
+    """lt_attn_bwd without a workspace argument, for callers that may not allocate device memory:
+    the scratch is a fixed array inside the library (``NOALLOC_MAX_SCRATCH_BYTES``).  Raises
+    ``LtError`` with status ``LT_ERR_WORKSPACE`` when the shape needs more than that.  Calls on one
+    device share the array, so do not let two of them overlap on the GPU."""
+    _check_layout(Q, K, V, O, dO, LSE, dQ, dK, dV)
+    B, Hq, Hkv, S, D = _dims(Q, K)
+    rc = _lib.lt_attn_bwd_noalloc(_ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(dO), _ptr(LSE), _ptr(dQ), _ptr(dK),
+                                  _ptr(dV), B, Hq, Hkv, S, D, int(bool(causal)), float(scale), _stream_ptr(stream))
+    if rc != LT_OK:
+        raise LtError("lt_attn_bwd_noalloc", rc)
 
 
 def lt_attn_fwd_bwd_host(Q, K, V, dO, O, LSE, dQ, dK, dV, causal, scale, arena, stream=None) -> None:

@@ -28,6 +28,9 @@
 // the S^T and dP^T products by one extra 16-element contraction step whose operands are
 // (256, 1, 0...) and the (hi, lo, 0...) split of the term, so the softmax warps never
 // touch LSE or delta.
+#include <mutex>
+#include <stdio.h>
+
 #include "lt_common.cuh"
 #include "lt_host.h"
 
@@ -890,6 +893,64 @@ int lt_attn_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, const lt_h
                 int causal, float scale, void *workspace, size_t workspace_bytes, lt_stream_t stream) {
     return lt_attn_bwd_profiled(Q, K, V, O, dO, LSE, dQ, dK, dV, B, Hq, Hkv, S, D, causal, scale, workspace,
                                 workspace_bytes, stream, nullptr, nullptr);
+}
+
+}  // extern "C"
+
+// ----------------------------------------------------------------------------- backward without a caller workspace
+// Scratch for lt_attn_bwd_noalloc: lives in the library image, so every GPU that loads the
+// library carries these bytes until the process exits.  In host code the array's name is
+// only a handle for the runtime; the address the kernels need is fetched once per device
+// with cudaGetSymbolAddress.
+namespace lt {
+constexpr size_t kNoAllocScratchBytes = LT_ATTN_BWD_NOALLOC_MAX_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+constexpr int kNoAllocMaxDevices = 64;
+static void *g_noalloc_scratch_addr[kNoAllocMaxDevices];  // device address of the array, per device ordinal
+static std::mutex g_noalloc_mutex;
+}  // namespace lt
+
+extern "C" {
+
+int lt_attn_bwd_noalloc(const lt_half *Q, const lt_half *K, const lt_half *V, const lt_half *O, const lt_half *dO,
+                        const float *LSE, lt_half *dQ, lt_half *dK, lt_half *dV, int B, int Hq, int Hkv, int S, int D,
+                        int causal, float scale, lt_stream_t stream) {
+    using namespace lt;
+    if (!Q || !K || !V || !O || !dO || !LSE || !dQ || !dK || !dV) return LT_ERR_INVALID_ARG;
+    int rc = check_shape(B, Hq, Hkv, S, D, scale);
+    if (rc != LT_OK) return rc;
+    const size_t need = lt_attn_bwd_workspace_bytes(B, Hq, Hkv, S, D);
+    if (need == 0 || need > kNoAllocScratchBytes) {
+        char msg[160];
+        snprintf(msg, sizeof(msg), "this shape needs %zu bytes of scratch but the built-in scratch holds %zu; "
+                 "use lt_attn_bwd with a caller workspace", need, kNoAllocScratchBytes);
+        set_last_error("lt_attn_bwd_noalloc", msg);
+        return LT_ERR_WORKSPACE;
+    }
+    if ((rc = check_device()) != LT_OK) return rc;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return record_cuda_error("cudaGetDevice", e);
+    if (dev < 0 || dev >= kNoAllocMaxDevices) {
+        set_last_error("lt_attn_bwd_noalloc", "device ordinal out of range");
+        return LT_ERR_UNSUPPORTED;
+    }
+    void *scratch = nullptr;
+    {
+        // first call on this device: look the array's device address up (no allocation happens)
+        std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+        if (!g_noalloc_scratch_addr[dev]) {
+            void *addr = nullptr;
+            e = cudaGetSymbolAddress(&addr, g_noalloc_scratch);
+            if (e != cudaSuccess) return record_cuda_error("cudaGetSymbolAddress(scratch)", e);
+            g_noalloc_scratch_addr[dev] = addr;
+        }
+        scratch = g_noalloc_scratch_addr[dev];
+    }
+    // lt_attn_bwd clears the status block and its preprocess kernel zeroes the dQ accumulator on
+    // every call, so nothing left in the scratch by an earlier call is read
+    return lt_attn_bwd(Q, K, V, O, dO, LSE, dQ, dK, dV, B, Hq, Hkv, S, D, causal, scale, scratch,
+                       kNoAllocScratchBytes, stream);
 }
 
 }  // extern "C"
