@@ -34,6 +34,9 @@ from paper_2606_10415_b200 import workloads  # noqa: E402
 METRIC = "attention-backward TFLOP/s (causal FLOPs)"
 UNIT = "TFLOP/s"
 NOMINAL_FP16_TFLOPS = 2250.0  # datasheet dense figure, context only
+# dram__bytes_read.sum + dram__bytes_write.sum of one bwd_main_kernel launch, from the ncu capture
+# summarised in profiles/bwd_main_kernel_llama2_7b.md (taken on the full configuration itself)
+MAIN_KERNEL_DRAM_BYTES = {"llama2_7b": 652.2e6}
 FALLBACK_PEAK_TFLOPS = 1590.0
 
 
@@ -176,6 +179,22 @@ class ClockSampler:
         return out
 
 
+# ------------------------------------------------------------------ multi-process helpers
+
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
+    if dist is None:
+        return [float(v) for v in values]
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def job_throughput(flops_per_rank, world, seconds_per_step):
+    """Whole-job metric for replicas: every rank processes its own copy of the workload."""
+    return world * flops_per_rank / seconds_per_step / 1e12
+
+
 # ------------------------------------------------------------------ GPU arm
 
 def run_ours(args, cfg):
@@ -287,14 +306,11 @@ def run_ours(args, cfg):
     d2h = sum(t.numel() * t.element_size() for t in (hdQ, hdK, hdV))
     del hO, hL
 
-    if dist is not None:
-        tt = torch.tensor([total_ms, e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms = tt.tolist()
+    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], dist, "cuda")
 
     if rank == 0:
         ms_per_step = total_ms / args.steps
-        value = world * cfg.flops / (ms_per_step * 1e-3) / 1e12
+        value = job_throughput(cfg.flops, world, ms_per_step * 1e-3)
         peak, _hbm, peak_kind = measured_peak()
         main_avg_ms = sum(main_ms) / len(main_ms)
         achieved = cfg.flops / (main_avg_ms * 1e-3) / 1e12
@@ -310,12 +326,14 @@ def run_ours(args, cfg):
             "pct_of_nominal_fp16_peak": 100.0 * value / world / NOMINAL_FP16_TFLOPS,
             "peak_source": peak_kind,
             "clocks": clocks,
-            "e2e": {"value": world * cfg.flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
+            "e2e": {"value": job_throughput(cfg.flops, world, e2e_ms * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
                     "includes": "H2D copies, lt_attn_fwd, lt_attn_bwd, D2H copies"},
             "gpu_launches": args.steps * lt.lt_attn_bwd_num_launches(),
             "roofline": {"bound": "tensor", "kernel": "bwd_main_kernel", "achieved": achieved, "peak": peak,
-                         "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                         "unit": "TFLOP/s", "frac": achieved / peak,
+                         "traffic": MAIN_KERNEL_DRAM_BYTES.get(cfg.name), "traffic_unit": "bytes per launch (ncu)",
+                         "algorithmic_hbm_bytes": _step_bytes(cfg) - 4.0 * cfg.B * cfg.Hq * cfg.S * cfg.D,
                          "peak_source": peak_kind + " bf16 burst", "avg_launch_ms": main_avg_ms,
                          "best_launch_ms": min(main_ms)},
             "fwd": {"value": fwd_flops / (fwd_ms * 1e-3) / 1e12, "unit": UNIT, "ms": fwd_ms},
