@@ -49,7 +49,11 @@ enum {
 };
 
 // ----------------------------------------------------------------------------- preprocess
-// One half-warp (D = 128) or quarter-warp (D = 64) per row: 16-byte loads of dO and O.
+// One half-warp (D = 128) or quarter-warp (D = 64) per row, 16-byte loads of dO and O; each
+// warp works on kPreUnroll groups of rows at a time so that enough loads are in flight to
+// keep HBM busy.
+constexpr int kPreUnroll = 4;
+
 template <int D>
 __global__ void __launch_bounds__(256)
 bwd_preprocess_kernel(const __half *__restrict__ dO, const __half *__restrict__ O, const float *__restrict__ lse,
@@ -57,19 +61,32 @@ bwd_preprocess_kernel(const __half *__restrict__ dO, const __half *__restrict__ 
                       long long n_rows, float inv_scale, unsigned int *status) {
     constexpr int kLanesPerRow = D / 8;
     constexpr int kRowsPerWarp = 32 / kLanesPerRow;
+    constexpr int kRowsPerTrip = kRowsPerWarp * kPreUnroll;
     const int lane = threadIdx.x & 31;
     const int sub = lane % kLanesPerRow;
     const long long warp_global = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
     const long long n_warps = (static_cast<long long>(gridDim.x) * blockDim.x) >> 5;
     float max_abs_delta = 0.f, max_norm2 = 0.f;
-    for (long long row0 = warp_global * kRowsPerWarp; row0 < n_rows; row0 += n_warps * kRowsPerWarp) {
-        const long long row = row0 + lane / kLanesPerRow;
-        float acc = 0.f, n2 = 0.f;
-        if (row < n_rows) {
-            const uint4 a = __ldg(reinterpret_cast<const uint4 *>(dO + row * D) + sub);
-            const uint4 b = __ldg(reinterpret_cast<const uint4 *>(O + row * D) + sub);
-            const __half2 *ah = reinterpret_cast<const __half2 *>(&a);
-            const __half2 *bh = reinterpret_cast<const __half2 *>(&b);
+    for (long long row0 = warp_global * kRowsPerTrip; row0 < n_rows; row0 += n_warps * kRowsPerTrip) {
+        uint4 a[kPreUnroll], b[kPreUnroll];
+        float l[kPreUnroll];
+#pragma unroll
+        for (int u = 0; u < kPreUnroll; ++u) {
+            const long long row = row0 + u * kRowsPerWarp + lane / kLanesPerRow;
+            a[u] = b[u] = make_uint4(0u, 0u, 0u, 0u);
+            l[u] = 0.f;
+            if (row < n_rows) {
+                a[u] = __ldcs(reinterpret_cast<const uint4 *>(dO + row * D) + sub);
+                b[u] = __ldcs(reinterpret_cast<const uint4 *>(O + row * D) + sub);
+                if (sub == 0) l[u] = __ldg(lse + row);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kPreUnroll; ++u) {
+            const long long row = row0 + u * kRowsPerWarp + lane / kLanesPerRow;
+            const __half2 *ah = reinterpret_cast<const __half2 *>(&a[u]);
+            const __half2 *bh = reinterpret_cast<const __half2 *>(&b[u]);
+            float acc = 0.f, n2 = 0.f;
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const float2 x = __half22float2(ah[e]);
@@ -79,23 +96,23 @@ bwd_preprocess_kernel(const __half *__restrict__ dO, const __half *__restrict__ 
                 n2 = fmaf(x.x, x.x, n2);
                 n2 = fmaf(x.y, x.y, n2);
             }
-            float4 *z = reinterpret_cast<float4 *>(dq_acc + row * D) + sub * 2;
-            z[0] = make_float4(0.f, 0.f, 0.f, 0.f);
-            z[1] = make_float4(0.f, 0.f, 0.f, 0.f);
-        }
 #pragma unroll
-        for (int off = kLanesPerRow / 2; off > 0; off >>= 1) {
-            acc += __shfl_xor_sync(0xffffffffu, acc, off);
-            n2 += __shfl_xor_sync(0xffffffffu, n2, off);
-        }
-        if (row < n_rows) {
-            if (sub == 0) {
-                // operand rows of the main kernel's extra contraction step: 256*hi + lo = value
-                delta_ext[row] = make_uint4(split_hi_lo(-acc), 0u, 0u, 0u);
-                lse_ext[row] = make_uint4(split_hi_lo(-lse[row] * inv_scale), 0u, 0u, 0u);
+            for (int off = kLanesPerRow / 2; off > 0; off >>= 1) {
+                acc += __shfl_xor_sync(0xffffffffu, acc, off);
+                n2 += __shfl_xor_sync(0xffffffffu, n2, off);
             }
-            max_abs_delta = fmaxf(max_abs_delta, fabsf(acc));
-            max_norm2 = fmaxf(max_norm2, n2);
+            if (row < n_rows) {
+                float4 *z = reinterpret_cast<float4 *>(dq_acc + row * D) + sub * 2;
+                z[0] = make_float4(0.f, 0.f, 0.f, 0.f);
+                z[1] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (sub == 0) {
+                    // operand rows of the main kernel's extra contraction step: 256*hi + lo = value
+                    delta_ext[row] = make_uint4(split_hi_lo(-acc), 0u, 0u, 0u);
+                    lse_ext[row] = make_uint4(split_hi_lo(-l[u] * inv_scale), 0u, 0u, 0u);
+                }
+                max_abs_delta = fmaxf(max_abs_delta, fabsf(acc));
+                max_norm2 = fmaxf(max_norm2, n2);
+            }
         }
     }
 #pragma unroll
@@ -815,7 +832,7 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     }
-    constexpr int kRowsPerBlock = 8 * (32 / (D / 8));
+    constexpr int kRowsPerBlock = 8 * (32 / (D / 8)) * kPreUnroll;
     const long long want = (n_rows + kRowsPerBlock - 1) / kRowsPerBlock;
     const int pre_blocks = static_cast<int>(want < static_cast<long long>(sms) * 16 ? want : sms * 16);
     bwd_preprocess_kernel<D><<<pre_blocks, 256, 0, stream>>>(reinterpret_cast<const __half *>(dO),
