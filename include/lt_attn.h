@@ -161,6 +161,14 @@ int lt_attn_fwd_num_launches(void);
 int lt_dbg_tile_gemm(const lt_half *A, const lt_half *B, float *C, int mode,
                      void *workspace, size_t workspace_bytes, lt_stream_t stream);
 
+/* Failure-path check used by the tests (no counterpart in the paper): launches one small
+ * kernel whose threads wait on a barrier that nothing ever completes.  The wait is bounded
+ * (about 10 ms of cycles), after which the kernel records a code in the status block of
+ * `workspace` and returns normally; lt_attn_check_status then reports
+ * LT_ERR_DEVICE_TIMEOUT and the CUDA context stays usable.  This is the same give-up path
+ * every wait inside the attention kernels takes. */
+int lt_dbg_wait_timeout(void *workspace, size_t workspace_bytes, lt_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

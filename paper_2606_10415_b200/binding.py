@@ -26,6 +26,7 @@ EXPORTS = (
     "lt_attn_bwd_profiled", "lt_attn_bwd_noalloc",
     "lt_attn_host_arena_bytes", "lt_attn_fwd_bwd_host", "lt_attn_check_status", "lt_status_string",
     "lt_last_cuda_error", "lt_attn_bwd_num_launches", "lt_attn_fwd_num_launches", "lt_dbg_tile_gemm",
+    "lt_dbg_wait_timeout",
 )
 
 
@@ -69,6 +70,8 @@ def _load() -> ctypes.CDLL:
     lib.lt_attn_fwd_num_launches.restype = i
     lib.lt_dbg_tile_gemm.argtypes = [vp, vp, vp, i, vp, sz, vp]
     lib.lt_dbg_tile_gemm.restype = i
+    lib.lt_dbg_wait_timeout.argtypes = [vp, sz, vp]
+    lib.lt_dbg_wait_timeout.restype = i
     return lib
 
 
@@ -209,6 +212,12 @@ def lt_dbg_tile_gemm(A, B, C, mode, workspace, stream=None) -> None:
                                workspace.numel() * workspace.element_size(), _stream_ptr(stream))
     if rc != LT_OK:
         raise LtError("lt_dbg_tile_gemm", rc)
+
+
+def lt_dbg_wait_timeout(workspace, stream=None) -> None:
+    rc = _lib.lt_dbg_wait_timeout(_ptr(workspace), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    if rc != LT_OK:
+        raise LtError("lt_dbg_wait_timeout", rc)
 
 
 def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:

@@ -172,7 +172,48 @@ dbg_tile_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
 
+// A wait that nothing satisfies: exercises the bounded-wait path (no fault, no endless loop).
+__global__ void dbg_wait_timeout_kernel(unsigned int *status, long long limit_cycles) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(&bar, 1);
+        mbar_fence_init();
+    }
+    __syncthreads();
+    // nobody ever arrives on `bar`; thread 0 gives up after `limit_cycles`, the others follow its flag
+    const long long t0 = clock64();
+    bool ok = false;
+    uint32_t spins = 0;
+    while (!(ok = mbar_try_wait(&bar, 0))) {
+        if ((++spins & 63u) == 0u) {
+            if (*reinterpret_cast<volatile int *>(&abort_flag)) break;
+            if (threadIdx.x == 0 && clock64() - t0 > limit_cycles) {
+                abort_flag = 1;
+                atomicCAS(status + kStatusWordTimeout, 0u, 901u);
+                break;
+            }
+        }
+    }
+    __syncthreads();
+}
+
 }  // namespace lt
+
+extern "C" int lt_dbg_wait_timeout(void *workspace, size_t workspace_bytes, lt_stream_t stream) {
+    using namespace lt;
+    if (!workspace || !aligned256(workspace) || workspace_bytes < static_cast<size_t>(kStatusBytes))
+        return LT_ERR_WORKSPACE;
+    int rc = check_device();
+    if (rc != LT_OK) return rc;
+    cudaError_t e = cudaMemsetAsync(workspace, 0, kStatusBytes, stream);
+    if (e != cudaSuccess) return record_cuda_error("cudaMemsetAsync", e);
+    dbg_wait_timeout_kernel<<<1, 128, 0, stream>>>(reinterpret_cast<unsigned int *>(workspace), 20000000LL);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return record_cuda_error("dbg_wait_timeout_kernel launch", e);
+    return LT_OK;
+}
 
 extern "C" int lt_dbg_tile_gemm(const lt_half *A, const lt_half *B, float *C, int mode, void *workspace,
                                 size_t workspace_bytes, lt_stream_t stream) {

@@ -81,6 +81,20 @@ def test_tile_gemm_operand_conventions(lt, mode):
     assert err < (2e-2 if mode == 5 else 1e-3), f"mode {mode}: max abs error {err}"
 
 
+def test_bounded_wait_reports_timeout_and_context_survives(lt):
+    """A wait that nothing satisfies gives up, records its code, and the next call still works."""
+    ws = lt.alloc_workspace(256)
+    lt.lt_dbg_wait_timeout(ws)
+    assert lt.lt_attn_check_status(ws) == lt.LT_ERR_DEVICE_TIMEOUT
+    assert "901" in lt.last_cuda_error()
+    # the context is intact: a normal kernel runs and reports ok
+    A = torch.eye(128).half().cuda()
+    C = torch.zeros(128, 128, device="cuda")
+    lt.lt_dbg_tile_gemm(A, A, C, 0, ws)
+    assert lt.lt_attn_check_status(ws) == lt.LT_OK
+    assert torch.equal(C.cpu(), torch.eye(128))
+
+
 # ------------------------------------------------------------------ forward
 
 FWD_SHAPES = [
