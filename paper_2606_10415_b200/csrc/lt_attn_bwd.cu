@@ -14,14 +14,15 @@
 // across workers): here a CTA owns one key/value tile, keeps dK_j and dV_j resident in
 // tensor memory for the whole loop, and the cross-CTA reduction falls on dQ instead.
 //
-// The main kernel is persistent (one CTA per SM walks a list of work items, heavy ones first)
+// The main kernel is persistent (one CTA per SM claims work items, heavy ones first, from a counter)
 // and warp specialised (14 warps):
 //   warp 0       TMA producer (one thread): K_j, V_j once; then a two-stage ring of Q_i and a
 //                single-buffered dO_i; the warp also owns the tensor-memory allocation
 //   warp 1       tensor-core issuer (one thread)
 //   warps 2-9    softmax / dS warps: warps 2-5 take query columns 0-63 of a tile pair,
 //                warps 6-9 columns 64-127; each thread owns one key row
-//   warps 10-13  dQ reduction: tensor memory -> fp32 red.global into the accumulator
+//   warps 10-13  dQ reduction (tensor memory -> shared memory -> bulk add.f32 into the fp32
+//                accumulator) and the per-item dK/dV epilogue
 // Transposed scores are used (S^T = K Q^T, dP^T = V dO^T) so that P^T, written back to
 // tensor memory as fp16, is directly the A operand of dV += P^T dO; dS^T is written both to
 // tensor memory (A operand of dK += dS^T Q) and to shared memory (operand of the dQ product).  The row terms -LSE_i/scale and -delta_i are added inside
@@ -45,7 +46,7 @@ enum {
     kWaitKV = 201, kWaitStageEmpty = 202, kWaitStageFull = 203, kWaitSFull = 204, kWaitPReady = 205,
     kWaitDpFull = 206, kWaitDsReady = 207, kWaitDsFree = 208, kWaitDqFull = 209, kWaitDqEmpty = 210,
     kWaitDkvFull = 211, kWaitDoFull = 212, kWaitDoEmpty = 213, kWaitAccFree = 214, kWaitScale = 215,
-    kBadSmemAlign = 220
+    kWaitItem = 200, kBadSmemAlign = 220
 };
 
 // ----------------------------------------------------------------------------- preprocess
@@ -195,6 +196,7 @@ constexpr int kDqStageBufs = 3, kDqStageRows = 16;
 constexpr int kExtBytes = 2048;            // 128 rows x 16 bytes: one operand of the extra contraction step
 constexpr float kPScaleLog2Max = 14.f;     // P is kept as P * 2^c with c <= 14 so that fp16(P') <= 16384
 constexpr int kBarComputeWarps = 2, kBarReduceWarps = 1;  // named barrier ids
+constexpr int kItemRing = 4;  // roles are never more than two items apart
 
 template <int D>
 struct BwdSmem {
@@ -215,6 +217,9 @@ struct BwdSmem {
     float dq_stage[D == 128 ? kDqStageBufs : 1][D == 128 ? kDqStageRows * 128 : 4];
     // per work item: K/V landed; dK/dV accumulators complete; accumulators read out; scale published
     uint64_t bar_kv, bar_dkv_full, bar_acc_free, bar_scale_ready;
+    // work items are claimed from a global counter by the producer and published to the other roles
+    uint64_t bar_item[kItemRing];
+    int item_ring[kItemRing];
     // per (query head, query tile) iteration
     uint64_t bar_q_full[kQStages], bar_q_empty[kQStages], bar_do_full, bar_do_empty;
     uint64_t bar_s_full, bar_p_ready, bar_dp_full, bar_ds_ready, bar_ds_free, bar_dq_full, bar_dq_empty;
@@ -292,7 +297,8 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         if (!smem_ok) atomicCAS(p.status + kStatusWordTimeout, 0u, static_cast<unsigned int>(kBadSmemAlign));
         mbar_init(&sm.bar_kv, 1);
         mbar_init(&sm.bar_dkv_full, 1);
-        mbar_init(&sm.bar_acc_free, kNumComputeWarps);
+        mbar_init(&sm.bar_acc_free, kNumReduceWarps);
+        for (int r = 0; r < kItemRing; ++r) mbar_init(&sm.bar_item[r], 1);
         mbar_init(&sm.bar_scale_ready, 1);
         for (int s = 0; s < kQStages; ++s) {
             mbar_init(&sm.bar_q_full[s], 1);
@@ -346,8 +352,19 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             bool ok = true;
             int it = 0, ic = 0;
             int last_q = -1, last_do = -1, kv_loads = 0;  // for the cleanup after an abandoned wait
-            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++ic) {
+            // claim the next unclaimed item (heavy ones have the low numbers) and publish it to the
+            // other roles; -1 tells everybody that the list is exhausted
+            auto claim = [&](int slot_ic) -> int {
+                const unsigned int v = atomicAdd(p.status + kStatusWordItemCounter, 1u);
+                const int item = v < static_cast<unsigned int>(n_items) ? static_cast<int>(v) : -1;
+                sm.item_ring[slot_ic % kItemRing] = item;
+                mbar_arrive(&sm.bar_item[slot_ic % kItemRing]);
+                return item;
+            };
+            int item = claim(0);
+            while (item >= 0 && ok) {
                 const BwdItem w = bwd_item(p, item);
+                int next_item = -1;
                 for (int n = 0; n < w.n_iter && ok; ++n, ++it) {
                     const int s = it & 1, k = it >> 1;
                     const long long q_row0 = bwd_q_row(p, w, n);
@@ -379,7 +396,22 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         }
                         ++kv_loads;
                     }
+                    if (n == w.n_iter - 1) {
+                        // with the last query tile of this item on its way, claim the next item and ask for
+                        // its K/V tiles to be brought into L2 while this item finishes
+                        next_item = claim(ic + 1);
+                        if (next_item >= 0) {
+                            const BwdItem wn = bwd_item(p, next_item);
+#pragma unroll
+                            for (int x = 0; x < kBoxes; ++x) {
+                                tma_prefetch_l2_2d(&map_k, x * 64, wn.kv_row0);
+                                tma_prefetch_l2_2d(&map_v, x * 64, wn.kv_row0);
+                            }
+                        }
+                    }
                 }
+                item = next_item;
+                ++ic;
             }
             LT_TRACE_END(kRoleProducer);
             if (*abort_flag) {
@@ -416,7 +448,10 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             };
             bool ok = true;
             int it = 0, ic = 0;
-            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++ic) {
+            for (;; ++ic) {
+                if (!(ok = LT_WAIT(&sm.bar_item[ic % kItemRing], (ic / kItemRing) & 1, kWaitItem))) break;
+                const int item = sm.item_ring[ic % kItemRing];
+                if (item < 0) break;
                 const BwdItem w = bwd_item(p, item);
                 ok = LT_WAIT(&sm.bar_kv, ic & 1, kWaitKV) &&
                      LT_WAIT(&sm.bar_q_full[it & 1], (it >> 1) & 1, kWaitStageFull);
@@ -479,7 +514,8 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     umma_commit(&sm.bar_dq_full);
                     umma_commit(&sm.bar_ds_free);
                 }
-                if (ok) umma_commit(&sm.bar_dkv_full);
+                if (!ok) break;
+                umma_commit(&sm.bar_dkv_full);
             }
             LT_TRACE_END(kRoleMma);
         }
@@ -537,14 +573,17 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             return true;
         };
 
-        for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++ic) {
-            const BwdItem w = bwd_item(p, item);
+        for (;; ++ic) {
+            // (after an abandoned wait the loop still comes here, so that the vote below is never short of a warp)
+            ok = ok && LT_WAIT(&sm.bar_item[ic % kItemRing], (ic / kItemRing) & 1, kWaitItem);
+            const int item = ok ? sm.item_ring[ic % kItemRing] : -1;
+            const BwdItem w = bwd_item(p, item < 0 ? 0 : item);
             // ---- per item: a power-of-two factor 2^c carried by dS before it is rounded to fp16, chosen
             // from a bound on |dS| <= |dP| + |delta| <= max||dO_row|| * max||V_row|| + max|delta| so that
             // the scaled values use fp16's normal range without overflow.  The factor rides on P
             // (P' = P * 2^c, c <= 14); dV and dQ/dK undo it exactly in their epilogues.
-            ok = ok && LT_WAIT(&sm.bar_kv, ic & 1, kWaitKV);
-            if (ok && half_sel == 0) {
+            ok = ok && (item < 0 || LT_WAIT(&sm.bar_kv, ic & 1, kWaitKV));
+            if (ok && item >= 0 && half_sel == 0) {
                 float n2 = 0.f;
 #pragma unroll
                 for (int x = 0; x < kBoxes; ++x) {
@@ -567,7 +606,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             }
             // all eight warps vote here, also when leaving after an abandoned wait, so nobody is left behind
             ok = named_barrier_and(kBarComputeWarps, kNumComputeWarps * 32, ok);
-            if (!ok) break;
+            if (!ok || item < 0) break;  // every warp sees the same item, so they leave together
             {
                 const float *rd = sm.red[ic & 1];
                 const float vmax2 = fmaxf(fmaxf(rd[0], rd[1]), fmaxf(rd[2], rd[3]));
@@ -583,8 +622,6 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     mbar_arrive(&sm.bar_scale_ready);  // the reduction warps read it
                 }
             }
-            const float inv_p_scale = exp2f(-p_scale_log2);  // 2^-c, exact
-
             ok = compute_p(w, 0, it);
             for (int n = 0; n < w.n_iter && ok; ++n, ++it) {
                 if (!(ok = LT_WAIT(&sm.bar_dp_full, it & 1, kWaitDpFull))) break;
@@ -623,34 +660,6 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 if (n + 1 < w.n_iter) ok = compute_p(w, n + 1, it + 1);
             }
 
-            // epilogue: the first four softmax warps write dK_j, the other four dV_j; thread = key row
-            if (ok && (ok = LT_WAIT(&sm.bar_dkv_full, ic & 1, kWaitDkvFull))) {
-                tc_fence_after_sync();
-                const float mult = half_sel == 0 ? p.scale * inv_p_scale : inv_p_scale;
-                const uint32_t col0 = half_sel == 0 ? kColdK : kColdV;
-                __half *dst = (half_sel == 0 ? p.dK : p.dV) + (static_cast<long long>(w.kv_row0) + row) * D;
-#pragma unroll
-                for (int c = 0; c < D / 32; ++c) {
-                    uint32_t r[32];
-                    tmem_ld32(tmem + lane_base + col0 + c * 32, r);
-                    tmem_wait_ld();
-                    if (c == D / 32 - 1) {
-                        // the accumulators are in registers: the next item may overwrite them
-                        tc_fence_before_sync();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&sm.bar_acc_free);
-                    }
-#pragma unroll
-                    for (int v8 = 0; v8 < 4; ++v8) {
-                        uint4 o;
-                        o.x = pack_half2(__uint_as_float(r[8 * v8 + 0]) * mult, __uint_as_float(r[8 * v8 + 1]) * mult);
-                        o.y = pack_half2(__uint_as_float(r[8 * v8 + 2]) * mult, __uint_as_float(r[8 * v8 + 3]) * mult);
-                        o.z = pack_half2(__uint_as_float(r[8 * v8 + 4]) * mult, __uint_as_float(r[8 * v8 + 5]) * mult);
-                        o.w = pack_half2(__uint_as_float(r[8 * v8 + 6]) * mult, __uint_as_float(r[8 * v8 + 7]) * mult);
-                        reinterpret_cast<uint4 *>(dst + c * 32)[v8] = o;
-                    }
-                }
-            }
         }
         LT_TRACE_END(kRoleCompute);
     } else {
@@ -659,14 +668,22 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         bool ok = smem_ok;
         int it = 0, ic = 0;
         LT_TRACE_BEGIN();
-        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++ic) {
+        for (;; ++ic) {
+            // the four reduction warps share named barriers (D = 128), so after every wait they vote
+            // and leave together
+            ok = ok && LT_WAIT(&sm.bar_item[ic % kItemRing], (ic / kItemRing) & 1, kWaitItem);
+            if constexpr (D == 128) ok = named_barrier_and(kBarReduceWarps, kNumReduceWarps * 32, ok);
+            if (!ok) break;
+            const int item = sm.item_ring[ic % kItemRing];
+            if (item < 0) break;
             const BwdItem w = bwd_item(p, item);
-            float dq_mult = 0.f;
+            float dq_mult = 0.f, inv_p_scale = 0.f;
             for (int n = 0; n < w.n_iter; ++n, ++it) {
                 ok = LT_WAIT(&sm.bar_dq_full, it & 1, kWaitDqFull);
                 if (ok && n == 0) {
                     ok = LT_WAIT(&sm.bar_scale_ready, ic & 1, kWaitScale);
-                    dq_mult = p.scale * exp2f(-sm.p_scale[ic & 1]);
+                    inv_p_scale = exp2f(-sm.p_scale[ic & 1]);  // 2^-c, exact
+                    dq_mult = p.scale * inv_p_scale;
                 }
                 // the four reduction warps share named barriers below, so they leave the loop together;
                 // the vote also tells them that the staging buffers of the previous tile are free
@@ -765,6 +782,44 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     }
                 }
                 LT_TRACE_SINCE(13, tr0);
+            }
+            if (!ok) break;
+            // item epilogue (these warps are idle while the pipeline of the next item fills):
+            // dK_j and dV_j leave tensor memory as fp16; thread = key row
+            ok = LT_WAIT(&sm.bar_dkv_full, ic & 1, kWaitDkvFull);
+            if constexpr (D == 128) ok = named_barrier_and(kBarReduceWarps, kNumReduceWarps * 32, ok);
+            if (!ok) break;
+            tc_fence_after_sync();
+            {
+                const int row = quad * 32 + lane;
+                const uint32_t lane_base = static_cast<uint32_t>(quad * 32) << 16;
+#pragma unroll
+                for (int which = 0; which < 2; ++which) {
+                    const float mult = which == 0 ? dq_mult : inv_p_scale;
+                    const uint32_t col0 = which == 0 ? kColdK : kColdV;
+                    __half *dst = (which == 0 ? p.dK : p.dV) + (static_cast<long long>(w.kv_row0) + row) * D;
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t r[32];
+                        tmem_ld32(tmem + lane_base + col0 + c * 32, r);
+                        tmem_wait_ld();
+                        if (which == 1 && c == D / 32 - 1) {
+                            // both accumulators have been read: the next item may overwrite them
+                            tc_fence_before_sync();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&sm.bar_acc_free);
+                        }
+#pragma unroll
+                        for (int v8 = 0; v8 < 4; ++v8) {
+                            uint4 o;
+                            o.x = pack_half2(__uint_as_float(r[8 * v8 + 0]) * mult, __uint_as_float(r[8 * v8 + 1]) * mult);
+                            o.y = pack_half2(__uint_as_float(r[8 * v8 + 2]) * mult, __uint_as_float(r[8 * v8 + 3]) * mult);
+                            o.z = pack_half2(__uint_as_float(r[8 * v8 + 4]) * mult, __uint_as_float(r[8 * v8 + 5]) * mult);
+                            o.w = pack_half2(__uint_as_float(r[8 * v8 + 6]) * mult, __uint_as_float(r[8 * v8 + 7]) * mult);
+                            reinterpret_cast<uint4 *>(dst + c * 32)[v8] = o;
+                        }
+                    }
+                }
             }
         }
         // shared memory must stay valid until the bulk reductions have read it

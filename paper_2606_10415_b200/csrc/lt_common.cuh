@@ -17,6 +17,7 @@ constexpr int kStatusBytes = 256;
 constexpr int kStatusWordTimeout = 0;
 constexpr int kStatusWordMaxAbsDelta = 1;
 constexpr int kStatusWordMaxDoNorm2 = 2;
+constexpr int kStatusWordItemCounter = 3;  // next unclaimed work item of the backward main kernel
 
 // A wait gives up after this many clock cycles (about one second) ...
 constexpr long long kWaitLimitCycles = 2000000000LL;
@@ -111,6 +112,14 @@ __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, u
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y)
         : "memory");
+}
+
+// Ask for a 2-D tile to be brought into L2 ahead of the load that will use it.
+__device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap *map, int x, int y) {
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(
+                     reinterpret_cast<uint64_t>(map)),
+                 "r"(x), "r"(y)
+                 : "memory");
 }
 
 // 1-D bulk copy global -> shared (both 16-byte aligned, size a multiple of 16 bytes);
