@@ -429,21 +429,35 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         // ================================================================= tensor-core issuer
         if (lane == 0 && smem_ok) {
             LT_TRACE_BEGIN();
-            const uint32_t sK = smem_u32(sm.k), sV = smem_u32(sm.v), sdS = smem_u32(sm.ds), sdO = smem_u32(sm.d_o);
-            const uint32_t s_ones = smem_u32(sm.ext_ones), s_zero = smem_u32(sm.ext_zero);
-            const uint64_t desc_ones = desc_kmajor_noswz(s_ones, s_zero - s_ones, 128);
+            // Every operand descriptor is a base computed once plus a compile-time constant in its
+            // address field (bits 0-13, units of 16 bytes; shared memory stays below 256 KB, so the
+            // sum never carries out of the field): the issuing thread then spends two integer adds
+            // per product and the tensor pipe, not this thread, sets the pace.
+            const uint32_t s_zero = smem_u32(sm.ext_zero);
+            const uint64_t dK_k = desc_kmajor(smem_u32(sm.k)), dV_k = desc_kmajor(smem_u32(sm.v));
+            const uint64_t dK_mn = desc_mnmajor(smem_u32(sm.k), kBoxBytesBwd);
+            const uint64_t ddS_mn = desc_mnmajor(smem_u32(sm.ds), kBoxBytesBwd);
+            const uint64_t ddO_k = desc_kmajor(smem_u32(sm.d_o)), ddO_mn = desc_mnmajor(smem_u32(sm.d_o), kBoxBytesBwd);
+            const uint64_t dQ_k0 = desc_kmajor(smem_u32(sm.q[0])), dQ_mn0 = desc_mnmajor(smem_u32(sm.q[0]), kBoxBytesBwd);
+            constexpr uint64_t kQStageStep = static_cast<uint64_t>(Smem::kTile) >> 4;  // next Q stage
+            const uint64_t desc_ones = desc_kmajor_noswz(smem_u32(sm.ext_ones), s_zero - smem_u32(sm.ext_ones), 128);
             const uint64_t desc_ext_do = desc_kmajor_noswz(smem_u32(sm.ext_do), s_zero - smem_u32(sm.ext_do), 128);
+            const uint64_t desc_ext_q0 = desc_kmajor_noswz(smem_u32(sm.ext_q[0]), s_zero - smem_u32(sm.ext_q[0]), 128);
+            const uint64_t desc_ext_q1 = desc_kmajor_noswz(smem_u32(sm.ext_q[1]), s_zero - smem_u32(sm.ext_q[1]), 128);
+            // address-field increments of contraction step kk: within a contraction-contiguous tile
+            // (32 bytes per step, next 64-column tile after four steps) and within a row-contracted
+            // tile (16 rows of 128 bytes per step)
+            auto koff = [](int kk) -> uint64_t { return static_cast<uint64_t>((kk >> 2) * (kBoxBytesBwd >> 4) + (kk & 3) * 2); };
+            auto roff = [](int kk) -> uint64_t { return static_cast<uint64_t>(kk * (2048 >> 4)); };
             constexpr uint32_t idesc_s = make_idesc(128, 128, false, false);
             constexpr uint32_t idesc_dv = make_idesc(128, D, false, true);
             constexpr uint32_t idesc_dq = make_idesc(128, D == 128 ? 128 : D, true, true);
             auto issue_s = [&](int t) {  // S^T = K_j Q_i^T - LSE_i / scale, for running iteration t
-                const uint32_t sQn = smem_u32(sm.q[t & 1]), s_ext = smem_u32(sm.ext_q[t & 1]);
+                const uint64_t dQ_k = dQ_k0 + (t & 1) * kQStageStep;
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t koff = (kk >> 2) * kBoxBytesBwd + (kk & 3) * 32;
-                    umma_ss(tmem + kColS, desc_kmajor(sK + koff), desc_kmajor(sQn + koff), idesc_s, kk > 0);
-                }
-                umma_ss(tmem + kColS, desc_ones, desc_kmajor_noswz(s_ext, s_zero - s_ext, 128), idesc_s, 1);
+                for (int kk = 0; kk < D / 16; ++kk)
+                    umma_ss(tmem + kColS, dK_k + koff(kk), dQ_k + koff(kk), idesc_s, kk > 0);
+                umma_ss(tmem + kColS, desc_ones, (t & 1) ? desc_ext_q1 : desc_ext_q0, idesc_s, 1);
                 umma_commit(&sm.bar_s_full);
             };
             bool ok = true;
@@ -460,17 +474,15 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 issue_s(it);
                 for (int n = 0; n < w.n_iter && ok; ++n, ++it) {
                     const int s = it & 1;
-                    const uint32_t sQ = smem_u32(sm.q[s]);
+                    const uint64_t dQ_mn = dQ_mn0 + s * kQStageStep;
                     // dP^T = V_j dO_i^T - delta_i   (its columns held the previous dQ partial until the
                     //                                reduce warps drained it)
                     if (!(ok = LT_WAIT(&sm.bar_do_full, it & 1, kWaitDoFull))) break;
                     if (it > 0 && !(ok = LT_WAIT(&sm.bar_dq_empty, (it - 1) & 1, kWaitDqEmpty))) break;
                     tc_fence_after_sync();
 #pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk) {
-                        const uint32_t koff = (kk >> 2) * kBoxBytesBwd + (kk & 3) * 32;
-                        umma_ss(tmem + kColdP, desc_kmajor(sV + koff), desc_kmajor(sdO + koff), idesc_s, kk > 0);
-                    }
+                    for (int kk = 0; kk < D / 16; ++kk)
+                        umma_ss(tmem + kColdP, dV_k + koff(kk), ddO_k + koff(kk), idesc_s, kk > 0);
                     umma_ss(tmem + kColdP, desc_ones, desc_ext_do, idesc_s, 1);
                     umma_commit(&sm.bar_dp_full);
                     // dV_j += P'^T dO_i   (A = P'^T from tensor memory; query columns 0-63 sit at columns
@@ -481,8 +493,8 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     tc_fence_after_sync();
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk)
-                        umma_ts(tmem + kColdV, tmem + kColS + (kk >> 2) * 64 + (kk & 3) * 8,
-                                desc_mnmajor(sdO + kk * 2048, kBoxBytesBwd), idesc_dv, (n > 0) | (kk > 0));
+                        umma_ts(tmem + kColdV, tmem + kColS + (kk >> 2) * 64 + (kk & 3) * 8, ddO_mn + roff(kk), idesc_dv,
+                                (n > 0) | (kk > 0));
                     umma_commit(&sm.bar_do_empty);
                     // the next S^T overwrites P'^T; the tensor pipe executes in issue order
                     if (n + 1 < w.n_iter) {
@@ -495,8 +507,8 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     //                       0-63 at columns 0-31 and 64-127 at columns 64-95 of the dP region)
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk)
-                        umma_ts(tmem + kColdK, tmem + kColdP + (kk >> 2) * 64 + (kk & 3) * 8,
-                                desc_mnmajor(sQ + kk * 2048, kBoxBytesBwd), idesc_dv, (n > 0) | (kk > 0));
+                        umma_ts(tmem + kColdK, tmem + kColdP + (kk >> 2) * 64 + (kk & 3) * 8, dQ_mn + roff(kk), idesc_dv,
+                                (n > 0) | (kk > 0));
                     umma_commit(&sm.bar_q_empty[s]);
                     // dQ_i partial (contraction over key rows); it overwrites the dP columns, which is safe
                     // after dK because the tensor pipe executes in issue order.  For D = 128 it is
@@ -505,11 +517,9 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk) {
                         if constexpr (D == 128)
-                            umma_ss(tmem + kColdP, desc_mnmajor(sK + kk * 2048, kBoxBytesBwd),
-                                    desc_mnmajor(sdS + kk * 2048, kBoxBytesBwd), idesc_dq, kk > 0);
+                            umma_ss(tmem + kColdP, dK_mn + roff(kk), ddS_mn + roff(kk), idesc_dq, kk > 0);
                         else
-                            umma_ss(tmem + kColdP, desc_mnmajor(sdS + kk * 2048, kBoxBytesBwd),
-                                    desc_mnmajor(sK + kk * 2048, kBoxBytesBwd), idesc_dq, kk > 0);
+                            umma_ss(tmem + kColdP, ddS_mn + roff(kk), dK_mn + roff(kk), idesc_dq, kk > 0);
                     }
                     umma_commit(&sm.bar_dq_full);
                     umma_commit(&sm.bar_ds_free);
