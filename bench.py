@@ -45,7 +45,7 @@ def parse_args():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--config", default="llama2_7b", choices=sorted(workloads.CONFIGS))
+    ap.add_argument("--config", default="llama2_7b", choices=sorted(workloads.ALL_CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the timed oracle leg (profiling runs)")
     ap.add_argument("--clock-sample-ms", type=int, default=600,
@@ -359,7 +359,7 @@ def _step_bytes(cfg) -> float:
 
 def main():
     args = parse_args()
-    cfg = workloads.CONFIGS[args.config]
+    cfg = workloads.ALL_CONFIGS[args.config]
     if args.impl == "reference":
         run_reference(args, cfg)
     else:
