@@ -2,9 +2,16 @@
 // log-sum-exp.  It produces the forward state the backward needs (the paper's Algorithm 1
 // takes saved probability tiles; this library keeps LSE and rebuilds P in the backward).
 //
-// One CTA per (batch, query head, query tile).  S = Q_i K_j^T and O += P V_j run on
-// tcgen05 tensor cores; S and O live in tensor memory; each thread owns one query row
-// for the online softmax.
+// One CTA per (batch, query head, pair of neighbouring 128-row query tiles).  Warp 0 streams
+// K_j / V_j tiles with TMA through two-stage rings, warp 1 issues S = Q_i K_j^T and
+// O += P V_j on the tcgen05 tensor cores, and each query tile has its own group of four
+// softmax warps (one thread per query row), so that the tensor cores work on one tile of the
+// pair while the other tile's scores are exponentiated.  S/P and O live in tensor memory.
+// The running row maximum is only raised when it grew by more than 2^8 since the output
+// was last rescaled, so most key tiles need no pass over O.
+#include <algorithm>
+#include <type_traits>
+
 #include "lt_common.cuh"
 #include "lt_host.h"
 
@@ -14,16 +21,24 @@ constexpr int kFwdTileRows = 128;
 constexpr int kFwdBoxBytes = 128 * 128;
 constexpr float kFwdLog2e = 1.4426950408889634f;
 constexpr float kFwdLn2 = 0.6931471805599453f;
+constexpr int kFwdThreads = 320;              // producer warp, issuer warp, 2 x 4 softmax warps
+constexpr int kFwdSoftmaxWarp0 = 2;
+constexpr float kFwdRescaleLog2 = 8.f;        // P <= 2^8 stays far inside fp16 range
 
-enum { kWaitFwdQ = 301, kWaitFwdKV = 302, kWaitFwdS = 303, kWaitFwdO = 304 };
+enum {
+    kWaitFwdQ = 301, kWaitFwdK = 302, kWaitFwdV = 303, kWaitFwdS = 304, kWaitFwdP = 305,
+    kWaitFwdO = 306, kWaitFwdKEmpty = 307, kWaitFwdVEmpty = 308, kWaitFwdDone = 309
+};
 
 template <int D>
 struct __align__(1024) FwdSmem {
     static constexpr int kBoxes = D / 64;
-    uint8_t q[kBoxes * kFwdBoxBytes];
-    uint8_t k[kBoxes * kFwdBoxBytes];
-    uint8_t v[kBoxes * kFwdBoxBytes];
-    uint64_t bar_q, bar_kv, bar_mma;
+    static constexpr int kTile = kBoxes * kFwdBoxBytes;
+    uint8_t q[2][kTile];   // the pair's two query tiles
+    uint8_t k[2][kTile];   // ring of key tiles
+    uint8_t v[2][kTile];   // ring of value tiles
+    uint64_t bar_q[2], bar_k_full[2], bar_k_empty[2], bar_v_full[2], bar_v_empty[2];
+    uint64_t bar_s_full[2], bar_p_ready[2], bar_o_done[2], bar_done;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -36,36 +51,69 @@ struct FwdParams {
     float scale;
 };
 
+#ifdef LT_FWD_TRACE
+// Development build only: summed clock() intervals.  [0..7] issuer, [8..15] softmax lane 0 of
+// every warp, [16] tiles processed by softmax warps, [17] key tiles seen by issuers, [18] CTA cycles.
+__device__ unsigned long long g_fwd_trace[32];
+#define LT_FT_DECL uint32_t ft_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}; uint32_t ft_t = clock()
+#define LT_FT(slot) do { const uint32_t ft_n = clock(); ft_acc[slot] += ft_n - ft_t; ft_t = ft_n; } while (0)
+#define LT_FT_FLUSH(base) do { for (int ft_i = 0; ft_i < 8; ++ft_i) if (ft_acc[ft_i]) atomicAdd(&g_fwd_trace[(base) + ft_i], static_cast<unsigned long long>(ft_acc[ft_i])); } while (0)
+#define LT_FT_COUNT(slot, n) atomicAdd(&g_fwd_trace[slot], static_cast<unsigned long long>(n))
+#else
+#define LT_FT_DECL
+#define LT_FT(slot)
+#define LT_FT_FLUSH(base)
+#define LT_FT_COUNT(slot, n)
+#endif
+
+// Registers are handed out per four warps, so ten warps get the 168-register cap of twelve.
 template <int D>
-__global__ void __launch_bounds__(128, 1)
+__global__ void __launch_bounds__(kFwdThreads, 1)
 fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
            const __grid_constant__ CUtensorMap map_v, const FwdParams p) {
     using Smem = FwdSmem<D>;
     constexpr int kBoxes = D / 64;
-    constexpr uint32_t kTileBytes = kBoxes * kFwdBoxBytes;
-    constexpr uint32_t kTmemCols = 256;
-    constexpr uint32_t kColS = 0, kColO = 128;
+    constexpr uint32_t kTileBytes = Smem::kTile;
+    constexpr uint32_t kTmemCols = 512;
+    constexpr uint32_t kColS = 0;     // tile t: S / P at columns [128 t, 128 t + 128)
+    constexpr uint32_t kColO = 256;   // tile t: O at columns [256 + D t, 256 + D t + D)
 
     extern __shared__ uint8_t smem_raw[];
     Smem &sm = *reinterpret_cast<Smem *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
+    const int lane = tid & 31;
 
-    // heavy (large i) query tiles get the low block ids
+    // heavy (late) query-tile pairs get the low block ids
     const int n_tiles = p.S / kFwdTileRows;
+    const int n_pairs = (n_tiles + 1) / 2;
     const int n_bh = p.B * p.Hq;
-    const int i = p.causal ? (n_tiles - 1 - blockIdx.x / n_bh) : (blockIdx.x / n_bh);
+    const int pr = p.causal ? (n_pairs - 1 - blockIdx.x / n_bh) : (blockIdx.x / n_bh);
     const int bh = blockIdx.x % n_bh;
     const int b = bh / p.Hq;
     const int h = bh % p.Hq;
     const int g = h / (p.Hq / p.Hkv);
-    const int j_last = p.causal ? i : n_tiles - 1;
+    const int i0 = 2 * pr;
+    const bool has_b = (i0 + 1) < n_tiles;
+    // last key tile of query tile t; -1 when the pair has no second tile
+    const int j_last0 = p.causal ? i0 : n_tiles - 1;
+    const int j_last1 = has_b ? (p.causal ? i0 + 1 : n_tiles - 1) : -1;
+    const int j_end = j_last0 > j_last1 ? j_last0 : j_last1;
 
     if (tid == 0) {
         sm.abort_flag = 0;
-        mbar_init(&sm.bar_q, 1);
-        mbar_init(&sm.bar_kv, 1);
-        mbar_init(&sm.bar_mma, 1);
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(&sm.bar_q[t], 1);
+            mbar_init(&sm.bar_k_full[t], 1);
+            mbar_init(&sm.bar_k_empty[t], 1);
+            mbar_init(&sm.bar_v_full[t], 1);
+            mbar_init(&sm.bar_v_empty[t], 1);
+            mbar_init(&sm.bar_s_full[t], 1);
+            mbar_init(&sm.bar_p_ready[t], 128);
+            mbar_init(&sm.bar_o_done[t], 1);
+        }
+        mbar_init(&sm.bar_done, 1);
         mbar_fence_init();
         tma_prefetch_desc(&map_q);
         tma_prefetch_desc(&map_k);
@@ -79,150 +127,301 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = sm.tmem_base;
-    const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
     volatile int *abort_flag = &sm.abort_flag;
 
-    const long long q_row0 = static_cast<long long>(bh) * p.S + static_cast<long long>(i) * kFwdTileRows;
+    const long long q_row0 = static_cast<long long>(bh) * p.S + static_cast<long long>(i0) * kFwdTileRows;
     const long long kv_head_row0 = (static_cast<long long>(b) * p.Hkv + g) * p.S;
-    if (tid == 0) {
-        mbar_arrive_expect_tx(&sm.bar_q, kTileBytes);
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0) {
+            for (int t = 0; t < (has_b ? 2 : 1); ++t) {
+                mbar_arrive_expect_tx(&sm.bar_q[t], kTileBytes);
 #pragma unroll
-        for (int x = 0; x < kBoxes; ++x)
-            tma_load_2d(sm.q + x * kFwdBoxBytes, &map_q, &sm.bar_q, x * 64, static_cast<int>(q_row0));
-    }
-    bool ok = __syncthreads_and(mbar_wait(&sm.bar_q, 0, abort_flag, p.status, kWaitFwdQ));
-
-    const uint32_t sQ = smem_u32(sm.q), sK = smem_u32(sm.k), sV = smem_u32(sm.v);
-    constexpr uint32_t idesc_s = make_idesc(128, 128, false, false);
-    constexpr uint32_t idesc_o = make_idesc(128, D, false, true);
-    const float scale_log2 = p.scale * kFwdLog2e;
-
-    float m = -INFINITY;  // running row maximum of scale*log2(e)*score
-    float l = 0.f;        // running sum of exp2(score - m)
-    uint32_t phase_kv = 0, phase_mma = 0;
-
-    for (int j = 0; j <= j_last && ok; ++j) {
-        if (tid == 0) {
-            const int kv_row0 = static_cast<int>(kv_head_row0 + static_cast<long long>(j) * kFwdTileRows);
-            mbar_arrive_expect_tx(&sm.bar_kv, 2 * kTileBytes);
+                for (int x = 0; x < kBoxes; ++x)
+                    tma_load_2d(sm.q[t] + x * kFwdBoxBytes, &map_q, &sm.bar_q[t], x * 64,
+                                static_cast<int>(q_row0) + t * kFwdTileRows);
+            }
+            bool ok = true;
+            int armed = 0;  // key/value tiles whose loads were started
+            for (int j = 0; j <= j_end; ++j) {
+                const int s = j & 1;
+                const uint32_t ph = (j >> 1) & 1;
+                const int kv_row0 = static_cast<int>(kv_head_row0 + static_cast<long long>(j) * kFwdTileRows);
+                if (j >= 2 && !(ok = mbar_wait(&sm.bar_k_empty[s], ph ^ 1, abort_flag, p.status, kWaitFwdKEmpty))) break;
+                mbar_arrive_expect_tx(&sm.bar_k_full[s], kTileBytes);
 #pragma unroll
-            for (int x = 0; x < kBoxes; ++x) {
-                tma_load_2d(sm.k + x * kFwdBoxBytes, &map_k, &sm.bar_kv, x * 64, kv_row0);
-                tma_load_2d(sm.v + x * kFwdBoxBytes, &map_v, &sm.bar_kv, x * 64, kv_row0);
+                for (int x = 0; x < kBoxes; ++x)
+                    tma_load_2d(sm.k[s] + x * kFwdBoxBytes, &map_k, &sm.bar_k_full[s], x * 64, kv_row0);
+                if (j >= 2 && !(ok = mbar_wait(&sm.bar_v_empty[s], ph ^ 1, abort_flag, p.status, kWaitFwdVEmpty))) {
+                    // the key tile just started still has to land before shared memory is given up
+                    for (int w = 0; w < (1 << 16) && !mbar_try_wait(&sm.bar_k_full[s], ph); ++w) {}
+                    break;
+                }
+                mbar_arrive_expect_tx(&sm.bar_v_full[s], kTileBytes);
+#pragma unroll
+                for (int x = 0; x < kBoxes; ++x)
+                    tma_load_2d(sm.v[s] + x * kFwdBoxBytes, &map_v, &sm.bar_v_full[s], x * 64, kv_row0);
+                armed = j + 1;
+            }
+            if (!ok || *abort_flag) {
+                // somebody gave up: wait (bounded) for the copies in flight before the CTA exits
+                for (int t = 0; t < (has_b ? 2 : 1); ++t)
+                    for (int w = 0; w < (1 << 16) && !mbar_try_wait(&sm.bar_q[t], 0); ++w) {}
+                for (int j = armed > 2 ? armed - 2 : 0; j < armed; ++j) {
+                    for (int w = 0; w < (1 << 16) && !mbar_try_wait(&sm.bar_k_full[j & 1], (j >> 1) & 1); ++w) {}
+                    for (int w = 0; w < (1 << 16) && !mbar_try_wait(&sm.bar_v_full[j & 1], (j >> 1) & 1); ++w) {}
+                }
             }
         }
-        ok = __syncthreads_and(mbar_wait(&sm.bar_kv, phase_kv, abort_flag, p.status, kWaitFwdKV));
-        phase_kv ^= 1;
-        if (!ok) break;
-
-        if (tid == 0) {
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            // descriptors of slot 0; slot 1 of each ring follows one tile later
+            const uint64_t dQ0 = desc_kmajor(smem_u32(sm.q[0])), dK0 = desc_kmajor(smem_u32(sm.k[0]));
+            const uint64_t dV0 = desc_mnmajor(smem_u32(sm.v[0]), kFwdBoxBytes);
+            constexpr uint64_t kSlotStep = static_cast<uint64_t>(kTileBytes) >> 4;
+            auto koff = [](int kk) -> uint64_t { return static_cast<uint64_t>((kk >> 2) * (kFwdBoxBytes >> 4) + (kk & 3) * 2); };
+            auto roff = [](int kk) -> uint64_t { return static_cast<uint64_t>(kk * (2048 >> 4)); };
+            constexpr uint32_t idesc_s = make_idesc(128, 128, false, false);
+            constexpr uint32_t idesc_o = make_idesc(128, D, false, true);
+            auto issue_s = [&](int t, int s) {  // S_t = Q_t K^T with the key tile in ring slot s
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk)
+                    umma_ss(tmem + kColS + t * 128, dQ0 + t * kSlotStep + koff(kk), dK0 + s * kSlotStep + koff(kk), idesc_s, kk > 0);
+                umma_commit(&sm.bar_s_full[t]);
+            };
+            auto issue_pv = [&](int t, int s, bool acc) {  // O_t (+)= P_t V, P_t read from tensor memory
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)
+                    umma_ts(tmem + kColO + t * D, tmem + kColS + t * 128 + kk * 8, dV0 + s * kSlotStep + roff(kk), idesc_o,
+                            acc | (kk > 0));
+                umma_commit(&sm.bar_o_done[t]);
+            };
+            bool ok = mbar_wait(&sm.bar_q[0], 0, abort_flag, p.status, kWaitFwdQ) &&
+                      (!has_b || mbar_wait(&sm.bar_q[1], 0, abort_flag, p.status, kWaitFwdQ)) &&
+                      mbar_wait(&sm.bar_k_full[0], 0, abort_flag, p.status, kWaitFwdK);
+            if (ok) {
+                tc_fence_after_sync();
+                issue_s(0, 0);
+                if (has_b) issue_s(1, 0);
+                umma_commit(&sm.bar_k_empty[0]);
+            }
+            LT_FT_DECL;
+            for (int j = 0; j <= j_end && ok; ++j) {
+                const int s = j & 1, sn = s ^ 1;
+                LT_FT(0);
+                if (!(ok = mbar_wait(&sm.bar_v_full[s], (j >> 1) & 1, abort_flag, p.status, kWaitFwdV))) break;
+                LT_FT(1);
+                bool k_next_ready = false;
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    const int j_last_t = t == 0 ? j_last0 : j_last1;
+                    if (j > j_last_t) continue;
+                    LT_FT(0);
+                    if (!(ok = mbar_wait(&sm.bar_p_ready[t], j & 1, abort_flag, p.status, kWaitFwdP))) break;
+                    LT_FT(2 + t);
+                    tc_fence_after_sync();
+                    LT_FT(0);
+                    issue_pv(t, s, j > 0);
+                    LT_FT(5);
+                    // the second tile of the pair, when it uses this key tile, uses it last
+                    const int last_user = (j <= j_last1) ? 1 : 0;
+                    if (t == last_user) umma_commit(&sm.bar_v_empty[s]);
+                    if (j + 1 <= j_last_t) {
+                        if (!k_next_ready) {
+                            LT_FT(0);
+                            if (!(ok = mbar_wait(&sm.bar_k_full[sn], ((j + 1) >> 1) & 1, abort_flag, p.status, kWaitFwdK))) break;
+                            LT_FT(4);
+                            tc_fence_after_sync();
+                            k_next_ready = true;
+                        }
+                        LT_FT(0);
+                        issue_s(t, sn);
+                        LT_FT(6);
+                        const int last_user_next = (j + 1 <= j_last1) ? 1 : 0;
+                        if (t == last_user_next) umma_commit(&sm.bar_k_empty[sn]);
+                    }
+                }
+            }
+            LT_FT(0);
+            LT_FT_FLUSH(0);
+            LT_FT_COUNT(17, j_end + 1);
+            // every product issued above has finished before tensor memory is released
+            umma_commit(&sm.bar_done);
+            if (!mbar_wait(&sm.bar_done, 0, abort_flag, p.status, kWaitFwdDone))
+                for (int w = 0; w < (1 << 16) && !mbar_try_wait(&sm.bar_done, 0); ++w) {}
+        }
+    } else {
+        // ------------------------------------------------------------------ softmax warps
+        const int t = (warp - kFwdSoftmaxWarp0) >> 2;   // which query tile of the pair
+        const int quad = warp & 3;                      // tensor-memory lane quadrant of this warp
+        const int row = quad * 32 + lane;               // query row inside the tile
+        const int j_last = t == 0 ? j_last0 : j_last1;
+        const int i = i0 + t;
+        const uint32_t lane_base = static_cast<uint32_t>(quad * 32) << 16;
+        const uint32_t tS = tmem + lane_base + kColS + t * 128;
+        const uint32_t tO = tmem + lane_base + kColO + t * D;
+        const float scale_log2 = p.scale * kFwdLog2e;
+        float m_used = -INFINITY;  // the maximum the stored P, l and O are relative to
+        float l = 0.f;             // running sum of exp2(score - m_used)
+        bool ok = true;
+        LT_FT_DECL;
+        for (int j = 0; j <= j_last; ++j) {
+            LT_FT(0);
+            ok = mbar_wait(&sm.bar_s_full[t], j & 1, abort_flag, p.status, kWaitFwdS);
+            LT_FT(1);
+            if (!(ok = __all_sync(0xffffffffu, ok))) break;
             tc_fence_after_sync();
+            // the whole score row of this key tile stays in registers
+            uint32_t sc[128];
 #pragma unroll
-            for (int kk = 0; kk < D / 16; ++kk) {
-                const uint32_t koff = (kk >> 2) * kFwdBoxBytes + (kk & 3) * 32;
-                umma_ss(tmem + kColS, desc_kmajor(sQ + koff), desc_kmajor(sK + koff), idesc_s, kk > 0);
-            }
-            umma_commit(&sm.bar_mma);
-        }
-        ok = __syncthreads_and(mbar_wait(&sm.bar_mma, phase_mma, abort_flag, p.status, kWaitFwdS));
-        phase_mma ^= 1;
-        tc_fence_after_sync();
-        if (!ok) break;
-
-        // thread = query row `tid`; columns = the 128 keys of tile j
-        float s[128];
-        const bool diag = p.causal && (j == i);
-        float row_max = -INFINITY;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            uint32_t r[32];
-            tmem_ld32(tmem + lane_base + kColS + c * 32, r);
+            for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sc[c * 32]));
             tmem_wait_ld();
+            LT_FT(2);
+            float rs[4] = {0.f, 0.f, 0.f, 0.f};  // independent partial row sums
+            auto tile_softmax = [&](auto diag_tag) {
+                constexpr bool kDiag = decltype(diag_tag)::value;
+                // row extremum of the raw scores over the unmasked keys: the maximum of
+                // scale*log2(e)*score is that factor times the largest (smallest, for a negative
+                // scale) raw score
+                // (eight independent running extrema: one warp per scheduler has no other work to
+                // cover the latency of a dependent chain)
+                float ex[8];
+                if (scale_log2 >= 0.f) {
 #pragma unroll
-            for (int e = 0; e < 32; ++e) {
-                float x = __uint_as_float(r[e]) * scale_log2;
-                if (diag && (c * 32 + e) > tid) x = -INFINITY;
-                s[c * 32 + e] = x;
-                row_max = fmaxf(row_max, x);
-            }
+                    for (int u = 0; u < 8; ++u) ex[u] = -INFINITY;
+#pragma unroll
+                    for (int e = 0; e < 64; ++e) {  // two keys per step: a three-input maximum
+                        const float a = (!kDiag || e <= row) ? __uint_as_float(sc[e]) : -INFINITY;
+                        const float c = (!kDiag || e + 64 <= row) ? __uint_as_float(sc[e + 64]) : -INFINITY;
+                        ex[e & 7] = fmaxf(ex[e & 7], fmaxf(a, c));
+                    }
+#pragma unroll
+                    for (int u = 4; u > 0; u >>= 1)
+#pragma unroll
+                        for (int w = 0; w < u; ++w) ex[w] = fmaxf(ex[w], ex[w + u]);
+                } else {
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) ex[u] = INFINITY;
+#pragma unroll
+                    for (int e = 0; e < 64; ++e) {
+                        const float a = (!kDiag || e <= row) ? __uint_as_float(sc[e]) : INFINITY;
+                        const float c = (!kDiag || e + 64 <= row) ? __uint_as_float(sc[e + 64]) : INFINITY;
+                        ex[e & 7] = fminf(ex[e & 7], fminf(a, c));
+                    }
+#pragma unroll
+                    for (int u = 4; u > 0; u >>= 1)
+#pragma unroll
+                        for (int w = 0; w < u; ++w) ex[w] = fminf(ex[w], ex[w + u]);
+                }
+                const float ext = ex[0];
+                const float row_max = ext * scale_log2;
+                LT_FT(3);
+                if (j == 0) {
+                    m_used = row_max;  // key 0 is never masked, so this is finite for finite inputs
+                } else {
+                    const bool raise = (row_max - m_used) > kFwdRescaleLog2;
+                    if (__any_sync(0xffffffffu, raise)) {
+                        // O must hold every earlier product before it is rescaled
+                        ok = mbar_wait(&sm.bar_o_done[t], (j - 1) & 1, abort_flag, p.status, kWaitFwdO);
+                        if (!(ok = __all_sync(0xffffffffu, ok))) return;
+                        tc_fence_after_sync();
+                        const float alpha = raise ? fast_exp2(m_used - row_max) : 1.f;
+#pragma unroll
+                        for (int c = 0; c < D / 16; ++c) {  // narrow pieces: the score row holds most registers
+                            uint32_t r[16];
+                            tmem_ld16(tO + c * 16, r);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
+                            tmem_st16(tO + c * 16, r);
+                        }
+                        l *= alpha;
+                        if (raise) m_used = row_max;
+                    }
+                }
+                LT_FT(4);
+                // P = exp2(score - m_used) as fp16 over the first 64 columns of the S region
+                const float neg_m = -m_used;
+#pragma unroll
+                for (int e = 0; e < 128; ++e) {
+                    const float x = fmaf(__uint_as_float(sc[e]), scale_log2, neg_m);
+                    float pe = fast_exp2(x);
+                    if (kDiag && e > row) pe = 0.f;
+                    rs[e & 3] += pe;
+                    sc[e] = __float_as_uint(pe);
+                }
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t out[16];
+#pragma unroll
+                    for (int e = 0; e < 32; e += 2)
+                        out[e / 2] = pack_half2(__uint_as_float(sc[c * 32 + e]), __uint_as_float(sc[c * 32 + e + 1]));
+                    tmem_st16(tS + c * 16, out);
+                }
+            };
+            if (p.causal && j == i) tile_softmax(std::true_type{});
+            else tile_softmax(std::false_type{});
+            if (!ok) break;
+            const float row_sum = (rs[0] + rs[1]) + (rs[2] + rs[3]);
+            l += row_sum;
+            LT_FT(5);
+            tmem_wait_st();
+            tc_fence_before_sync();
+            mbar_arrive(&sm.bar_p_ready[t]);
+            LT_FT(6);
         }
-        const float m_new = fmaxf(m, row_max);
-        const float alpha = fast_exp2(m - m_new);  // 0 on the first tile (m = -inf)
-        float row_sum = 0.f;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            uint32_t out[16];
-#pragma unroll
-            for (int e = 0; e < 32; e += 2) {
-                const float p0 = fast_exp2(s[c * 32 + e] - m_new);
-                const float p1 = fast_exp2(s[c * 32 + e + 1] - m_new);
-                // sum the values the tensor core will see (fp16-rounded) so that O / l is consistent
-                const __half2 hp = __floats2half2_rn(p0, p1);
-                const float2 back = __half22float2(hp);
-                row_sum += back.x + back.y;
-                out[e / 2] = *reinterpret_cast<const uint32_t *>(&hp);
-            }
-            tmem_st16(tmem + lane_base + kColS + c * 16, out);
+#ifdef LT_FWD_TRACE
+        if (lane == 0) {
+            LT_FT_FLUSH(8);
+            LT_FT_COUNT(16, j_last + 1);
         }
-        l = l * alpha + row_sum;
-        m = m_new;
-        if (j > 0) {
-            // rescale the running output
+#endif
+
+        if (ok && j_last >= 0) {
+            ok = mbar_wait(&sm.bar_o_done[t], j_last & 1, abort_flag, p.status, kWaitFwdO);
+            ok = __all_sync(0xffffffffu, ok);
+        }
+        if (ok && j_last >= 0) {
+            tc_fence_after_sync();
+            const float inv_l = 1.f / l;
+            const long long q_row = q_row0 + static_cast<long long>(t) * kFwdTileRows + row;
+            __half *o_row = p.O + q_row * D;
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
                 uint32_t r[32];
-                tmem_ld32(tmem + lane_base + kColO + c * 32, r);
+                tmem_ld32(tO + c * 32, r);
                 tmem_wait_ld();
 #pragma unroll
-                for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
-                tmem_st32(tmem + lane_base + kColO + c * 32, r);
+                for (int v8 = 0; v8 < 4; ++v8) {
+                    uint4 o;
+                    o.x = pack_half2(__uint_as_float(r[8 * v8 + 0]) * inv_l, __uint_as_float(r[8 * v8 + 1]) * inv_l);
+                    o.y = pack_half2(__uint_as_float(r[8 * v8 + 2]) * inv_l, __uint_as_float(r[8 * v8 + 3]) * inv_l);
+                    o.z = pack_half2(__uint_as_float(r[8 * v8 + 4]) * inv_l, __uint_as_float(r[8 * v8 + 5]) * inv_l);
+                    o.w = pack_half2(__uint_as_float(r[8 * v8 + 6]) * inv_l, __uint_as_float(r[8 * v8 + 7]) * inv_l);
+                    reinterpret_cast<uint4 *>(o_row + c * 32)[v8] = o;
+                }
             }
+            p.lse[q_row] = (m_used + log2f(l)) * kFwdLn2;
         }
-        tmem_wait_st();
-        tc_fence_before_sync();
-        __syncthreads();
-
-        if (tid == 0) {
-            tc_fence_after_sync();
-            // O += P V_j   (A = P from tensor memory, contraction over the key rows of V)
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk)
-                umma_ts(tmem + kColO, tmem + kColS + kk * 8, desc_mnmajor(sV + kk * 2048, kFwdBoxBytes), idesc_o,
-                        (j > 0) | (kk > 0));
-            umma_commit(&sm.bar_mma);
-        }
-        ok = __syncthreads_and(mbar_wait(&sm.bar_mma, phase_mma, abort_flag, p.status, kWaitFwdO));
-        phase_mma ^= 1;
-        tc_fence_after_sync();
     }
 
-    if (ok) {
-        const float inv_l = 1.f / l;
-        __half *o_row = p.O + (q_row0 + tid) * D;
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-            uint32_t r[32];
-            tmem_ld32(tmem + lane_base + kColO + c * 32, r);
-            tmem_wait_ld();
-#pragma unroll
-            for (int v8 = 0; v8 < 4; ++v8) {
-                uint4 o;
-                o.x = pack_half2(__uint_as_float(r[8 * v8 + 0]) * inv_l, __uint_as_float(r[8 * v8 + 1]) * inv_l);
-                o.y = pack_half2(__uint_as_float(r[8 * v8 + 2]) * inv_l, __uint_as_float(r[8 * v8 + 3]) * inv_l);
-                o.z = pack_half2(__uint_as_float(r[8 * v8 + 4]) * inv_l, __uint_as_float(r[8 * v8 + 5]) * inv_l);
-                o.w = pack_half2(__uint_as_float(r[8 * v8 + 6]) * inv_l, __uint_as_float(r[8 * v8 + 7]) * inv_l);
-                reinterpret_cast<uint4 *>(o_row + c * 32)[v8] = o;
-            }
-        }
-        p.lse[q_row0 + tid] = (m + log2f(l)) * kFwdLn2;
-    } else if (tid == 0) {
-        for (int t = 0; t < (1 << 16) && !mbar_try_wait(&sm.bar_q, 0); ++t) {}
-        for (int t = 0; t < (1 << 16) && !mbar_try_wait(&sm.bar_kv, phase_kv ^ 1); ++t) {}
-    }
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
+
+#ifdef LT_FWD_TRACE
+extern "C" int lt_dbg_fwd_trace(unsigned long long *out, int reset) {
+    if (out && cudaMemcpyFromSymbol(out, g_fwd_trace, sizeof(g_fwd_trace)) != cudaSuccess) return LT_ERR_CUDA;
+    if (reset) {
+        static unsigned long long zeros[32];
+        if (cudaMemcpyToSymbol(g_fwd_trace, zeros, sizeof(zeros)) != cudaSuccess) return LT_ERR_CUDA;
+    }
+    return LT_OK;
+}
+#endif
 
 template <int D>
 static int launch_fwd(const lt_half *Q, const lt_half *K, const lt_half *V, lt_half *O, float *LSE, int B, int Hq,
@@ -240,11 +439,13 @@ static int launch_fwd(const lt_half *Q, const lt_half *K, const lt_half *V, lt_h
     prm.status = reinterpret_cast<unsigned int *>(workspace);
     prm.B = B; prm.Hq = Hq; prm.Hkv = Hkv; prm.S = S; prm.causal = causal ? 1 : 0;
     prm.scale = scale;
-    const size_t smem = sizeof(FwdSmem<D>) + 1024;
+    // at least 120 KB, so that one CTA (which takes all 512 tensor-memory columns) lives on an SM
+    const size_t smem = std::max<size_t>(sizeof(FwdSmem<D>) + 1024, 120 * 1024);
     e = cudaFuncSetAttribute(fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return record_cuda_error("cudaFuncSetAttribute(fwd)", e);
-    const int grid = B * Hq * (S / kFwdTileRows);
-    fwd_kernel<D><<<grid, 128, smem, stream>>>(mq, mk, mv, prm);
+    const int n_tiles = S / kFwdTileRows;
+    const int grid = B * Hq * ((n_tiles + 1) / 2);
+    fwd_kernel<D><<<grid, kFwdThreads, smem, stream>>>(mq, mk, mv, prm);
     e = cudaGetLastError();
     if (e != cudaSuccess) return record_cuda_error("fwd_kernel launch", e);
     return LT_OK;
