@@ -14,7 +14,8 @@
  *     dK and dV are summed over the Hq / Hkv query heads of a group.
  *   - scores = scale * Q K^T with a finite, non-zero scale; causal != 0 hides key j from query i when j > i.
  *     LSE_i = ln sum_j exp(scores_ij) over visible keys (natural logarithm).
- *   - Supported shapes: D in {64, 128}, S a positive multiple of 128, Hq % Hkv == 0.
+ *   - Supported shapes: D in {64, 128}, any S >= 1 (a last tile of fewer than 128 rows is
+ *     handled inside the kernels; workspace arrays are sized for S rounded up to 128), Hq % Hkv == 0.
  *     Anything else returns LT_ERR_UNSUPPORTED and launches nothing.
  *   - Unless a function says otherwise pointers are DEVICE pointers, 16-byte aligned,
  *     owned by the caller, and must stay valid until the stream reaches the end of the

@@ -59,7 +59,9 @@ template <int D>
 __global__ void __launch_bounds__(256)
 bwd_preprocess_kernel(const __half *__restrict__ dO, const __half *__restrict__ O, const float *__restrict__ lse,
                       uint4 *__restrict__ delta_ext, uint4 *__restrict__ lse_ext, float *__restrict__ dq_acc,
-                      long long n_rows, float inv_scale, unsigned int *status) {
+                      long long n_rows, int S, int S_pad, float inv_scale, unsigned int *status) {
+    // `n_rows` counts rows of the padded row space (every head rounded up to S_pad rows), the
+    // indexing of delta_ext, lse_ext and dq_acc; padding rows get zeros everywhere.
     constexpr int kLanesPerRow = D / 8;
     constexpr int kRowsPerWarp = 32 / kLanesPerRow;
     constexpr int kRowsPerTrip = kRowsPerWarp * kPreUnroll;
@@ -76,10 +78,16 @@ bwd_preprocess_kernel(const __half *__restrict__ dO, const __half *__restrict__ 
             const long long row = row0 + u * kRowsPerWarp + lane / kLanesPerRow;
             a[u] = b[u] = make_uint4(0u, 0u, 0u, 0u);
             l[u] = 0.f;
-            if (row < n_rows) {
-                a[u] = __ldcs(reinterpret_cast<const uint4 *>(dO + row * D) + sub);
-                b[u] = __ldcs(reinterpret_cast<const uint4 *>(O + row * D) + sub);
-                if (sub == 0) l[u] = __ldg(lse + row);
+            long long src = row;  // row of dO / O / LSE behind padded row `row`, -1 for padding
+            if (S != S_pad) {
+                const long long head = row / S_pad;
+                const int s_in = static_cast<int>(row - head * S_pad);
+                src = s_in < S ? head * S + s_in : -1;
+            }
+            if (row < n_rows && src >= 0) {
+                a[u] = __ldcs(reinterpret_cast<const uint4 *>(dO + src * D) + sub);
+                b[u] = __ldcs(reinterpret_cast<const uint4 *>(O + src * D) + sub);
+                if (sub == 0) l[u] = __ldg(lse + src);
             }
         }
 #pragma unroll
@@ -130,11 +138,18 @@ bwd_preprocess_kernel(const __half *__restrict__ dO, const __half *__restrict__ 
 
 // ----------------------------------------------------------------------------- finalize
 __global__ void __launch_bounds__(256)
-bwd_finalize_kernel(const float *__restrict__ dq_acc, __half *__restrict__ dQ, long long n_vec8) {
+bwd_finalize_kernel(const float *__restrict__ dq_acc, __half *__restrict__ dQ, long long n_vec8, int vec_per_head,
+                    int vec_per_padded_head) {
+    // n_vec8 groups of eight output elements; the accumulator is indexed in the padded row space
     const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
     for (long long v = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; v < n_vec8; v += stride) {
-        const float4 a = __ldcs(reinterpret_cast<const float4 *>(dq_acc) + 2 * v);
-        const float4 b = __ldcs(reinterpret_cast<const float4 *>(dq_acc) + 2 * v + 1);
+        long long src = v;
+        if (vec_per_head != vec_per_padded_head) {
+            const long long head = v / vec_per_head;
+            src = head * vec_per_padded_head + (v - head * vec_per_head);
+        }
+        const float4 a = __ldcs(reinterpret_cast<const float4 *>(dq_acc) + 2 * src);
+        const float4 b = __ldcs(reinterpret_cast<const float4 *>(dq_acc) + 2 * src + 1);
         uint4 o;
         o.x = pack_half2(a.x, a.y);
         o.y = pack_half2(a.z, a.w);
@@ -238,18 +253,18 @@ struct BwdParams {
     __half *dK;
     __half *dV;
     unsigned int *status;
-    int B, Hq, Hkv, S, causal;
+    int B, Hq, Hkv, S, S_pad, causal;  // S_pad: S rounded up to whole 128-row tiles
     float scale;
 };
 
 // One work item = key tile j of (batch b, kv head g).  Items are numbered so that the heavy
 // ones (small j under a causal mask) come first; CTA c takes items c, c + gridDim.x, ...
 struct BwdItem {
-    int j, b, g, i_first, tiles_per_head, n_iter, kv_row0;
+    int j, b, g, i_first, tiles_per_head, n_iter, kv_head;
 };
 __device__ __forceinline__ BwdItem bwd_item(const BwdParams &p, int item) {
     BwdItem w;
-    const int n_tiles = p.S / kTileRows;
+    const int n_tiles = (p.S + kTileRows - 1) / kTileRows;  // the last tile may be ragged
     const int n_bg = p.B * p.Hkv;
     w.j = item / n_bg;
     const int bg = item - w.j * n_bg;
@@ -258,15 +273,24 @@ __device__ __forceinline__ BwdItem bwd_item(const BwdParams &p, int item) {
     w.i_first = p.causal ? w.j : 0;
     w.tiles_per_head = n_tiles - w.i_first;
     w.n_iter = (p.Hq / p.Hkv) * w.tiles_per_head;  // flattened (query head of the group, query tile) loop
-    w.kv_row0 = (w.b * p.Hkv + w.g) * p.S + w.j * kTileRows;
+    w.kv_head = w.b * p.Hkv + w.g;
     return w;
 }
-// iteration n of an item -> first row of its query tile in the [B*Hq*S, D] view
-__device__ __forceinline__ long long bwd_q_row(const BwdParams &p, const BwdItem &w, int n) {
+// Iteration n of an item -> its query tile: flattened (batch, query head) index, first row
+// inside the head, and the tile's first row in the padded row space of the workspace arrays
+// (every head rounded up to whole tiles, so tiles never straddle heads).
+struct BwdQTile {
+    int head, s0;
+    long long padded_row0;
+};
+__device__ __forceinline__ BwdQTile bwd_q_tile(const BwdParams &p, const BwdItem &w, int n) {
     const int hh = n / w.tiles_per_head;
     const int i = w.i_first + (n - hh * w.tiles_per_head);
-    return (static_cast<long long>(w.b) * p.Hq + w.g * (p.Hq / p.Hkv) + hh) * p.S +
-           static_cast<long long>(i) * kTileRows;
+    BwdQTile q;
+    q.head = w.b * p.Hq + w.g * (p.Hq / p.Hkv) + hh;
+    q.s0 = i * kTileRows;
+    q.padded_row0 = static_cast<long long>(q.head) * p.S_pad + q.s0;
+    return q;
 }
 
 template <int D>
@@ -288,7 +312,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
     const int lane = tid & 31;
-    const int n_items = (p.S / kTileRows) * p.B * p.Hkv;
+    const int n_items = (p.S_pad / kTileRows) * p.B * p.Hkv;
 
     // the swizzled tiles need 1024-byte alignment; the shared window is expected to give it
     const bool smem_ok = (smem_u32(smem_raw) & 1023u) == 0u;
@@ -367,22 +391,20 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 int next_item = -1;
                 for (int n = 0; n < w.n_iter && ok; ++n, ++it) {
                     const int s = it & 1, k = it >> 1;
-                    const long long q_row0 = bwd_q_row(p, w, n);
+                    const BwdQTile qt = bwd_q_tile(p, w, n);
                     if (k >= 1 && !(ok = LT_WAIT(&sm.bar_q_empty[s], (k - 1) & 1, kWaitStageEmpty))) break;
                     mbar_arrive_expect_tx(&sm.bar_q_full[s], kTileBytes + kExtBytes);
 #pragma unroll
                     for (int x = 0; x < kBoxes; ++x)
-                        tma_load_2d(sm.q[s] + x * kBoxBytesBwd, &map_q, &sm.bar_q_full[s], x * 64,
-                                    static_cast<int>(q_row0));
-                    bulk_load_1d(sm.ext_q[s], p.lse_ext + q_row0, kExtBytes, &sm.bar_q_full[s]);
+                        tma_load_3d(sm.q[s] + x * kBoxBytesBwd, &map_q, &sm.bar_q_full[s], x * 64, qt.s0, qt.head);
+                    bulk_load_1d(sm.ext_q[s], p.lse_ext + qt.padded_row0, kExtBytes, &sm.bar_q_full[s]);
                     last_q = it;
                     if (it >= 1 && !(ok = LT_WAIT(&sm.bar_do_empty, (it - 1) & 1, kWaitDoEmpty))) break;
                     mbar_arrive_expect_tx(&sm.bar_do_full, kTileBytes + kExtBytes);
 #pragma unroll
                     for (int x = 0; x < kBoxes; ++x)
-                        tma_load_2d(sm.d_o + x * kBoxBytesBwd, &map_do, &sm.bar_do_full, x * 64,
-                                    static_cast<int>(q_row0));
-                    bulk_load_1d(sm.ext_do, p.delta_ext + q_row0, kExtBytes, &sm.bar_do_full);
+                        tma_load_3d(sm.d_o + x * kBoxBytesBwd, &map_do, &sm.bar_do_full, x * 64, qt.s0, qt.head);
+                    bulk_load_1d(sm.ext_do, p.delta_ext + qt.padded_row0, kExtBytes, &sm.bar_do_full);
                     last_do = it;
                     if (n == 0) {
                         // K_j and V_j follow the first query tile: they may only be overwritten once every
@@ -391,8 +413,8 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         mbar_arrive_expect_tx(&sm.bar_kv, 2 * kTileBytes);
 #pragma unroll
                         for (int x = 0; x < kBoxes; ++x) {
-                            tma_load_2d(sm.k + x * kBoxBytesBwd, &map_k, &sm.bar_kv, x * 64, w.kv_row0);
-                            tma_load_2d(sm.v + x * kBoxBytesBwd, &map_v, &sm.bar_kv, x * 64, w.kv_row0);
+                            tma_load_3d(sm.k + x * kBoxBytesBwd, &map_k, &sm.bar_kv, x * 64, w.j * kTileRows, w.kv_head);
+                            tma_load_3d(sm.v + x * kBoxBytesBwd, &map_v, &sm.bar_kv, x * 64, w.j * kTileRows, w.kv_head);
                         }
                         ++kv_loads;
                     }
@@ -404,8 +426,8 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                             const BwdItem wn = bwd_item(p, next_item);
 #pragma unroll
                             for (int x = 0; x < kBoxes; ++x) {
-                                tma_prefetch_l2_2d(&map_k, x * 64, wn.kv_row0);
-                                tma_prefetch_l2_2d(&map_v, x * 64, wn.kv_row0);
+                                tma_prefetch_l2_3d(&map_k, x * 64, wn.j * kTileRows, wn.kv_head);
+                                tma_prefetch_l2_3d(&map_v, x * 64, wn.j * kTileRows, wn.kv_head);
                             }
                         }
                     }
@@ -566,6 +588,12 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 for (int e = 0; e < 64; ++e)
                     if (row > static_cast<int>(cbase) + e) pv[e] = 0u;
             }
+            if (w.j * kTileRows + row >= p.S) {
+                // a key row past the end of the sequence (ragged last tile): its zero-filled K row has
+                // score 0, which LSE does not bound, so its P is not a probability; hide it
+#pragma unroll
+                for (int e = 0; e < 64; ++e) pv[e] = 0u;
+            }
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
                 uint32_t out[16];
@@ -701,7 +729,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 if (!ok) break;
                 tc_fence_after_sync();
                 LT_TRACE_MARK(tr0);
-                float *dq_tile = p.dq_acc + bwd_q_row(p, w, n) * D;
+                float *dq_tile = p.dq_acc + bwd_q_tile(p, w, n).padded_row0 * D;
                 if constexpr (D == 128) {
                     // dQ^T: this thread holds head-dim element d = 32*quad + lane of all 128 query rows.
                     // Sixteen query rows at a time are scaled, staged in shared memory exactly as they lie
@@ -807,7 +835,8 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 for (int which = 0; which < 2; ++which) {
                     const float mult = which == 0 ? dq_mult : inv_p_scale;
                     const uint32_t col0 = which == 0 ? kColdK : kColdV;
-                    __half *dst = (which == 0 ? p.dK : p.dV) + (static_cast<long long>(w.kv_row0) + row) * D;
+                    const int s_row = w.j * kTileRows + row;  // rows past S are never stored
+                    __half *dst = (which == 0 ? p.dK : p.dV) + (static_cast<long long>(w.kv_head) * p.S + s_row) * D;
 #pragma unroll
                     for (int c = 0; c < D / 32; ++c) {
                         uint32_t r[32];
@@ -826,7 +855,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                             o.y = pack_half2(__uint_as_float(r[8 * v8 + 2]) * mult, __uint_as_float(r[8 * v8 + 3]) * mult);
                             o.z = pack_half2(__uint_as_float(r[8 * v8 + 4]) * mult, __uint_as_float(r[8 * v8 + 5]) * mult);
                             o.w = pack_half2(__uint_as_float(r[8 * v8 + 6]) * mult, __uint_as_float(r[8 * v8 + 7]) * mult);
-                            reinterpret_cast<uint4 *>(dst + c * 32)[v8] = o;
+                            if (s_row < p.S) reinterpret_cast<uint4 *>(dst + c * 32)[v8] = o;
                         }
                     }
                 }
@@ -873,7 +902,8 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
                       const float *LSE, lt_half *dQ, lt_half *dK, lt_half *dV, int B, int Hq, int Hkv, int S,
                       int causal, float scale, void *workspace, cudaStream_t stream, cudaEvent_t ev_main_begin,
                       cudaEvent_t ev_main_end) {
-    const long long n_rows = static_cast<long long>(B) * Hq * S;
+    const int S_pad = static_cast<int>(padded_rows(S));
+    const long long n_rows = static_cast<long long>(B) * Hq * S_pad;  // padded row space of the workspace arrays
     uint8_t *ws = static_cast<uint8_t *>(workspace);
     unsigned int *status = reinterpret_cast<unsigned int *>(ws);
     const size_t ext_bytes = round256(static_cast<size_t>(n_rows) * 16);
@@ -883,10 +913,10 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
 
     CUtensorMap mq, mk, mv, mdo;
     int rc;
-    if ((rc = make_tile_map(&mq, Q, n_rows, D, 128)) != LT_OK) return rc;
-    if ((rc = make_tile_map(&mdo, dO, n_rows, D, 128)) != LT_OK) return rc;
-    if ((rc = make_tile_map(&mk, K, static_cast<uint64_t>(B) * Hkv * S, D, 128)) != LT_OK) return rc;
-    if ((rc = make_tile_map(&mv, V, static_cast<uint64_t>(B) * Hkv * S, D, 128)) != LT_OK) return rc;
+    if ((rc = make_head_map(&mq, Q, static_cast<uint64_t>(B) * Hq, S, D, 128)) != LT_OK) return rc;
+    if ((rc = make_head_map(&mdo, dO, static_cast<uint64_t>(B) * Hq, S, D, 128)) != LT_OK) return rc;
+    if ((rc = make_head_map(&mk, K, static_cast<uint64_t>(B) * Hkv, S, D, 128)) != LT_OK) return rc;
+    if ((rc = make_head_map(&mv, V, static_cast<uint64_t>(B) * Hkv, S, D, 128)) != LT_OK) return rc;
 
     cudaError_t e = cudaMemsetAsync(status, 0, kStatusBytes, stream);
     if (e != cudaSuccess) return record_cuda_error("cudaMemsetAsync(status)", e);
@@ -902,7 +932,7 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
     const int pre_blocks = static_cast<int>(want < static_cast<long long>(sms) * 16 ? want : sms * 16);
     bwd_preprocess_kernel<D><<<pre_blocks, 256, 0, stream>>>(reinterpret_cast<const __half *>(dO),
                                                              reinterpret_cast<const __half *>(O), LSE, delta_ext,
-                                                             lse_ext, dq_acc, n_rows, 1.f / scale, status);
+                                                             lse_ext, dq_acc, n_rows, S, S_pad, 1.f / scale, status);
     e = cudaGetLastError();
     if (e != cudaSuccess) return record_cuda_error("bwd_preprocess_kernel launch", e);
 
@@ -913,12 +943,12 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
     prm.dK = reinterpret_cast<__half *>(dK);
     prm.dV = reinterpret_cast<__half *>(dV);
     prm.status = status;
-    prm.B = B; prm.Hq = Hq; prm.Hkv = Hkv; prm.S = S; prm.causal = causal ? 1 : 0;
+    prm.B = B; prm.Hq = Hq; prm.Hkv = Hkv; prm.S = S; prm.S_pad = S_pad; prm.causal = causal ? 1 : 0;
     prm.scale = scale;
     const size_t smem = sizeof(BwdSmem<D>);
     e = cudaFuncSetAttribute(bwd_main_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return record_cuda_error("cudaFuncSetAttribute(bwd_main)", e);
-    const int n_items = B * Hkv * (S / kTileRows);
+    const int n_items = B * Hkv * (S_pad / kTileRows);
     const int grid = n_items < sms ? n_items : sms;  // persistent: one CTA per SM walks the item list
     if (ev_main_begin && (e = cudaEventRecord(ev_main_begin, stream)) != cudaSuccess)
         return record_cuda_error("cudaEventRecord", e);
@@ -928,10 +958,11 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
     if (ev_main_end && (e = cudaEventRecord(ev_main_end, stream)) != cudaSuccess)
         return record_cuda_error("cudaEventRecord", e);
 
-    const long long n_vec8 = n_rows * D / 8;
+    const long long n_vec8 = static_cast<long long>(B) * Hq * S * D / 8;
     const long long fwant = (n_vec8 + 255) / 256;
     const int fin_blocks = static_cast<int>(fwant < static_cast<long long>(sms) * 16 ? fwant : sms * 16);
-    bwd_finalize_kernel<<<fin_blocks, 256, 0, stream>>>(dq_acc, reinterpret_cast<__half *>(dQ), n_vec8);
+    bwd_finalize_kernel<<<fin_blocks, 256, 0, stream>>>(dq_acc, reinterpret_cast<__half *>(dQ), n_vec8, S * (D / 8),
+                                                        S_pad * (D / 8));
     e = cudaGetLastError();
     if (e != cudaSuccess) return record_cuda_error("bwd_finalize_kernel launch", e);
     return LT_OK;
@@ -943,7 +974,7 @@ extern "C" {
 
 size_t lt_attn_bwd_workspace_bytes(int B, int Hq, int Hkv, int S, int D) {
     if (lt::check_shape(B, Hq, Hkv, S, D, 1.0f) != LT_OK) return 0;
-    const size_t n_rows = static_cast<size_t>(B) * Hq * S;
+    const size_t n_rows = static_cast<size_t>(B) * Hq * static_cast<size_t>(lt::padded_rows(S));
     return lt::kStatusBytes + 2 * lt::round256(n_rows * 16) + lt::round256(n_rows * D * 4);
 }
 

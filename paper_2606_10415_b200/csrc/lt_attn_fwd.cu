@@ -85,7 +85,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
     const int lane = tid & 31;
 
     // heavy (late) query-tile pairs get the low block ids
-    const int n_tiles = p.S / kFwdTileRows;
+    const int n_tiles = (p.S + kFwdTileRows - 1) / kFwdTileRows;  // the last tile may be ragged
     const int n_pairs = (n_tiles + 1) / 2;
     const int n_bh = p.B * p.Hq;
     const int pr = p.causal ? (n_pairs - 1 - blockIdx.x / n_bh) : (blockIdx.x / n_bh);
@@ -129,8 +129,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
     const uint32_t tmem = sm.tmem_base;
     volatile int *abort_flag = &sm.abort_flag;
 
-    const long long q_row0 = static_cast<long long>(bh) * p.S + static_cast<long long>(i0) * kFwdTileRows;
-    const long long kv_head_row0 = (static_cast<long long>(b) * p.Hkv + g) * p.S;
+    const int kv_head = b * p.Hkv + g;
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer
@@ -139,20 +138,19 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
                 mbar_arrive_expect_tx(&sm.bar_q[t], kTileBytes);
 #pragma unroll
                 for (int x = 0; x < kBoxes; ++x)
-                    tma_load_2d(sm.q[t] + x * kFwdBoxBytes, &map_q, &sm.bar_q[t], x * 64,
-                                static_cast<int>(q_row0) + t * kFwdTileRows);
+                    tma_load_3d(sm.q[t] + x * kFwdBoxBytes, &map_q, &sm.bar_q[t], x * 64, (i0 + t) * kFwdTileRows, bh);
             }
             bool ok = true;
             int armed = 0;  // key/value tiles whose loads were started
             for (int j = 0; j <= j_end; ++j) {
                 const int s = j & 1;
                 const uint32_t ph = (j >> 1) & 1;
-                const int kv_row0 = static_cast<int>(kv_head_row0 + static_cast<long long>(j) * kFwdTileRows);
+                const int kv_row0 = j * kFwdTileRows;  // inside the head; rows past S arrive as zeros
                 if (j >= 2 && !(ok = mbar_wait(&sm.bar_k_empty[s], ph ^ 1, abort_flag, p.status, kWaitFwdKEmpty))) break;
                 mbar_arrive_expect_tx(&sm.bar_k_full[s], kTileBytes);
 #pragma unroll
                 for (int x = 0; x < kBoxes; ++x)
-                    tma_load_2d(sm.k[s] + x * kFwdBoxBytes, &map_k, &sm.bar_k_full[s], x * 64, kv_row0);
+                    tma_load_3d(sm.k[s] + x * kFwdBoxBytes, &map_k, &sm.bar_k_full[s], x * 64, kv_row0, kv_head);
                 if (j >= 2 && !(ok = mbar_wait(&sm.bar_v_empty[s], ph ^ 1, abort_flag, p.status, kWaitFwdVEmpty))) {
                     // the key tile just started still has to land before shared memory is given up
                     for (int w = 0; w < (1 << 16) && !mbar_try_wait(&sm.bar_k_full[s], ph); ++w) {}
@@ -161,7 +159,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
                 mbar_arrive_expect_tx(&sm.bar_v_full[s], kTileBytes);
 #pragma unroll
                 for (int x = 0; x < kBoxes; ++x)
-                    tma_load_2d(sm.v[s] + x * kFwdBoxBytes, &map_v, &sm.bar_v_full[s], x * 64, kv_row0);
+                    tma_load_3d(sm.v[s] + x * kFwdBoxBytes, &map_v, &sm.bar_v_full[s], x * 64, kv_row0, kv_head);
                 armed = j + 1;
             }
             if (!ok || *abort_flag) {
@@ -263,6 +261,10 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
         const uint32_t tS = tmem + lane_base + kColS + t * 128;
         const uint32_t tO = tmem + lane_base + kColO + t * D;
         const float scale_log2 = p.scale * kFwdLog2e;
+        // last visible key of a masked tile: the row's own index on a causal diagonal tile, the end of
+        // the sequence on the ragged last key tile without a causal mask
+        const int tail_keys = p.S - (n_tiles - 1) * kFwdTileRows;
+        const int last_key = p.causal ? row : tail_keys - 1;
         float m_used = -INFINITY;  // the maximum the stored P, l and O are relative to
         float l = 0.f;             // running sum of exp2(score - m_used)
         bool ok = true;
@@ -281,7 +283,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
             LT_FT(2);
             float rs[4] = {0.f, 0.f, 0.f, 0.f};  // independent partial row sums
             auto tile_softmax = [&](auto diag_tag) {
-                constexpr bool kDiag = decltype(diag_tag)::value;
+                constexpr bool kMasked = decltype(diag_tag)::value;  // keys past `last_key` are invisible
                 // row extremum of the raw scores over the unmasked keys: the maximum of
                 // scale*log2(e)*score is that factor times the largest (smallest, for a negative
                 // scale) raw score
@@ -293,8 +295,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
                     for (int u = 0; u < 8; ++u) ex[u] = -INFINITY;
 #pragma unroll
                     for (int e = 0; e < 64; ++e) {  // two keys per step: a three-input maximum
-                        const float a = (!kDiag || e <= row) ? __uint_as_float(sc[e]) : -INFINITY;
-                        const float c = (!kDiag || e + 64 <= row) ? __uint_as_float(sc[e + 64]) : -INFINITY;
+                        const float a = (!kMasked || e <= last_key) ? __uint_as_float(sc[e]) : -INFINITY;
+                        const float c = (!kMasked || e + 64 <= last_key) ? __uint_as_float(sc[e + 64]) : -INFINITY;
                         ex[e & 7] = fmaxf(ex[e & 7], fmaxf(a, c));
                     }
 #pragma unroll
@@ -306,8 +308,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
                     for (int u = 0; u < 8; ++u) ex[u] = INFINITY;
 #pragma unroll
                     for (int e = 0; e < 64; ++e) {
-                        const float a = (!kDiag || e <= row) ? __uint_as_float(sc[e]) : INFINITY;
-                        const float c = (!kDiag || e + 64 <= row) ? __uint_as_float(sc[e + 64]) : INFINITY;
+                        const float a = (!kMasked || e <= last_key) ? __uint_as_float(sc[e]) : INFINITY;
+                        const float c = (!kMasked || e + 64 <= last_key) ? __uint_as_float(sc[e + 64]) : INFINITY;
                         ex[e & 7] = fminf(ex[e & 7], fminf(a, c));
                     }
 #pragma unroll
@@ -348,7 +350,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
                 for (int e = 0; e < 128; ++e) {
                     const float x = fmaf(__uint_as_float(sc[e]), scale_log2, neg_m);
                     float pe = fast_exp2(x);
-                    if (kDiag && e > row) pe = 0.f;
+                    if (kMasked && e > last_key) pe = 0.f;
                     rs[e & 3] += pe;
                     sc[e] = __float_as_uint(pe);
                 }
@@ -361,7 +363,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
                     tmem_st16(tS + c * 16, out);
                 }
             };
-            if (p.causal && j == i) tile_softmax(std::true_type{});
+            if (p.causal ? (j == i) : (j == n_tiles - 1 && tail_keys < kFwdTileRows)) tile_softmax(std::true_type{});
             else tile_softmax(std::false_type{});
             if (!ok) break;
             const float row_sum = (rs[0] + rs[1]) + (rs[2] + rs[3]);
@@ -386,7 +388,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
         if (ok && j_last >= 0) {
             tc_fence_after_sync();
             const float inv_l = 1.f / l;
-            const long long q_row = q_row0 + static_cast<long long>(t) * kFwdTileRows + row;
+            const int s_row = i * kFwdTileRows + row;  // rows past S belong to nobody
+            const long long q_row = static_cast<long long>(bh) * p.S + s_row;
             __half *o_row = p.O + q_row * D;
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
@@ -400,10 +403,10 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
                     o.y = pack_half2(__uint_as_float(r[8 * v8 + 2]) * inv_l, __uint_as_float(r[8 * v8 + 3]) * inv_l);
                     o.z = pack_half2(__uint_as_float(r[8 * v8 + 4]) * inv_l, __uint_as_float(r[8 * v8 + 5]) * inv_l);
                     o.w = pack_half2(__uint_as_float(r[8 * v8 + 6]) * inv_l, __uint_as_float(r[8 * v8 + 7]) * inv_l);
-                    reinterpret_cast<uint4 *>(o_row + c * 32)[v8] = o;
+                    if (s_row < p.S) reinterpret_cast<uint4 *>(o_row + c * 32)[v8] = o;
                 }
             }
-            p.lse[q_row] = (m_used + log2f(l)) * kFwdLn2;
+            if (s_row < p.S) p.lse[q_row] = (m_used + log2f(l)) * kFwdLn2;
         }
     }
 
@@ -428,9 +431,9 @@ static int launch_fwd(const lt_half *Q, const lt_half *K, const lt_half *V, lt_h
                       int Hkv, int S, int causal, float scale, void *workspace, cudaStream_t stream) {
     CUtensorMap mq, mk, mv;
     int rc;
-    if ((rc = make_tile_map(&mq, Q, static_cast<uint64_t>(B) * Hq * S, D, 128)) != LT_OK) return rc;
-    if ((rc = make_tile_map(&mk, K, static_cast<uint64_t>(B) * Hkv * S, D, 128)) != LT_OK) return rc;
-    if ((rc = make_tile_map(&mv, V, static_cast<uint64_t>(B) * Hkv * S, D, 128)) != LT_OK) return rc;
+    if ((rc = make_head_map(&mq, Q, static_cast<uint64_t>(B) * Hq, S, D, 128)) != LT_OK) return rc;
+    if ((rc = make_head_map(&mk, K, static_cast<uint64_t>(B) * Hkv, S, D, 128)) != LT_OK) return rc;
+    if ((rc = make_head_map(&mv, V, static_cast<uint64_t>(B) * Hkv, S, D, 128)) != LT_OK) return rc;
     cudaError_t e = cudaMemsetAsync(workspace, 0, kStatusBytes, stream);
     if (e != cudaSuccess) return record_cuda_error("cudaMemsetAsync(status)", e);
     FwdParams prm;
@@ -443,7 +446,7 @@ static int launch_fwd(const lt_half *Q, const lt_half *K, const lt_half *V, lt_h
     const size_t smem = std::max<size_t>(sizeof(FwdSmem<D>) + 1024, 120 * 1024);
     e = cudaFuncSetAttribute(fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return record_cuda_error("cudaFuncSetAttribute(fwd)", e);
-    const int n_tiles = S / kFwdTileRows;
+    const int n_tiles = (S + kFwdTileRows - 1) / kFwdTileRows;
     const int grid = B * Hq * ((n_tiles + 1) / 2);
     fwd_kernel<D><<<grid, kFwdThreads, smem, stream>>>(mq, mk, mv, prm);
     e = cudaGetLastError();

@@ -38,9 +38,8 @@ int check_shape(int B, int Hq, int Hkv, int S, int D, float scale) {
     if (Hq % Hkv != 0) return LT_ERR_INVALID_ARG;
     if (!isfinite(scale) || scale == 0.f) return LT_ERR_INVALID_ARG;
     if (D != 64 && D != 128) return LT_ERR_UNSUPPORTED;
-    if (S % 128 != 0) return LT_ERR_UNSUPPORTED;
-    // row indices of the [B*H*S, D] tensor views must fit a 32-bit TMA coordinate
-    if (static_cast<long long>(B) * Hq * S >= (1LL << 31)) return LT_ERR_UNSUPPORTED;
+    // padded row indices (every head rounded up to whole 128-row tiles) must fit 32 bits
+    if (static_cast<long long>(B) * Hq * padded_rows(S) >= (1LL << 31)) return LT_ERR_UNSUPPORTED;
     return LT_OK;
 }
 
@@ -70,6 +69,26 @@ int make_tile_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t co
     cuuint32_t box[2] = {64u, box_rows};
     cuuint32_t estr[2] = {1u, 1u};
     CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        char buf[64];
+        snprintf(buf, sizeof(buf), "CUresult %d", static_cast<int>(r));
+        set_last_error("cuTensorMapEncodeTiled", buf);
+        return LT_ERR_CUDA;
+    }
+    return LT_OK;
+}
+
+int make_head_map(CUtensorMap *map, const void *base, uint64_t heads, uint64_t rows_per_head, uint64_t cols,
+                  uint32_t box_rows) {
+    EncodeTiledFn enc = get_encoder();
+    if (!enc) return LT_ERR_CUDA;
+    cuuint64_t dims[3] = {cols, rows_per_head, heads};
+    cuuint64_t strides[2] = {cols * sizeof(__half), rows_per_head * cols * sizeof(__half)};
+    cuuint32_t box[3] = {64u, box_rows, 1u};
+    cuuint32_t estr[3] = {1u, 1u, 1u};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {

@@ -29,5 +29,11 @@ inline size_t round256(size_t n) { return (n + 255u) & ~static_cast<size_t>(255u
 // fp16 matrix [rows, cols] row-major viewed as a 2-D tensor; tiles of box_rows x 64
 // columns are fetched with the 128-byte swizzle.  Returns LT_OK or LT_ERR_CUDA.
 int make_tile_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+// 3-D view [heads][rows_per_head][cols] of a contiguous fp16 tensor with boxes of 64 columns x
+// box_rows rows x 1 head (128-byte swizzle); rows past the end of a head are filled with zeros.
+int make_head_map(CUtensorMap *map, const void *base, uint64_t heads, uint64_t rows_per_head, uint64_t cols,
+                  uint32_t box_rows);
+// sequence length rounded up to whole 128-row tiles
+inline long long padded_rows(int S) { return (static_cast<long long>(S) + 127) / 128 * 128; }
 
 }  // namespace lt

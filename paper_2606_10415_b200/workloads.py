@@ -62,12 +62,14 @@ CONFIGS = {
 
 # Further workloads: the other sequence lengths and the layer shape the paper's Attention-BP
 # measurement uses (Section 6.6: a LLaMA-2-7B layer at S = 1024, 2048, 4096 and a Qwen2.5-32B
-# layer at S = 2048), and an unmasked variant.  Same value distributions and seed.
+# layer at S = 2048), an unmasked variant and a ragged length.  Same value distributions and seed.
 EXTRA_CONFIGS = {
     "llama2_7b_s1024": _cfg("llama2_7b_s1024", 1, 32, 32, 1024, 128, _STD128, 1e-2),
     "llama2_7b_s2048": _cfg("llama2_7b_s2048", 1, 32, 32, 2048, 128, _STD128, 1e-2),
     "qwen25_32b_gqa_s2048": _cfg("qwen25_32b_gqa_s2048", 1, 40, 8, 2048, 128, _STD128, 1e-2),
     "llama2_7b_full_mask_off": _cfg("llama2_7b_full_mask_off", 1, 32, 32, 4096, 128, _STD128, 1e-2, causal=False),
+    # a length that is not a whole number of 128-row tiles (the last tile holds 56 rows)
+    "llama2_7b_s3000_ragged": _cfg("llama2_7b_s3000_ragged", 1, 32, 32, 3000, 128, _STD128, 1e-2),
 }
 ALL_CONFIGS = {**CONFIGS, **EXTRA_CONFIGS}
 

@@ -43,7 +43,10 @@ def test_workspace_sizes(binding):
     assert binding.lt_attn_bwd_workspace_bytes(1, 32, 32, 4096, 128) == 256 + 2 * 2097152 + 67108864
     assert binding.lt_attn_fwd_workspace_bytes(1, 2, 2, 128, 64) == 256
     # unsupported shapes report 0
-    assert binding.lt_attn_bwd_workspace_bytes(1, 2, 2, 100, 64) == 0
+    assert binding.lt_attn_bwd_workspace_bytes(1, 2, 2, 0, 64) == 0
+    # a ragged length is padded to whole 128-row tiles inside the workspace
+    assert binding.lt_attn_bwd_workspace_bytes(1, 2, 2, 100, 64) == binding.lt_attn_bwd_workspace_bytes(1, 2, 2, 128, 64)
+    assert binding.lt_attn_bwd_workspace_bytes(1, 2, 2, 129, 64) == binding.lt_attn_bwd_workspace_bytes(1, 2, 2, 256, 64)
     assert binding.lt_attn_bwd_workspace_bytes(1, 2, 2, 128, 96) == 0
     assert binding.lt_attn_bwd_workspace_bytes(1, 3, 2, 128, 64) == 0
     assert binding.lt_attn_host_arena_bytes(1, 2, 2, 128, 64) > binding.lt_attn_bwd_workspace_bytes(1, 2, 2, 128, 64)
@@ -68,7 +71,7 @@ def test_bwd_rejects_bad_arguments_without_launching(binding):
     assert b.lt_attn_bwd_raw(*_bwd_args(Hq=3, Hkv=2)) == b.LT_ERR_INVALID_ARG
     assert b.lt_attn_bwd_raw(*_bwd_args(scale=float("nan"))) == b.LT_ERR_INVALID_ARG
     assert b.lt_attn_bwd_raw(*_bwd_args(scale=0.0)) == b.LT_ERR_INVALID_ARG
-    assert b.lt_attn_bwd_raw(*_bwd_args(S=100)) == b.LT_ERR_UNSUPPORTED
+    assert b.lt_attn_bwd_raw(*_bwd_args(S=100, ws_bytes=1 << 10)) == b.LT_ERR_WORKSPACE  # ragged S is a shape like any other
     assert b.lt_attn_bwd_raw(*_bwd_args(D=96)) == b.LT_ERR_UNSUPPORTED
     assert b.lt_attn_bwd_raw(*_bwd_args(ptr=0x1004)) == b.LT_ERR_UNSUPPORTED  # misaligned
     assert b.lt_attn_bwd_raw(*_bwd_args(ws=0)) == b.LT_ERR_WORKSPACE
@@ -86,7 +89,6 @@ def test_fwd_rejects_bad_arguments_without_launching(binding):
     a[4] = 0
     assert b.lt_attn_fwd_raw(*a) == b.LT_ERR_INVALID_ARG
     assert b.lt_attn_fwd_raw(*args(S=0)) == b.LT_ERR_INVALID_ARG
-    assert b.lt_attn_fwd_raw(*args(S=192)) == b.LT_ERR_UNSUPPORTED
     assert b.lt_attn_fwd_raw(*args(D=256)) == b.LT_ERR_UNSUPPORTED
     assert b.lt_attn_fwd_raw(*args(ws_bytes=16)) == b.LT_ERR_WORKSPACE
 

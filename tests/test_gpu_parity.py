@@ -100,6 +100,9 @@ def test_bounded_wait_reports_timeout_and_context_survives(lt):
 FWD_SHAPES = [
     (1, 2, 2, 128, 64, True), (1, 2, 2, 128, 128, True), (2, 4, 2, 384, 64, True),
     (1, 5, 1, 512, 128, True), (1, 2, 2, 256, 128, False), (2, 2, 1, 384, 64, False),
+    # ragged last tiles: shorter than one tile, one row past a tile, odd tile counts
+    (2, 2, 1, 1, 64, True), (1, 2, 2, 100, 128, True), (2, 4, 2, 129, 64, True), (1, 3, 1, 333, 128, True),
+    (1, 2, 2, 100, 128, False), (2, 2, 1, 257, 64, False), (1, 2, 1, 200, 128, False),
 ]
 
 
@@ -128,7 +131,7 @@ def test_delta_preprocess_matches_oracle(lt, oracle):
     ws = lt.alloc_workspace(lt.lt_attn_bwd_workspace_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.S, cfg.D))
     lt.lt_attn_bwd(Qd, Kd, Vd, Od, dOd, Ld, dQ, dK, dV, True, cfg.scale, ws)
     assert lt.lt_attn_check_status(ws) == lt.LT_OK
-    n = cfg.B * cfg.Hq * cfg.S
+    n = cfg.B * cfg.Hq * cfg.S  # S is a whole number of tiles here, so the row space has no padding
     rows = ws[256:256 + 16 * n].view(torch.float16).cpu().double().numpy().reshape(n, 8)
     assert np.all(rows[:, 2:] == 0)
     delta = -(256.0 * rows[:, 0] + rows[:, 1]).reshape(cfg.B, cfg.Hq, cfg.S)
@@ -141,6 +144,9 @@ BWD_SHAPES = [
     (1, 2, 2, 128, 64, True), (1, 2, 2, 128, 128, True), (1, 1, 1, 256, 128, True),
     (2, 4, 2, 384, 64, True), (1, 5, 1, 512, 128, True), (2, 8, 1, 256, 128, True),
     (1, 2, 2, 256, 128, False), (2, 4, 2, 384, 64, False), (1, 1, 1, 128, 128, False),
+    # ragged last tiles
+    (2, 2, 1, 3, 64, True), (1, 2, 2, 100, 128, True), (2, 4, 2, 129, 64, True), (1, 6, 2, 333, 128, True),
+    (1, 2, 2, 100, 128, False), (2, 2, 1, 257, 64, False), (1, 4, 1, 200, 128, False),
 ]
 
 
@@ -252,6 +258,7 @@ def test_llama2_70b_gqa_config_sampled_groups(lt, oracle):
     ("llama2_7b_s1024", [(0, 0), (0, 31)]),
     ("llama2_7b_s2048", [(0, 5)]),
     ("qwen25_32b_gqa_s2048", [(0, 3)]),
+    ("llama2_7b_s3000_ragged", [(0, 9)]),
     ("llama2_7b_full_mask_off", [(0, 9)]),
 ])
 def test_other_sequence_lengths_and_unmasked(lt, oracle, name, units):
