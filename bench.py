@@ -38,6 +38,7 @@ NOMINAL_FP16_TFLOPS = 2250.0  # datasheet dense figure, context only
 # summarised in profiles/bwd_main_kernel_llama2_7b.md (taken on the full configuration itself)
 MAIN_KERNEL_DRAM_BYTES = {"llama2_7b": 688.0e6}
 FALLBACK_PEAK_TFLOPS = 1590.0
+FALLBACK_SUSTAINED_TFLOPS = 1400.0
 
 
 def parse_args():
@@ -65,6 +66,16 @@ def measured_peak():
         d = json.loads(path.read_text())
         return float(d["bf16_tflops"]), float(d.get("hbm_gbs", 0.0)), "measured"
     return FALLBACK_PEAK_TFLOPS, 6650.0, "fallback"
+
+
+def measured_sustained_peak():
+    """Dense bf16 throughput of back-to-back GEMMs under the power cap (the fp16 rate is the same)."""
+    path = ROOT / "MEASURED_PEAKS.json"
+    if path.exists():
+        d = json.loads(path.read_text())
+        if "bf16_tflops_sustained" in d:
+            return float(d["bf16_tflops_sustained"]), "measured"
+    return FALLBACK_SUSTAINED_TFLOPS, "fallback"
 
 
 # ------------------------------------------------------------------ CPU oracle legs
@@ -281,6 +292,19 @@ def run_ours(args, cfg):
         raise SystemExit("backward kernel reported: " + lt.last_cuda_error())
     main_ms = [a.elapsed_time(b) for a, b in kernel_events]
 
+    # the main kernel timed alone: single launches with the GPU idle in between (the way the burst
+    # GEMM peak was taken: best of 10)
+    iso_ms = []
+    ia, ib = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ia.record()
+    ib.record()
+    for _ in range(10):
+        torch.cuda.synchronize()
+        time.sleep(0.03)
+        step(ia, ib)
+        torch.cuda.synchronize()
+        iso_ms.append(ia.elapsed_time(ib))
+
     # end to end through the host-buffer entry point: pinned host inputs, host outputs
     pin = [t.pin_memory() for t in (Qh, Kh, Vh, dOh)]
     hO = torch.empty_like(Qh).pin_memory()
@@ -312,8 +336,11 @@ def run_ours(args, cfg):
         ms_per_step = total_ms / args.steps
         value = job_throughput(cfg.flops, world, ms_per_step * 1e-3)
         peak, _hbm, peak_kind = measured_peak()
+        sustained_peak, sustained_kind = measured_sustained_peak()
         main_avg_ms = sum(main_ms) / len(main_ms)
         achieved = cfg.flops / (main_avg_ms * 1e-3) / 1e12
+        iso_best_ms = min(iso_ms)
+        iso_achieved = cfg.flops / (iso_best_ms * 1e-3) / 1e12
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
@@ -323,6 +350,7 @@ def run_ours(args, cfg):
                        if _step_bytes(cfg) > 126e6 else "working set fits L2",
                        "multi_gpu": "replicas only" if world > 1 else "single"},
             "pct_of_measured_peak": 100.0 * value / world / peak,
+            "pct_of_measured_sustained_peak": 100.0 * value / world / sustained_peak,
             "pct_of_nominal_fp16_peak": 100.0 * value / world / NOMINAL_FP16_TFLOPS,
             "peak_source": peak_kind,
             "clocks": clocks,
@@ -330,12 +358,20 @@ def run_ours(args, cfg):
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
                     "includes": "H2D copies, lt_attn_fwd, lt_attn_bwd, D2H copies"},
             "gpu_launches": args.steps * lt.lt_attn_bwd_num_launches(),
-            "roofline": {"bound": "tensor", "kernel": "bwd_main_kernel", "achieved": achieved, "peak": peak,
-                         "unit": "TFLOP/s", "frac": achieved / peak,
+            # The average launch inside the timed loop runs at sustained, power-capped clocks, so it is
+            # set against the sustained GEMM figure; the same average against the burst figure and a
+            # launch timed alone against the burst figure are given beside it.
+            "roofline": {"bound": "tensor", "kernel": "bwd_main_kernel", "achieved": achieved,
+                         "peak": sustained_peak, "unit": "TFLOP/s", "frac": achieved / sustained_peak,
                          "traffic": MAIN_KERNEL_DRAM_BYTES.get(cfg.name), "traffic_unit": "bytes per launch (ncu)",
                          "algorithmic_hbm_bytes": _step_bytes(cfg) - 4.0 * cfg.B * cfg.Hq * cfg.S * cfg.D,
-                         "peak_source": peak_kind + " bf16 burst", "avg_launch_ms": main_avg_ms,
-                         "best_launch_ms": min(main_ms)},
+                         "peak_source": sustained_kind + " bf16 sustained (kernel timed inside the step loop)",
+                         "avg_launch_ms": main_avg_ms, "best_launch_ms": min(main_ms),
+                         "burst_peak": peak, "frac_of_burst_peak": achieved / peak,
+                         "timed_alone": {"best_launch_ms": iso_best_ms, "achieved": iso_achieved, "peak": peak,
+                                         "frac": iso_achieved / peak,
+                                         "how": "best of 10 single launches, GPU idle 30 ms before each; "
+                                                + peak_kind + " bf16 burst peak"}},
             "fwd": {"value": fwd_flops / (fwd_ms * 1e-3) / 1e12, "unit": UNIT, "ms": fwd_ms},
         }
         if not args.no_cpu_baseline and world == 1:

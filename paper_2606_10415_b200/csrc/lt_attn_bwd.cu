@@ -89,6 +89,12 @@ bwd_preprocess_kernel(const __half *__restrict__ dO, const __half *__restrict__ 
                 b[u] = __ldcs(reinterpret_cast<const uint4 *>(O + src * D) + sub);
                 if (sub == 0) l[u] = __ldg(lse + src);
             }
+            if (row < n_rows) {
+                // the zero fill does not depend on the loads: issue it while they are in flight
+                float4 *z = reinterpret_cast<float4 *>(dq_acc + row * D) + sub * 2;
+                z[0] = make_float4(0.f, 0.f, 0.f, 0.f);
+                z[1] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
         }
 #pragma unroll
         for (int u = 0; u < kPreUnroll; ++u) {
@@ -111,9 +117,6 @@ bwd_preprocess_kernel(const __half *__restrict__ dO, const __half *__restrict__ 
                 n2 += __shfl_xor_sync(0xffffffffu, n2, off);
             }
             if (row < n_rows) {
-                float4 *z = reinterpret_cast<float4 *>(dq_acc + row * D) + sub * 2;
-                z[0] = make_float4(0.f, 0.f, 0.f, 0.f);
-                z[1] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (sub == 0) {
                     // operand rows of the main kernel's extra contraction step: 256*hi + lo = value
                     delta_ext[row] = make_uint4(split_hi_lo(-acc), 0u, 0u, 0u);
@@ -129,10 +132,21 @@ bwd_preprocess_kernel(const __half *__restrict__ dO, const __half *__restrict__ 
         max_abs_delta = fmaxf(max_abs_delta, __shfl_xor_sync(0xffffffffu, max_abs_delta, off));
         max_norm2 = fmaxf(max_norm2, __shfl_xor_sync(0xffffffffu, max_norm2, off));
     }
+    // one pair of atomics per block, and only when it would raise the stored maximum: thousands of
+    // atomics on the same two words would otherwise queue up behind one another in L2
+    __shared__ float block_max[2][8];
     if (lane == 0) {
+        block_max[0][threadIdx.x >> 5] = max_abs_delta;
+        block_max[1][threadIdx.x >> 5] = max_norm2;
+    }
+    __syncthreads();
+    if (threadIdx.x < 2) {
+        float m = 0.f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) m = fmaxf(m, block_max[threadIdx.x][w]);
         // non-negative floats order like their bit patterns; NaN/inf inputs simply saturate the bound
-        atomicMax(status + kStatusWordMaxAbsDelta, __float_as_uint(max_abs_delta));
-        atomicMax(status + kStatusWordMaxDoNorm2, __float_as_uint(max_norm2));
+        unsigned int *word = status + (threadIdx.x == 0 ? kStatusWordMaxAbsDelta : kStatusWordMaxDoNorm2);
+        if (__float_as_uint(m) > *reinterpret_cast<volatile unsigned int *>(word)) atomicMax(word, __float_as_uint(m));
     }
 }
 
