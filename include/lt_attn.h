@@ -121,6 +121,33 @@ int lt_attn_bwd_noalloc(const lt_half *Q, const lt_half *K, const lt_half *V,
                         int B, int Hq, int Hkv, int S, int D, int causal, float scale,
                         lt_stream_t stream);
 
+/* Layouts other than contiguous [B,H,S,D].  Each tensor is described by the element strides of
+ * its batch, head and row (sequence position) indices; the D elements of a row are always
+ * contiguous.  Element (b, h, s, d) lives at base + b*batch + h*head + s*row + d.  A fused
+ * QKV projection output [B, S, (Hq + 2 Hkv) * D], or a [B,S,H,D] tensor, is such a view.
+ * Every stride must be a positive multiple of 8 elements (16 bytes) and row >= D; views must not
+ * overlap themselves.  LSE is always contiguous [B,Hq,S].  The paper fixes no memory layout. */
+typedef struct lt_tensor_strides {
+    long long batch, head, row;
+} lt_tensor_strides;
+typedef struct lt_attn_layout {
+    lt_tensor_strides q, k, v, o, d_o, dq, dk, dv;  /* the forward reads q, k, v, o only */
+} lt_attn_layout;
+
+/* lt_attn_fwd / lt_attn_bwd on strided views.  `layout` is a HOST pointer read during the call
+ * (NULL means contiguous [B,H,S,D], i.e. exactly lt_attn_fwd / lt_attn_bwd).  Same workspace
+ * sizes, status codes and error behaviour; a stride that breaks the rules above returns
+ * LT_ERR_UNSUPPORTED and launches nothing. */
+int lt_attn_fwd_strided(const lt_half *Q, const lt_half *K, const lt_half *V,
+                        lt_half *O, float *LSE, const lt_attn_layout *layout,
+                        int B, int Hq, int Hkv, int S, int D, int causal, float scale,
+                        void *workspace, size_t workspace_bytes, lt_stream_t stream);
+int lt_attn_bwd_strided(const lt_half *Q, const lt_half *K, const lt_half *V,
+                        const lt_half *O, const lt_half *dO, const float *LSE,
+                        lt_half *dQ, lt_half *dK, lt_half *dV, const lt_attn_layout *layout,
+                        int B, int Hq, int Hkv, int S, int D, int causal, float scale,
+                        void *workspace, size_t workspace_bytes, lt_stream_t stream);
+
 /* Same computation as lt_attn_fwd followed by lt_attn_bwd, but every tensor pointer is
  * a HOST pointer (pinned memory makes the copies asynchronous).  `arena` is a caller-
  * owned DEVICE buffer of at least lt_attn_host_arena_bytes() bytes, 256-byte aligned,

@@ -23,11 +23,21 @@ LT_ERR_DEVICE_TIMEOUT = 5
 
 EXPORTS = (
     "lt_attn_fwd_workspace_bytes", "lt_attn_bwd_workspace_bytes", "lt_attn_fwd", "lt_attn_bwd",
-    "lt_attn_bwd_profiled", "lt_attn_bwd_noalloc",
+    "lt_attn_bwd_profiled", "lt_attn_bwd_noalloc", "lt_attn_fwd_strided", "lt_attn_bwd_strided",
     "lt_attn_host_arena_bytes", "lt_attn_fwd_bwd_host", "lt_attn_check_status", "lt_status_string",
     "lt_last_cuda_error", "lt_attn_bwd_num_launches", "lt_attn_fwd_num_launches", "lt_dbg_tile_gemm",
     "lt_dbg_wait_timeout",
 )
+
+
+class TensorStrides(ctypes.Structure):
+    """Element strides of the batch, head and row indices (``lt_tensor_strides``)."""
+    _fields_ = [("batch", ctypes.c_longlong), ("head", ctypes.c_longlong), ("row", ctypes.c_longlong)]
+
+
+class AttnLayout(ctypes.Structure):
+    """``lt_attn_layout``: strides of q, k, v, o, d_o, dq, dk, dv in that order."""
+    _fields_ = [(n, TensorStrides) for n in ("q", "k", "v", "o", "d_o", "dq", "dk", "dv")]
 
 
 class LtError(RuntimeError):
@@ -56,6 +66,10 @@ def _load() -> ctypes.CDLL:
     lib.lt_attn_bwd.restype = i
     lib.lt_attn_bwd_profiled.argtypes = [vp] * 9 + [i] * 6 + [f, vp, sz, vp, vp, vp]
     lib.lt_attn_bwd_profiled.restype = i
+    lib.lt_attn_fwd_strided.argtypes = [vp] * 5 + [ctypes.POINTER(AttnLayout)] + [i] * 6 + [f, vp, sz, vp]
+    lib.lt_attn_fwd_strided.restype = i
+    lib.lt_attn_bwd_strided.argtypes = [vp] * 9 + [ctypes.POINTER(AttnLayout)] + [i] * 6 + [f, vp, sz, vp]
+    lib.lt_attn_bwd_strided.restype = i
     lib.lt_attn_bwd_noalloc.argtypes = [vp] * 9 + [i] * 6 + [f, vp]
     lib.lt_attn_bwd_noalloc.restype = i
     lib.lt_attn_fwd_bwd_host.argtypes = [vp] * 9 + [i] * 6 + [f, vp, sz, vp]
@@ -156,6 +170,42 @@ def lt_attn_bwd(Q, K, V, O, dO, LSE, dQ, dK, dV, causal, scale, workspace, strea
                           workspace.numel() * workspace.element_size(), _stream_ptr(stream))
     if rc != LT_OK:
         raise LtError("lt_attn_bwd", rc)
+
+
+def _strides_of(t: torch.Tensor) -> TensorStrides:
+    """Strides of a logical ``[B, H, S, D]`` view (any permutation or slice with unit D stride)."""
+    if t.dim() != 4 or t.stride(3) != 1:
+        raise ValueError("expected a [B, H, S, D] view whose last dimension is contiguous")
+    return TensorStrides(int(t.stride(0)), int(t.stride(1)), int(t.stride(2)))
+
+
+def lt_attn_fwd_strided(Q, K, V, O, LSE, causal, scale, workspace, stream=None) -> None:
+    """lt_attn_fwd on ``[B, H, S, D]`` *views* (e.g. a permuted [B,S,H,D] tensor or slices of a fused
+    QKV buffer); the strides are taken from the tensors.  LSE must be contiguous."""
+    _check_layout(LSE)
+    B, Hq, Hkv, S, D = _dims(Q, K)
+    lay = AttnLayout()
+    lay.q, lay.k, lay.v, lay.o = (_strides_of(t) for t in (Q, K, V, O))
+    rc = _lib.lt_attn_fwd_strided(_ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(LSE), ctypes.byref(lay), B, Hq, Hkv, S, D,
+                                  int(bool(causal)), float(scale), _ptr(workspace),
+                                  workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    if rc != LT_OK:
+        raise LtError("lt_attn_fwd_strided", rc)
+
+
+def lt_attn_bwd_strided(Q, K, V, O, dO, LSE, dQ, dK, dV, causal, scale, workspace, stream=None) -> None:
+    """lt_attn_bwd on ``[B, H, S, D]`` views; the strides are taken from the tensors.  LSE contiguous."""
+    _check_layout(LSE)
+    B, Hq, Hkv, S, D = _dims(Q, K)
+    lay = AttnLayout()
+    lay.q, lay.k, lay.v, lay.o, lay.d_o, lay.dq, lay.dk, lay.dv = (
+        _strides_of(t) for t in (Q, K, V, O, dO, dQ, dK, dV))
+    rc = _lib.lt_attn_bwd_strided(_ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(dO), _ptr(LSE), _ptr(dQ), _ptr(dK),
+                                  _ptr(dV), ctypes.byref(lay), B, Hq, Hkv, S, D, int(bool(causal)), float(scale),
+                                  _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                  _stream_ptr(stream))
+    if rc != LT_OK:
+        raise LtError("lt_attn_bwd_strided", rc)
 
 
 def lt_attn_bwd_profiled(Q, K, V, O, dO, LSE, dQ, dK, dV, causal, scale, workspace, stream=None,

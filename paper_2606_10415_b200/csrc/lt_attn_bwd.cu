@@ -59,7 +59,8 @@ template <int D>
 __global__ void __launch_bounds__(256)
 bwd_preprocess_kernel(const __half *__restrict__ dO, const __half *__restrict__ O, const float *__restrict__ lse,
                       uint4 *__restrict__ delta_ext, uint4 *__restrict__ lse_ext, float *__restrict__ dq_acc,
-                      long long n_rows, int S, int S_pad, float inv_scale, unsigned int *status) {
+                      long long n_rows, int S, int S_pad, int Hq, lt_tensor_strides do_st, lt_tensor_strides o_st,
+                      int plain, float inv_scale, unsigned int *status) {
     // `n_rows` counts rows of the padded row space (every head rounded up to S_pad rows), the
     // indexing of delta_ext, lse_ext and dq_acc; padding rows get zeros everywhere.
     constexpr int kLanesPerRow = D / 8;
@@ -78,16 +79,23 @@ bwd_preprocess_kernel(const __half *__restrict__ dO, const __half *__restrict__ 
             const long long row = row0 + u * kRowsPerWarp + lane / kLanesPerRow;
             a[u] = b[u] = make_uint4(0u, 0u, 0u, 0u);
             l[u] = 0.f;
-            long long src = row;  // row of dO / O / LSE behind padded row `row`, -1 for padding
-            if (S != S_pad) {
-                const long long head = row / S_pad;
-                const int s_in = static_cast<int>(row - head * S_pad);
-                src = s_in < S ? head * S + s_in : -1;
+            // rows of dO, O and LSE behind padded row `row` (`plain`: contiguous tensors and no padding,
+            // so all three are row `row` itself)
+            long long src_do = row * D, src_o = row * D, src_lse = row;
+            bool valid = row < n_rows;
+            if (!plain && valid) {
+                const int bh = static_cast<int>(row / S_pad);
+                const int s_in = static_cast<int>(row - static_cast<long long>(bh) * S_pad);
+                const int bb = bh / Hq, hh = bh - bb * Hq;
+                valid = s_in < S;
+                src_do = bb * do_st.batch + hh * do_st.head + s_in * do_st.row;
+                src_o = bb * o_st.batch + hh * o_st.head + s_in * o_st.row;
+                src_lse = static_cast<long long>(bh) * S + s_in;
             }
-            if (row < n_rows && src >= 0) {
-                a[u] = __ldcs(reinterpret_cast<const uint4 *>(dO + src * D) + sub);
-                b[u] = __ldcs(reinterpret_cast<const uint4 *>(O + src * D) + sub);
-                if (sub == 0) l[u] = __ldg(lse + src);
+            if (valid) {
+                a[u] = __ldcs(reinterpret_cast<const uint4 *>(dO + src_do) + sub);
+                b[u] = __ldcs(reinterpret_cast<const uint4 *>(O + src_o) + sub);
+                if (sub == 0) l[u] = __ldg(lse + src_lse);
             }
             if (row < n_rows) {
                 // the zero fill does not depend on the loads: issue it while they are in flight
@@ -153,14 +161,19 @@ bwd_preprocess_kernel(const __half *__restrict__ dO, const __half *__restrict__ 
 // ----------------------------------------------------------------------------- finalize
 __global__ void __launch_bounds__(256)
 bwd_finalize_kernel(const float *__restrict__ dq_acc, __half *__restrict__ dQ, long long n_vec8, int vec_per_head,
-                    int vec_per_padded_head) {
-    // n_vec8 groups of eight output elements; the accumulator is indexed in the padded row space
+                    int vec_per_padded_head, int vec_per_row, int Hq, lt_tensor_strides dq_st, int plain) {
+    // n_vec8 groups of eight output elements, numbered over the logical [B,Hq,S,D]; the accumulator
+    // is indexed in the padded row space (`plain`: contiguous dQ and no padding, so both are group v)
     const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
     for (long long v = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; v < n_vec8; v += stride) {
-        long long src = v;
-        if (vec_per_head != vec_per_padded_head) {
-            const long long head = v / vec_per_head;
-            src = head * vec_per_padded_head + (v - head * vec_per_head);
+        long long src = v, dst = v * 8;
+        if (!plain) {
+            const int bh = static_cast<int>(v / vec_per_head);
+            const int rem = static_cast<int>(v - static_cast<long long>(bh) * vec_per_head);
+            const int s_in = rem / vec_per_row, c = rem - s_in * vec_per_row;
+            const int bb = bh / Hq, hh = bh - bb * Hq;
+            src = static_cast<long long>(bh) * vec_per_padded_head + rem;
+            dst = bb * dq_st.batch + hh * dq_st.head + s_in * dq_st.row + c * 8;
         }
         const float4 a = __ldcs(reinterpret_cast<const float4 *>(dq_acc) + 2 * src);
         const float4 b = __ldcs(reinterpret_cast<const float4 *>(dq_acc) + 2 * src + 1);
@@ -169,7 +182,7 @@ bwd_finalize_kernel(const float *__restrict__ dq_acc, __half *__restrict__ dQ, l
         o.y = pack_half2(a.z, a.w);
         o.z = pack_half2(b.x, b.y);
         o.w = pack_half2(b.z, b.w);
-        reinterpret_cast<uint4 *>(dQ)[v] = o;
+        *reinterpret_cast<uint4 *>(dQ + dst) = o;
     }
 }
 
@@ -269,12 +282,13 @@ struct BwdParams {
     unsigned int *status;
     int B, Hq, Hkv, S, S_pad, causal;  // S_pad: S rounded up to whole 128-row tiles
     float scale;
+    lt_tensor_strides dk_st, dv_st;  // element strides of dK and dV
 };
 
 // One work item = key tile j of (batch b, kv head g).  Items are numbered so that the heavy
 // ones (small j under a causal mask) come first; CTA c takes items c, c + gridDim.x, ...
 struct BwdItem {
-    int j, b, g, i_first, tiles_per_head, n_iter, kv_head;
+    int j, b, g, i_first, tiles_per_head, n_iter;
 };
 __device__ __forceinline__ BwdItem bwd_item(const BwdParams &p, int item) {
     BwdItem w;
@@ -287,23 +301,22 @@ __device__ __forceinline__ BwdItem bwd_item(const BwdParams &p, int item) {
     w.i_first = p.causal ? w.j : 0;
     w.tiles_per_head = n_tiles - w.i_first;
     w.n_iter = (p.Hq / p.Hkv) * w.tiles_per_head;  // flattened (query head of the group, query tile) loop
-    w.kv_head = w.b * p.Hkv + w.g;
     return w;
 }
-// Iteration n of an item -> its query tile: flattened (batch, query head) index, first row
-// inside the head, and the tile's first row in the padded row space of the workspace arrays
+// Iteration n of an item -> its query tile: batch, query head, first row inside the head, and the tile's first row in the padded row space of the workspace arrays
 // (every head rounded up to whole tiles, so tiles never straddle heads).
 struct BwdQTile {
-    int head, s0;
+    int b, h, s0;
     long long padded_row0;
 };
 __device__ __forceinline__ BwdQTile bwd_q_tile(const BwdParams &p, const BwdItem &w, int n) {
     const int hh = n / w.tiles_per_head;
     const int i = w.i_first + (n - hh * w.tiles_per_head);
     BwdQTile q;
-    q.head = w.b * p.Hq + w.g * (p.Hq / p.Hkv) + hh;
+    q.b = w.b;
+    q.h = w.g * (p.Hq / p.Hkv) + hh;
     q.s0 = i * kTileRows;
-    q.padded_row0 = static_cast<long long>(q.head) * p.S_pad + q.s0;
+    q.padded_row0 = (static_cast<long long>(w.b) * p.Hq + q.h) * p.S_pad + q.s0;
     return q;
 }
 
@@ -410,14 +423,14 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     mbar_arrive_expect_tx(&sm.bar_q_full[s], kTileBytes + kExtBytes);
 #pragma unroll
                     for (int x = 0; x < kBoxes; ++x)
-                        tma_load_3d(sm.q[s] + x * kBoxBytesBwd, &map_q, &sm.bar_q_full[s], x * 64, qt.s0, qt.head);
+                        tma_load_4d(sm.q[s] + x * kBoxBytesBwd, &map_q, &sm.bar_q_full[s], x * 64, qt.s0, qt.h, qt.b);
                     bulk_load_1d(sm.ext_q[s], p.lse_ext + qt.padded_row0, kExtBytes, &sm.bar_q_full[s]);
                     last_q = it;
                     if (it >= 1 && !(ok = LT_WAIT(&sm.bar_do_empty, (it - 1) & 1, kWaitDoEmpty))) break;
                     mbar_arrive_expect_tx(&sm.bar_do_full, kTileBytes + kExtBytes);
 #pragma unroll
                     for (int x = 0; x < kBoxes; ++x)
-                        tma_load_3d(sm.d_o + x * kBoxBytesBwd, &map_do, &sm.bar_do_full, x * 64, qt.s0, qt.head);
+                        tma_load_4d(sm.d_o + x * kBoxBytesBwd, &map_do, &sm.bar_do_full, x * 64, qt.s0, qt.h, qt.b);
                     bulk_load_1d(sm.ext_do, p.delta_ext + qt.padded_row0, kExtBytes, &sm.bar_do_full);
                     last_do = it;
                     if (n == 0) {
@@ -427,8 +440,8 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         mbar_arrive_expect_tx(&sm.bar_kv, 2 * kTileBytes);
 #pragma unroll
                         for (int x = 0; x < kBoxes; ++x) {
-                            tma_load_3d(sm.k + x * kBoxBytesBwd, &map_k, &sm.bar_kv, x * 64, w.j * kTileRows, w.kv_head);
-                            tma_load_3d(sm.v + x * kBoxBytesBwd, &map_v, &sm.bar_kv, x * 64, w.j * kTileRows, w.kv_head);
+                            tma_load_4d(sm.k + x * kBoxBytesBwd, &map_k, &sm.bar_kv, x * 64, w.j * kTileRows, w.g, w.b);
+                            tma_load_4d(sm.v + x * kBoxBytesBwd, &map_v, &sm.bar_kv, x * 64, w.j * kTileRows, w.g, w.b);
                         }
                         ++kv_loads;
                     }
@@ -440,8 +453,8 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                             const BwdItem wn = bwd_item(p, next_item);
 #pragma unroll
                             for (int x = 0; x < kBoxes; ++x) {
-                                tma_prefetch_l2_3d(&map_k, x * 64, wn.j * kTileRows, wn.kv_head);
-                                tma_prefetch_l2_3d(&map_v, x * 64, wn.j * kTileRows, wn.kv_head);
+                                tma_prefetch_l2_4d(&map_k, x * 64, wn.j * kTileRows, wn.g, wn.b);
+                                tma_prefetch_l2_4d(&map_v, x * 64, wn.j * kTileRows, wn.g, wn.b);
                             }
                         }
                     }
@@ -850,7 +863,8 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     const float mult = which == 0 ? dq_mult : inv_p_scale;
                     const uint32_t col0 = which == 0 ? kColdK : kColdV;
                     const int s_row = w.j * kTileRows + row;  // rows past S are never stored
-                    __half *dst = (which == 0 ? p.dK : p.dV) + (static_cast<long long>(w.kv_head) * p.S + s_row) * D;
+                    const lt_tensor_strides &st = which == 0 ? p.dk_st : p.dv_st;
+                    __half *dst = (which == 0 ? p.dK : p.dV) + w.b * st.batch + w.g * st.head + s_row * st.row;
 #pragma unroll
                     for (int c = 0; c < D / 32; ++c) {
                         uint32_t r[32];
@@ -913,10 +927,17 @@ extern "C" int lt_dbg_bwd_trace(unsigned long long *out, int reset) {
 
 template <int D>
 static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, const lt_half *O, const lt_half *dO,
-                      const float *LSE, lt_half *dQ, lt_half *dK, lt_half *dV, int B, int Hq, int Hkv, int S,
-                      int causal, float scale, void *workspace, cudaStream_t stream, cudaEvent_t ev_main_begin,
-                      cudaEvent_t ev_main_end) {
+                      const float *LSE, lt_half *dQ, lt_half *dK, lt_half *dV, const lt_attn_layout &lay, int B,
+                      int Hq, int Hkv, int S, int causal, float scale, void *workspace, cudaStream_t stream,
+                      cudaEvent_t ev_main_begin, cudaEvent_t ev_main_end) {
     const int S_pad = static_cast<int>(padded_rows(S));
+    // fast addressing in the two streaming kernels when nothing is padded or strided
+    auto is_contig = [&](const lt_tensor_strides &st, int H) {
+        const lt_tensor_strides c = contiguous_strides(H, S, D);
+        return st.batch == c.batch && st.head == c.head && st.row == c.row;
+    };
+    const int plain_pre = (S == S_pad && is_contig(lay.d_o, Hq) && is_contig(lay.o, Hq)) ? 1 : 0;
+    const int plain_fin = (S == S_pad && is_contig(lay.dq, Hq)) ? 1 : 0;
     const long long n_rows = static_cast<long long>(B) * Hq * S_pad;  // padded row space of the workspace arrays
     uint8_t *ws = static_cast<uint8_t *>(workspace);
     unsigned int *status = reinterpret_cast<unsigned int *>(ws);
@@ -927,10 +948,10 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
 
     CUtensorMap mq, mk, mv, mdo;
     int rc;
-    if ((rc = make_head_map(&mq, Q, static_cast<uint64_t>(B) * Hq, S, D, 128)) != LT_OK) return rc;
-    if ((rc = make_head_map(&mdo, dO, static_cast<uint64_t>(B) * Hq, S, D, 128)) != LT_OK) return rc;
-    if ((rc = make_head_map(&mk, K, static_cast<uint64_t>(B) * Hkv, S, D, 128)) != LT_OK) return rc;
-    if ((rc = make_head_map(&mv, V, static_cast<uint64_t>(B) * Hkv, S, D, 128)) != LT_OK) return rc;
+    if ((rc = make_bhsd_map(&mq, Q, B, Hq, S, D, lay.q, 128)) != LT_OK) return rc;
+    if ((rc = make_bhsd_map(&mdo, dO, B, Hq, S, D, lay.d_o, 128)) != LT_OK) return rc;
+    if ((rc = make_bhsd_map(&mk, K, B, Hkv, S, D, lay.k, 128)) != LT_OK) return rc;
+    if ((rc = make_bhsd_map(&mv, V, B, Hkv, S, D, lay.v, 128)) != LT_OK) return rc;
 
     cudaError_t e = cudaMemsetAsync(status, 0, kStatusBytes, stream);
     if (e != cudaSuccess) return record_cuda_error("cudaMemsetAsync(status)", e);
@@ -946,7 +967,8 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
     const int pre_blocks = static_cast<int>(want < static_cast<long long>(sms) * 16 ? want : sms * 16);
     bwd_preprocess_kernel<D><<<pre_blocks, 256, 0, stream>>>(reinterpret_cast<const __half *>(dO),
                                                              reinterpret_cast<const __half *>(O), LSE, delta_ext,
-                                                             lse_ext, dq_acc, n_rows, S, S_pad, 1.f / scale, status);
+                                                             lse_ext, dq_acc, n_rows, S, S_pad, Hq, lay.d_o, lay.o, plain_pre,
+                                                             1.f / scale, status);
     e = cudaGetLastError();
     if (e != cudaSuccess) return record_cuda_error("bwd_preprocess_kernel launch", e);
 
@@ -959,6 +981,8 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
     prm.status = status;
     prm.B = B; prm.Hq = Hq; prm.Hkv = Hkv; prm.S = S; prm.S_pad = S_pad; prm.causal = causal ? 1 : 0;
     prm.scale = scale;
+    prm.dk_st = lay.dk;
+    prm.dv_st = lay.dv;
     const size_t smem = sizeof(BwdSmem<D>);
     e = cudaFuncSetAttribute(bwd_main_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return record_cuda_error("cudaFuncSetAttribute(bwd_main)", e);
@@ -976,7 +1000,7 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
     const long long fwant = (n_vec8 + 255) / 256;
     const int fin_blocks = static_cast<int>(fwant < static_cast<long long>(sms) * 16 ? fwant : sms * 16);
     bwd_finalize_kernel<<<fin_blocks, 256, 0, stream>>>(dq_acc, reinterpret_cast<__half *>(dQ), n_vec8, S * (D / 8),
-                                                        S_pad * (D / 8));
+                                                        S_pad * (D / 8), D / 8, Hq, lay.dq, plain_fin);
     e = cudaGetLastError();
     if (e != cudaSuccess) return record_cuda_error("bwd_finalize_kernel launch", e);
     return LT_OK;
@@ -994,14 +1018,16 @@ size_t lt_attn_bwd_workspace_bytes(int B, int Hq, int Hkv, int S, int D) {
 
 int lt_attn_bwd_num_launches(void) { return 3; }
 
-int lt_attn_bwd_profiled(const lt_half *Q, const lt_half *K, const lt_half *V, const lt_half *O, const lt_half *dO,
-                         const float *LSE, lt_half *dQ, lt_half *dK, lt_half *dV, int B, int Hq, int Hkv, int S,
-                         int D, int causal, float scale, void *workspace, size_t workspace_bytes,
-                         lt_stream_t stream, lt_event_t main_begin, lt_event_t main_end) {
+static int bwd_entry(const lt_half *Q, const lt_half *K, const lt_half *V, const lt_half *O, const lt_half *dO,
+                     const float *LSE, lt_half *dQ, lt_half *dK, lt_half *dV, const lt_attn_layout *layout, int B,
+                     int Hq, int Hkv, int S, int D, int causal, float scale, void *workspace, size_t workspace_bytes,
+                     lt_stream_t stream, lt_event_t main_begin, lt_event_t main_end) {
     using namespace lt;
     if (!Q || !K || !V || !O || !dO || !LSE || !dQ || !dK || !dV) return LT_ERR_INVALID_ARG;
     int rc = check_shape(B, Hq, Hkv, S, D, scale);
     if (rc != LT_OK) return rc;
+    const lt_attn_layout lay = layout ? *layout : contiguous_layout(Hq, Hkv, S, D);
+    if (layout && (rc = check_layout(lay, D)) != LT_OK) return rc;
     const void *ptrs[] = {Q, K, V, O, dO, LSE, dQ, dK, dV};
     for (const void *ptr : ptrs)
         if (!aligned16(ptr)) return LT_ERR_UNSUPPORTED;
@@ -1009,10 +1035,26 @@ int lt_attn_bwd_profiled(const lt_half *Q, const lt_half *K, const lt_half *V, c
         return LT_ERR_WORKSPACE;
     if ((rc = check_device()) != LT_OK) return rc;
     if (D == 64)
-        return launch_bwd<64>(Q, K, V, O, dO, LSE, dQ, dK, dV, B, Hq, Hkv, S, causal, scale, workspace, stream,
+        return launch_bwd<64>(Q, K, V, O, dO, LSE, dQ, dK, dV, lay, B, Hq, Hkv, S, causal, scale, workspace, stream,
                               main_begin, main_end);
-    return launch_bwd<128>(Q, K, V, O, dO, LSE, dQ, dK, dV, B, Hq, Hkv, S, causal, scale, workspace, stream,
+    return launch_bwd<128>(Q, K, V, O, dO, LSE, dQ, dK, dV, lay, B, Hq, Hkv, S, causal, scale, workspace, stream,
                            main_begin, main_end);
+}
+
+int lt_attn_bwd_profiled(const lt_half *Q, const lt_half *K, const lt_half *V, const lt_half *O, const lt_half *dO,
+                         const float *LSE, lt_half *dQ, lt_half *dK, lt_half *dV, int B, int Hq, int Hkv, int S,
+                         int D, int causal, float scale, void *workspace, size_t workspace_bytes,
+                         lt_stream_t stream, lt_event_t main_begin, lt_event_t main_end) {
+    return bwd_entry(Q, K, V, O, dO, LSE, dQ, dK, dV, nullptr, B, Hq, Hkv, S, D, causal, scale, workspace,
+                     workspace_bytes, stream, main_begin, main_end);
+}
+
+int lt_attn_bwd_strided(const lt_half *Q, const lt_half *K, const lt_half *V, const lt_half *O, const lt_half *dO,
+                        const float *LSE, lt_half *dQ, lt_half *dK, lt_half *dV, const lt_attn_layout *layout, int B,
+                        int Hq, int Hkv, int S, int D, int causal, float scale, void *workspace,
+                        size_t workspace_bytes, lt_stream_t stream) {
+    return bwd_entry(Q, K, V, O, dO, LSE, dQ, dK, dV, layout, B, Hq, Hkv, S, D, causal, scale, workspace,
+                     workspace_bytes, stream, nullptr, nullptr);
 }
 
 int lt_attn_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, const lt_half *O, const lt_half *dO,

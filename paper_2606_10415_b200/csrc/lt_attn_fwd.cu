@@ -49,6 +49,7 @@ struct FwdParams {
     unsigned int *status;
     int B, Hq, Hkv, S, causal;
     float scale;
+    lt_tensor_strides o_st;  // element strides of O
 };
 
 #ifdef LT_FWD_TRACE
@@ -129,7 +130,6 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
     const uint32_t tmem = sm.tmem_base;
     volatile int *abort_flag = &sm.abort_flag;
 
-    const int kv_head = b * p.Hkv + g;
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer
@@ -138,7 +138,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
                 mbar_arrive_expect_tx(&sm.bar_q[t], kTileBytes);
 #pragma unroll
                 for (int x = 0; x < kBoxes; ++x)
-                    tma_load_3d(sm.q[t] + x * kFwdBoxBytes, &map_q, &sm.bar_q[t], x * 64, (i0 + t) * kFwdTileRows, bh);
+                    tma_load_4d(sm.q[t] + x * kFwdBoxBytes, &map_q, &sm.bar_q[t], x * 64, (i0 + t) * kFwdTileRows, h, b);
             }
             bool ok = true;
             int armed = 0;  // key/value tiles whose loads were started
@@ -150,7 +150,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
                 mbar_arrive_expect_tx(&sm.bar_k_full[s], kTileBytes);
 #pragma unroll
                 for (int x = 0; x < kBoxes; ++x)
-                    tma_load_3d(sm.k[s] + x * kFwdBoxBytes, &map_k, &sm.bar_k_full[s], x * 64, kv_row0, kv_head);
+                    tma_load_4d(sm.k[s] + x * kFwdBoxBytes, &map_k, &sm.bar_k_full[s], x * 64, kv_row0, g, b);
                 if (j >= 2 && !(ok = mbar_wait(&sm.bar_v_empty[s], ph ^ 1, abort_flag, p.status, kWaitFwdVEmpty))) {
                     // the key tile just started still has to land before shared memory is given up
                     for (int w = 0; w < (1 << 16) && !mbar_try_wait(&sm.bar_k_full[s], ph); ++w) {}
@@ -159,7 +159,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
                 mbar_arrive_expect_tx(&sm.bar_v_full[s], kTileBytes);
 #pragma unroll
                 for (int x = 0; x < kBoxes; ++x)
-                    tma_load_3d(sm.v[s] + x * kFwdBoxBytes, &map_v, &sm.bar_v_full[s], x * 64, kv_row0, kv_head);
+                    tma_load_4d(sm.v[s] + x * kFwdBoxBytes, &map_v, &sm.bar_v_full[s], x * 64, kv_row0, g, b);
                 armed = j + 1;
             }
             if (!ok || *abort_flag) {
@@ -389,8 +389,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
             tc_fence_after_sync();
             const float inv_l = 1.f / l;
             const int s_row = i * kFwdTileRows + row;  // rows past S belong to nobody
-            const long long q_row = static_cast<long long>(bh) * p.S + s_row;
-            __half *o_row = p.O + q_row * D;
+            const long long q_row = static_cast<long long>(bh) * p.S + s_row;  // LSE is contiguous
+            __half *o_row = p.O + b * p.o_st.batch + h * p.o_st.head + s_row * p.o_st.row;
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
                 uint32_t r[32];
@@ -427,18 +427,20 @@ extern "C" int lt_dbg_fwd_trace(unsigned long long *out, int reset) {
 #endif
 
 template <int D>
-static int launch_fwd(const lt_half *Q, const lt_half *K, const lt_half *V, lt_half *O, float *LSE, int B, int Hq,
-                      int Hkv, int S, int causal, float scale, void *workspace, cudaStream_t stream) {
+static int launch_fwd(const lt_half *Q, const lt_half *K, const lt_half *V, lt_half *O, float *LSE,
+                      const lt_attn_layout &lay, int B, int Hq, int Hkv, int S, int causal, float scale,
+                      void *workspace, cudaStream_t stream) {
     CUtensorMap mq, mk, mv;
     int rc;
-    if ((rc = make_head_map(&mq, Q, static_cast<uint64_t>(B) * Hq, S, D, 128)) != LT_OK) return rc;
-    if ((rc = make_head_map(&mk, K, static_cast<uint64_t>(B) * Hkv, S, D, 128)) != LT_OK) return rc;
-    if ((rc = make_head_map(&mv, V, static_cast<uint64_t>(B) * Hkv, S, D, 128)) != LT_OK) return rc;
+    if ((rc = make_bhsd_map(&mq, Q, B, Hq, S, D, lay.q, 128)) != LT_OK) return rc;
+    if ((rc = make_bhsd_map(&mk, K, B, Hkv, S, D, lay.k, 128)) != LT_OK) return rc;
+    if ((rc = make_bhsd_map(&mv, V, B, Hkv, S, D, lay.v, 128)) != LT_OK) return rc;
     cudaError_t e = cudaMemsetAsync(workspace, 0, kStatusBytes, stream);
     if (e != cudaSuccess) return record_cuda_error("cudaMemsetAsync(status)", e);
     FwdParams prm;
     prm.O = reinterpret_cast<__half *>(O);
     prm.lse = LSE;
+    prm.o_st = lay.o;
     prm.status = reinterpret_cast<unsigned int *>(workspace);
     prm.B = B; prm.Hq = Hq; prm.Hkv = Hkv; prm.S = S; prm.causal = causal ? 1 : 0;
     prm.scale = scale;
@@ -467,18 +469,31 @@ int lt_attn_fwd_num_launches(void) { return 1; }
 
 int lt_attn_fwd(const lt_half *Q, const lt_half *K, const lt_half *V, lt_half *O, float *LSE, int B, int Hq, int Hkv,
                 int S, int D, int causal, float scale, void *workspace, size_t workspace_bytes, lt_stream_t stream) {
+    return lt_attn_fwd_strided(Q, K, V, O, LSE, nullptr, B, Hq, Hkv, S, D, causal, scale, workspace, workspace_bytes,
+                               stream);
+}
+
+int lt_attn_fwd_strided(const lt_half *Q, const lt_half *K, const lt_half *V, lt_half *O, float *LSE,
+                        const lt_attn_layout *layout, int B, int Hq, int Hkv, int S, int D, int causal, float scale,
+                        void *workspace, size_t workspace_bytes, lt_stream_t stream) {
     using namespace lt;
     if (!Q || !K || !V || !O || !LSE) return LT_ERR_INVALID_ARG;
     int rc = check_shape(B, Hq, Hkv, S, D, scale);
     if (rc != LT_OK) return rc;
+    lt_attn_layout lay = contiguous_layout(Hq, Hkv, S, D);
+    if (layout) {
+        // the forward reads q, k, v, o only; the other entries may be left unset
+        lay.q = layout->q; lay.k = layout->k; lay.v = layout->v; lay.o = layout->o;
+        if ((rc = check_layout(lay, D)) != LT_OK) return rc;
+    }
     const void *ptrs[] = {Q, K, V, O, LSE};
     for (const void *ptr : ptrs)
         if (!aligned16(ptr)) return LT_ERR_UNSUPPORTED;
     if (!workspace || !aligned256(workspace) || workspace_bytes < lt_attn_fwd_workspace_bytes(B, Hq, Hkv, S, D))
         return LT_ERR_WORKSPACE;
     if ((rc = check_device()) != LT_OK) return rc;
-    if (D == 64) return launch_fwd<64>(Q, K, V, O, LSE, B, Hq, Hkv, S, causal, scale, workspace, stream);
-    return launch_fwd<128>(Q, K, V, O, LSE, B, Hq, Hkv, S, causal, scale, workspace, stream);
+    if (D == 64) return launch_fwd<64>(Q, K, V, O, LSE, lay, B, Hq, Hkv, S, causal, scale, workspace, stream);
+    return launch_fwd<128>(Q, K, V, O, LSE, lay, B, Hq, Hkv, S, causal, scale, workspace, stream);
 }
 
 size_t lt_attn_host_arena_bytes(int B, int Hq, int Hkv, int S, int D) {

@@ -80,15 +80,17 @@ int make_tile_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t co
     return LT_OK;
 }
 
-int make_head_map(CUtensorMap *map, const void *base, uint64_t heads, uint64_t rows_per_head, uint64_t cols,
-                  uint32_t box_rows) {
+int make_bhsd_map(CUtensorMap *map, const void *base, uint64_t B, uint64_t H, uint64_t S, uint64_t D,
+                  const lt_tensor_strides &st, uint32_t box_rows) {
     EncodeTiledFn enc = get_encoder();
     if (!enc) return LT_ERR_CUDA;
-    cuuint64_t dims[3] = {cols, rows_per_head, heads};
-    cuuint64_t strides[2] = {cols * sizeof(__half), rows_per_head * cols * sizeof(__half)};
-    cuuint32_t box[3] = {64u, box_rows, 1u};
-    cuuint32_t estr[3] = {1u, 1u, 1u};
-    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+    cuuint64_t dims[4] = {D, S, H, B};
+    cuuint64_t strides[3] = {static_cast<cuuint64_t>(st.row) * sizeof(__half),
+                             static_cast<cuuint64_t>(st.head) * sizeof(__half),
+                             static_cast<cuuint64_t>(st.batch) * sizeof(__half)};
+    cuuint32_t box[4] = {64u, box_rows, 1u, 1u};
+    cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -96,6 +98,24 @@ int make_head_map(CUtensorMap *map, const void *base, uint64_t heads, uint64_t r
         snprintf(buf, sizeof(buf), "CUresult %d", static_cast<int>(r));
         set_last_error("cuTensorMapEncodeTiled", buf);
         return LT_ERR_CUDA;
+    }
+    return LT_OK;
+}
+
+lt_attn_layout contiguous_layout(int Hq, int Hkv, int S, int D) {
+    lt_attn_layout lay;
+    lay.q = lay.o = lay.d_o = lay.dq = contiguous_strides(Hq, S, D);
+    lay.k = lay.v = lay.dk = lay.dv = contiguous_strides(Hkv, S, D);
+    return lay;
+}
+
+int check_layout(const lt_attn_layout &lay, int D) {
+    const lt_tensor_strides *all[] = {&lay.q, &lay.k, &lay.v, &lay.o, &lay.d_o, &lay.dq, &lay.dk, &lay.dv};
+    for (const lt_tensor_strides *st : all) {
+        const long long v[3] = {st->batch, st->head, st->row};
+        for (long long x : v)
+            if (x <= 0 || (x % 8) != 0 || x >= (1LL << 38)) return LT_ERR_UNSUPPORTED;
+        if (st->row < D) return LT_ERR_UNSUPPORTED;
     }
     return LT_OK;
 }

@@ -29,10 +29,22 @@ inline size_t round256(size_t n) { return (n + 255u) & ~static_cast<size_t>(255u
 // fp16 matrix [rows, cols] row-major viewed as a 2-D tensor; tiles of box_rows x 64
 // columns are fetched with the 128-byte swizzle.  Returns LT_OK or LT_ERR_CUDA.
 int make_tile_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows);
-// 3-D view [heads][rows_per_head][cols] of a contiguous fp16 tensor with boxes of 64 columns x
-// box_rows rows x 1 head (128-byte swizzle); rows past the end of a head are filled with zeros.
-int make_head_map(CUtensorMap *map, const void *base, uint64_t heads, uint64_t rows_per_head, uint64_t cols,
-                  uint32_t box_rows);
+// 4-D view [batch][head][row][element] of an fp16 tensor with the given element strides (boxes of
+// 64 elements x box_rows rows of one head, 128-byte swizzle, zero fill past the last row).
+int make_bhsd_map(CUtensorMap *map, const void *base, uint64_t B, uint64_t H, uint64_t S, uint64_t D,
+                  const lt_tensor_strides &st, uint32_t box_rows);
+// strides of a contiguous [B,H,S,D] tensor
+inline lt_tensor_strides contiguous_strides(int H, int S, int D) {
+    lt_tensor_strides st;
+    st.row = D;
+    st.head = static_cast<long long>(S) * D;
+    st.batch = static_cast<long long>(H) * S * D;
+    return st;
+}
+// every tensor contiguous [B,H,S,D]
+lt_attn_layout contiguous_layout(int Hq, int Hkv, int S, int D);
+// LT_OK if every stride of the layout is a positive multiple of 8 elements and rows hold D elements
+int check_layout(const lt_attn_layout &lay, int D);
 // sequence length rounded up to whole 128-row tiles
 inline long long padded_rows(int S) { return (static_cast<long long>(S) + 127) / 128 * 128; }
 

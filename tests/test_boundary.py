@@ -100,3 +100,35 @@ def test_no_gpu_means_a_loud_error_not_a_fallback(binding):
     # arguments are valid, so the call reaches the device check and must fail there
     rc = binding.lt_attn_bwd_raw(*_bwd_args())
     assert rc in (binding.LT_ERR_CUDA, binding.LT_ERR_UNSUPPORTED)
+
+
+def test_strided_entry_points_reject_bad_strides(binding):
+    """Layout checks happen on the host before anything is launched."""
+    import ctypes
+    b = binding
+    lib = b._lib
+
+    def layout(**over):
+        lay = b.AttnLayout()
+        for name in ("q", "k", "v", "o", "d_o", "dq", "dk", "dv"):
+            setattr(lay, name, b.TensorStrides(2 * 128 * 64, 128 * 64, 64))
+        for name, st in over.items():
+            setattr(lay, name, b.TensorStrides(*st))
+        return lay
+
+    def bwd(lay, ws_bytes=1 << 20):
+        return lib.lt_attn_bwd_strided(*([0x1000] * 9), ctypes.byref(lay), 1, 2, 2, 128, 64, 1, 0.125, 0x10000,
+                                       ws_bytes, 0)
+
+    def fwd(lay, ws_bytes=256):
+        return lib.lt_attn_fwd_strided(*([0x1000] * 5), ctypes.byref(lay), 1, 2, 2, 128, 64, 1, 0.125, 0x10000,
+                                       ws_bytes, 0)
+
+    # a valid layout gets past the stride checks (and then fails for lack of a workspace / device)
+    assert bwd(layout(), ws_bytes=16) == b.LT_ERR_WORKSPACE
+    assert bwd(layout(dk=(2 * 128 * 64, 128 * 64, 60))) == b.LT_ERR_UNSUPPORTED      # row stride below D
+    assert bwd(layout(q=(2 * 128 * 64, 128 * 64 + 4, 64))) == b.LT_ERR_UNSUPPORTED   # not a multiple of 8 elements
+    assert bwd(layout(d_o=(0, 128 * 64, 64))) == b.LT_ERR_UNSUPPORTED                # zero stride
+    assert fwd(layout(o=(2 * 128 * 64, 128 * 64, -64))) == b.LT_ERR_UNSUPPORTED
+    # the forward ignores the gradient entries: it gets as far as the workspace check (nothing is launched)
+    assert fwd(layout(dq=(1, 1, 1)), ws_bytes=16) == b.LT_ERR_WORKSPACE

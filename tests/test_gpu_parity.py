@@ -210,6 +210,77 @@ def test_host_buffer_entry_point(lt, oracle):
     check_grads((dQ, dK, dV), ref, "host entry")
 
 
+# ------------------------------------------------------------------ strided layouts
+
+def _strided_case(lt, oracle, cfg, make_views):
+    """Run forward and backward on [B,H,S,D] views built by `make_views` and compare with the
+    oracle on contiguous copies of the same values."""
+    Q, K, V, dO = workloads.make_inputs(cfg)
+    Qv, Kv, Vv, Ov, dOv, dQv, dKv, dVv = make_views(Q, K, V, dO)
+    LSE = torch.empty(Q.shape[:3], dtype=torch.float32, device="cuda")
+    fws = lt.alloc_workspace(lt.lt_attn_fwd_workspace_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.S, cfg.D))
+    lt.lt_attn_fwd_strided(Qv, Kv, Vv, Ov, LSE, cfg.causal, cfg.scale, fws)
+    assert lt.lt_attn_check_status(fws) == lt.LT_OK, lt.last_cuda_error()
+    Qn, Kn, Vn, dOn = (t.double().numpy() for t in (Q, K, V, dO))
+    O_ref, LSE_ref = oracle.attn_fwd(Qn, Kn, Vn, cfg.causal, cfg.scale)
+    assert rel_fro(Ov.cpu().double().numpy(), O_ref) <= FWD_O_REL_FRO_TOL
+    assert max_abs(LSE.cpu().double().numpy(), LSE_ref) <= FWD_LSE_ABS_TOL
+    ws = lt.alloc_workspace(lt.lt_attn_bwd_workspace_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.S, cfg.D))
+    ws.fill_(0xFF)
+    lt.lt_attn_bwd_strided(Qv, Kv, Vv, Ov, dOv, LSE, dQv, dKv, dVv, cfg.causal, cfg.scale, ws)
+    assert lt.lt_attn_check_status(ws) == lt.LT_OK, lt.last_cuda_error()
+    ref = oracle.attn_bwd(Qn, Kn, Vn, dOn, cfg.causal, cfg.scale)
+    check_grads((dQv.cpu(), dKv.cpu(), dVv.cpu()), ref, f"strided {cfg}")
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,S,D,causal", [
+    (2, 4, 2, 256, 128, True), (1, 3, 3, 200, 64, True), (2, 2, 1, 130, 128, False),
+])
+def test_bshd_layout_matches_oracle(lt, oracle, B, Hq, Hkv, S, D, causal):
+    """Every tensor stored [B,S,H,D] and handed over as a permuted [B,H,S,D] view."""
+    cfg = workloads.custom(B, Hq, Hkv, S, D, causal, qkv_std=1.0, do_std=1.0, seed=31 + S)
+
+    def views(Q, K, V, dO):
+        def bshd(t):
+            return t.permute(0, 2, 1, 3).contiguous().cuda().permute(0, 2, 1, 3)
+
+        def out_like(t):
+            return torch.full_like(t.permute(0, 2, 1, 3).contiguous(), float("nan"), device="cuda").permute(0, 2, 1, 3)
+
+        return bshd(Q), bshd(K), bshd(V), out_like(Q), bshd(dO), out_like(Q), out_like(K), out_like(V)
+
+    _strided_case(lt, oracle, cfg, views)
+
+
+def test_fused_qkv_buffer_matches_oracle(lt, oracle):
+    """Q, K, V are slices of one [B, S, (Hq + 2 Hkv) * D] projection output; dQ, dK, dV are written
+    into the matching slices of one gradient buffer; untouched bytes of that buffer stay as they were."""
+    B, Hq, Hkv, S, D = 2, 4, 2, 300, 128
+    cfg = workloads.custom(B, Hq, Hkv, S, D, True, seed=77)
+    width = (Hq + 2 * Hkv) * D
+    pad = 64  # spare elements at the end of every row, never written
+
+    def views(Q, K, V, dO):
+        buf = torch.zeros(B, S, width + pad, dtype=torch.float16, device="cuda")
+        grad = torch.full((B, S, width + pad), 7.0, dtype=torch.float16, device="cuda")
+
+        def split(t):
+            q = t[..., :Hq * D].unflatten(-1, (Hq, D)).permute(0, 2, 1, 3)
+            k = t[..., Hq * D:(Hq + Hkv) * D].unflatten(-1, (Hkv, D)).permute(0, 2, 1, 3)
+            v = t[..., (Hq + Hkv) * D:width].unflatten(-1, (Hkv, D)).permute(0, 2, 1, 3)
+            return q, k, v
+
+        q, k, v = split(buf)
+        q.copy_(Q.cuda()); k.copy_(K.cuda()); v.copy_(V.cuda())
+        dq, dk, dv = split(grad)
+        views.grad = grad
+        O = torch.empty(B, Hq, S, D, dtype=torch.float16, device="cuda")
+        return q, k, v, O, dO.cuda(), dq, dk, dv
+
+    _strided_case(lt, oracle, cfg, views)
+    assert torch.all(views.grad[..., width:] == 7.0)
+
+
 # ------------------------------------------------------------------ benchmark configurations, full size
 
 def _full_size_check(lt, oracle, name, units):
