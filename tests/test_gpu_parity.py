@@ -197,6 +197,73 @@ def test_zero_dO_gives_zero_gradients(lt):
         assert torch.count_nonzero(g) == 0
 
 
+@pytest.mark.parametrize("do_std", [1e-3, 30.0])
+def test_gradient_magnitude_extremes(lt, oracle, do_std):
+    """The fp16 dS operand carries a per-work-item power-of-two factor chosen from a bound on
+    |dP - delta|; upstream gradients far below and above the usual range must keep the relative
+    accuracy.  (Below about 1e-3 the fp16 outputs themselves go subnormal, which no kernel can mend.)"""
+    cfg = workloads.custom(1, 4, 2, 384, 128, True, qkv_std=128.0 ** -0.25, do_std=do_std, seed=21)
+    Q, K, V, dO = workloads.make_inputs(cfg)
+    Qn, Kn, Vn, dOn = (t.double().numpy() for t in (Q, K, V, dO))
+    O_ref, LSE_ref = oracle.attn_fwd(Qn, Kn, Vn, True, cfg.scale)
+    ref = oracle.attn_bwd(Qn, Kn, Vn, dOn, True, cfg.scale)
+    got = run_bwd(lt, Q, K, V, torch.from_numpy(O_ref).half(), dO, torch.from_numpy(LSE_ref).float(), cfg)
+    for name, g, r in zip(("dQ", "dK", "dV"), got, ref):
+        g = g.double().numpy()
+        assert np.all(np.isfinite(g)), name
+        assert rel_fro(g, r) <= REL_FRO_TOL, f"{name} at dO std {do_std}: {rel_fro(g, r):.3e}"
+
+
+def test_sharp_softmax_and_large_scores(lt, oracle):
+    """Large |scores| (std 4 after scaling): rows dominated by one key, LSE far from 0, probabilities
+    spanning the whole fp16 range; also exercises the forward's running-maximum updates."""
+    cfg = workloads.custom(1, 2, 2, 512, 64, True, qkv_std=2.0, do_std=1.0, seed=22)
+    Q, K, V, dO = workloads.make_inputs(cfg)
+    O, LSE = run_fwd(lt, Q, K, V, cfg)
+    Qn, Kn, Vn, dOn = (t.double().numpy() for t in (Q, K, V, dO))
+    O_ref, LSE_ref = oracle.attn_fwd(Qn, Kn, Vn, True, cfg.scale)
+    assert rel_fro(O.cpu().double().numpy(), O_ref) <= FWD_O_REL_FRO_TOL
+    assert max_abs(LSE.cpu().double().numpy(), LSE_ref) <= 4 * FWD_LSE_ABS_TOL  # |LSE| itself is ~50 here
+    got = run_bwd(lt, Q, K, V, O.cpu(), dO, LSE.cpu(), cfg)
+    ref = oracle.attn_bwd(Qn, Kn, Vn, dOn, True, cfg.scale)
+    check_grads(got, ref, "sharp softmax")
+
+
+def test_negative_scale(lt, oracle):
+    """A negative softmax scale is legal (finite, non-zero): the row maximum then comes from the
+    smallest raw score."""
+    cfg = workloads.custom(1, 2, 1, 256, 128, True, qkv_std=1.0, do_std=1.0, seed=23)
+    Q, K, V, dO = workloads.make_inputs(cfg)
+    scale = -cfg.scale
+    Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+    O = torch.empty_like(Qd)
+    LSE = torch.empty(Q.shape[:3], dtype=torch.float32, device="cuda")
+    fws = lt.alloc_workspace(lt.lt_attn_fwd_workspace_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.S, cfg.D))
+    lt.lt_attn_fwd(Qd, Kd, Vd, O, LSE, True, scale, fws)
+    assert lt.lt_attn_check_status(fws) == lt.LT_OK
+    Qn, Kn, Vn, dOn = (t.double().numpy() for t in (Q, K, V, dO))
+    O_ref, LSE_ref = oracle.attn_fwd(Qn, Kn, Vn, True, scale)
+    assert rel_fro(O.cpu().double().numpy(), O_ref) <= FWD_O_REL_FRO_TOL
+    assert max_abs(LSE.cpu().double().numpy(), LSE_ref) <= FWD_LSE_ABS_TOL
+    dQ, dK, dV = torch.empty_like(Qd), torch.empty_like(Kd), torch.empty_like(Vd)
+    ws = lt.alloc_workspace(lt.lt_attn_bwd_workspace_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.S, cfg.D))
+    lt.lt_attn_bwd(Qd, Kd, Vd, O, dO.cuda(), LSE, dQ, dK, dV, True, scale, ws)
+    assert lt.lt_attn_check_status(ws) == lt.LT_OK
+    ref = oracle.attn_bwd(Qn, Kn, Vn, dOn, True, scale)
+    check_grads((dQ.cpu(), dK.cpu(), dV.cpu()), ref, "negative scale")
+
+
+def test_long_sequence_and_wide_group(lt, oracle):
+    """S = 8192 (64 key tiles, long dQ accumulation chains) with a group of 16 query heads on one
+    key/value head."""
+    cfg = workloads.custom(1, 16, 1, 8192, 128, True, seed=24)
+    Q, K, V, dO = workloads.make_inputs(cfg)
+    O, LSE = run_fwd(lt, Q, K, V, cfg)
+    got = run_bwd(lt, Q, K, V, O.cpu(), dO, LSE.cpu(), cfg)
+    ref = oracle.attn_bwd(*(t.double().numpy() for t in (Q, K, V, dO)), True, cfg.scale)
+    check_grads(got, ref, "S=8192, group of 16")
+
+
 def test_host_buffer_entry_point(lt, oracle):
     cfg = workloads.custom(1, 4, 2, 256, 128, True, seed=13)
     Q, K, V, dO = (t.pin_memory() for t in workloads.make_inputs(cfg))
