@@ -52,6 +52,8 @@ typedef struct CUstream_st *lt_stream_t;
 typedef struct CUevent_st *lt_event_t;
 /* fp16 storage type (bit pattern of an IEEE binary16). */
 typedef unsigned short lt_half;
+/* bfloat16 storage (the upper 16 bits of an IEEE binary32) */
+typedef unsigned short lt_bf16;
 
 /* Bytes of caller-owned device workspace the calls below need; 0 means the shape is
  * not supported.  The workspace must be 256-byte aligned.  Layout (backward): a
@@ -147,6 +149,23 @@ int lt_attn_bwd_strided(const lt_half *Q, const lt_half *K, const lt_half *V,
                         lt_half *dQ, lt_half *dK, lt_half *dV, const lt_attn_layout *layout,
                         int B, int Hq, int Hkv, int S, int D, int causal, float scale,
                         void *workspace, size_t workspace_bytes, lt_stream_t stream);
+
+/* The same two computations with every 16-bit tensor (Q, K, V, O, dO, dQ, dK, dV) in bfloat16
+ * instead of fp16; LSE stays fp32.  Products run on the same tensor-core path with bf16 operands
+ * and fp32 accumulation; P and dS are rounded to bf16 (8 significant bits) before their products, so
+ * the gradients carry about 2^-9 relative rounding per element where the fp16 path carries 2^-11.
+ * `layout` as for the strided entry points (NULL = contiguous [B,H,S,D]).  Workspace sizes, status
+ * codes and error behaviour are those of lt_attn_fwd / lt_attn_bwd.  The paper's datapath is FP16
+ * (Section 4.1); bf16 is the format most current training stacks hand to the same operator. */
+int lt_attn_fwd_bf16(const lt_bf16 *Q, const lt_bf16 *K, const lt_bf16 *V,
+                     lt_bf16 *O, float *LSE, const lt_attn_layout *layout,
+                     int B, int Hq, int Hkv, int S, int D, int causal, float scale,
+                     void *workspace, size_t workspace_bytes, lt_stream_t stream);
+int lt_attn_bwd_bf16(const lt_bf16 *Q, const lt_bf16 *K, const lt_bf16 *V,
+                     const lt_bf16 *O, const lt_bf16 *dO, const float *LSE,
+                     lt_bf16 *dQ, lt_bf16 *dK, lt_bf16 *dV, const lt_attn_layout *layout,
+                     int B, int Hq, int Hkv, int S, int D, int causal, float scale,
+                     void *workspace, size_t workspace_bytes, lt_stream_t stream);
 
 /* Same computation as lt_attn_fwd followed by lt_attn_bwd, but every tensor pointer is
  * a HOST pointer (pinned memory makes the copies asynchronous).  `arena` is a caller-

@@ -24,6 +24,7 @@ LT_ERR_DEVICE_TIMEOUT = 5
 EXPORTS = (
     "lt_attn_fwd_workspace_bytes", "lt_attn_bwd_workspace_bytes", "lt_attn_fwd", "lt_attn_bwd",
     "lt_attn_bwd_profiled", "lt_attn_bwd_noalloc", "lt_attn_fwd_strided", "lt_attn_bwd_strided",
+    "lt_attn_fwd_bf16", "lt_attn_bwd_bf16",
     "lt_attn_host_arena_bytes", "lt_attn_fwd_bwd_host", "lt_attn_check_status", "lt_status_string",
     "lt_last_cuda_error", "lt_attn_bwd_num_launches", "lt_attn_fwd_num_launches", "lt_dbg_tile_gemm",
     "lt_dbg_wait_timeout",
@@ -70,6 +71,10 @@ def _load() -> ctypes.CDLL:
     lib.lt_attn_fwd_strided.restype = i
     lib.lt_attn_bwd_strided.argtypes = [vp] * 9 + [ctypes.POINTER(AttnLayout)] + [i] * 6 + [f, vp, sz, vp]
     lib.lt_attn_bwd_strided.restype = i
+    lib.lt_attn_fwd_bf16.argtypes = lib.lt_attn_fwd_strided.argtypes
+    lib.lt_attn_fwd_bf16.restype = i
+    lib.lt_attn_bwd_bf16.argtypes = lib.lt_attn_bwd_strided.argtypes
+    lib.lt_attn_bwd_bf16.restype = i
     lib.lt_attn_bwd_noalloc.argtypes = [vp] * 9 + [i] * 6 + [f, vp]
     lib.lt_attn_bwd_noalloc.restype = i
     lib.lt_attn_fwd_bwd_host.argtypes = [vp] * 9 + [i] * 6 + [f, vp, sz, vp]
@@ -206,6 +211,41 @@ def lt_attn_bwd_strided(Q, K, V, O, dO, LSE, dQ, dK, dV, causal, scale, workspac
                                   _stream_ptr(stream))
     if rc != LT_OK:
         raise LtError("lt_attn_bwd_strided", rc)
+
+
+def _require_dtype(dtype, *tensors):
+    for t in tensors:
+        if t.dtype != dtype:
+            raise ValueError(f"expected {dtype} tensors, got {t.dtype}")
+
+
+def lt_attn_fwd_bf16(Q, K, V, O, LSE, causal, scale, workspace, stream=None) -> None:
+    """lt_attn_fwd with bfloat16 Q, K, V, O ([B, H, S, D] views; strides are taken from the tensors)."""
+    _require_dtype(torch.bfloat16, Q, K, V, O)
+    _check_layout(LSE)
+    B, Hq, Hkv, S, D = _dims(Q, K)
+    lay = AttnLayout()
+    lay.q, lay.k, lay.v, lay.o = (_strides_of(t) for t in (Q, K, V, O))
+    rc = _lib.lt_attn_fwd_bf16(_ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(LSE), ctypes.byref(lay), B, Hq, Hkv, S, D,
+                               int(bool(causal)), float(scale), _ptr(workspace),
+                               workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    if rc != LT_OK:
+        raise LtError("lt_attn_fwd_bf16", rc)
+
+
+def lt_attn_bwd_bf16(Q, K, V, O, dO, LSE, dQ, dK, dV, causal, scale, workspace, stream=None) -> None:
+    """lt_attn_bwd with bfloat16 tensors ([B, H, S, D] views; strides are taken from the tensors)."""
+    _require_dtype(torch.bfloat16, Q, K, V, O, dO, dQ, dK, dV)
+    _check_layout(LSE)
+    B, Hq, Hkv, S, D = _dims(Q, K)
+    lay = AttnLayout()
+    lay.q, lay.k, lay.v, lay.o, lay.d_o, lay.dq, lay.dk, lay.dv = (
+        _strides_of(t) for t in (Q, K, V, O, dO, dQ, dK, dV))
+    rc = _lib.lt_attn_bwd_bf16(_ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(dO), _ptr(LSE), _ptr(dQ), _ptr(dK), _ptr(dV),
+                               ctypes.byref(lay), B, Hq, Hkv, S, D, int(bool(causal)), float(scale), _ptr(workspace),
+                               workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    if rc != LT_OK:
+        raise LtError("lt_attn_bwd_bf16", rc)
 
 
 def lt_attn_bwd_profiled(Q, K, V, O, dO, LSE, dQ, dK, dV, causal, scale, workspace, stream=None,

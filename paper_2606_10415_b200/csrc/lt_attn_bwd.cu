@@ -55,7 +55,7 @@ enum {
 // keep HBM busy.
 constexpr int kPreUnroll = 4;
 
-template <int D>
+template <int D, bool kBf16>
 __global__ void __launch_bounds__(256)
 bwd_preprocess_kernel(const __half *__restrict__ dO, const __half *__restrict__ O, const float *__restrict__ lse,
                       uint4 *__restrict__ delta_ext, uint4 *__restrict__ lse_ext, float *__restrict__ dq_acc,
@@ -107,13 +107,13 @@ bwd_preprocess_kernel(const __half *__restrict__ dO, const __half *__restrict__ 
 #pragma unroll
         for (int u = 0; u < kPreUnroll; ++u) {
             const long long row = row0 + u * kRowsPerWarp + lane / kLanesPerRow;
-            const __half2 *ah = reinterpret_cast<const __half2 *>(&a[u]);
-            const __half2 *bh = reinterpret_cast<const __half2 *>(&b[u]);
+            const uint32_t *ah = reinterpret_cast<const uint32_t *>(&a[u]);
+            const uint32_t *bh = reinterpret_cast<const uint32_t *>(&b[u]);
             float acc = 0.f, n2 = 0.f;
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                const float2 x = __half22float2(ah[e]);
-                const float2 y = __half22float2(bh[e]);
+                const float2 x = unpack2<kBf16>(ah[e]);
+                const float2 y = unpack2<kBf16>(bh[e]);
                 acc = fmaf(x.x, y.x, acc);
                 acc = fmaf(x.y, y.y, acc);
                 n2 = fmaf(x.x, x.x, n2);
@@ -127,8 +127,8 @@ bwd_preprocess_kernel(const __half *__restrict__ dO, const __half *__restrict__ 
             if (row < n_rows) {
                 if (sub == 0) {
                     // operand rows of the main kernel's extra contraction step: 256*hi + lo = value
-                    delta_ext[row] = make_uint4(split_hi_lo(-acc), 0u, 0u, 0u);
-                    lse_ext[row] = make_uint4(split_hi_lo(-l[u] * inv_scale), 0u, 0u, 0u);
+                    delta_ext[row] = split_ext<kBf16>(-acc);
+                    lse_ext[row] = split_ext<kBf16>(-l[u] * inv_scale);
                 }
                 max_abs_delta = fmaxf(max_abs_delta, fabsf(acc));
                 max_norm2 = fmaxf(max_norm2, n2);
@@ -159,6 +159,7 @@ bwd_preprocess_kernel(const __half *__restrict__ dO, const __half *__restrict__ 
 }
 
 // ----------------------------------------------------------------------------- finalize
+template <bool kBf16>
 __global__ void __launch_bounds__(256)
 bwd_finalize_kernel(const float *__restrict__ dq_acc, __half *__restrict__ dQ, long long n_vec8, int vec_per_head,
                     int vec_per_padded_head, int vec_per_row, int Hq, lt_tensor_strides dq_st, int plain) {
@@ -178,10 +179,10 @@ bwd_finalize_kernel(const float *__restrict__ dq_acc, __half *__restrict__ dQ, l
         const float4 a = __ldcs(reinterpret_cast<const float4 *>(dq_acc) + 2 * src);
         const float4 b = __ldcs(reinterpret_cast<const float4 *>(dq_acc) + 2 * src + 1);
         uint4 o;
-        o.x = pack_half2(a.x, a.y);
-        o.y = pack_half2(a.z, a.w);
-        o.z = pack_half2(b.x, b.y);
-        o.w = pack_half2(b.z, b.w);
+        o.x = pack2<kBf16>(a.x, a.y);
+        o.y = pack2<kBf16>(a.z, a.w);
+        o.z = pack2<kBf16>(b.x, b.y);
+        o.w = pack2<kBf16>(b.z, b.w);
         *reinterpret_cast<uint4 *>(dQ + dst) = o;
     }
 }
@@ -320,7 +321,7 @@ __device__ __forceinline__ BwdQTile bwd_q_tile(const BwdParams &p, const BwdItem
     return q;
 }
 
-template <int D>
+template <int D, bool kBf16>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
@@ -376,9 +377,9 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     }
     if (warp == 1) {
         // constant operands of the extra contraction step
-        const __half2 ones = __halves2half2(__float2half_rn(256.f), __float2half_rn(1.f));
+        const uint2 mult = ext_multipliers<kBf16>();
         for (int r = lane; r < kTileRows; r += 32) {
-            reinterpret_cast<uint4 *>(sm.ext_ones)[r] = make_uint4(*reinterpret_cast<const uint32_t *>(&ones), 0u, 0u, 0u);
+            reinterpret_cast<uint4 *>(sm.ext_ones)[r] = make_uint4(mult.x, mult.y, 0u, 0u);
             reinterpret_cast<uint4 *>(sm.ext_zero)[r] = make_uint4(0u, 0u, 0u, 0u);
         }
         fence_proxy_async_smem();
@@ -498,9 +499,9 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             // tile (16 rows of 128 bytes per step)
             auto koff = [](int kk) -> uint64_t { return static_cast<uint64_t>((kk >> 2) * (kBoxBytesBwd >> 4) + (kk & 3) * 2); };
             auto roff = [](int kk) -> uint64_t { return static_cast<uint64_t>(kk * (2048 >> 4)); };
-            constexpr uint32_t idesc_s = make_idesc(128, 128, false, false);
-            constexpr uint32_t idesc_dv = make_idesc(128, D, false, true);
-            constexpr uint32_t idesc_dq = make_idesc(128, D == 128 ? 128 : D, true, true);
+            constexpr uint32_t idesc_s = make_idesc(128, 128, false, false, kBf16);
+            constexpr uint32_t idesc_dv = make_idesc(128, D, false, true, kBf16);
+            constexpr uint32_t idesc_dq = make_idesc(128, D == 128 ? 128 : D, true, true, kBf16);
             auto issue_s = [&](int t) {  // S^T = K_j Q_i^T - LSE_i / scale, for running iteration t
                 const uint64_t dQ_k = dQ_k0 + (t & 1) * kQStageStep;
 #pragma unroll
@@ -626,7 +627,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 uint32_t out[16];
 #pragma unroll
                 for (int e = 0; e < 16; ++e)
-                    out[e] = pack_half2(__uint_as_float(pv[c * 32 + 2 * e]), __uint_as_float(pv[c * 32 + 2 * e + 1]));
+                    out[e] = pack2<kBf16>(__uint_as_float(pv[c * 32 + 2 * e]), __uint_as_float(pv[c * 32 + 2 * e + 1]));
                 // in place: these columns lie inside the 64 columns this thread has just read
                 tmem_st16(tmem + lane_base + kColS + cbase + c * 16, out);
             }
@@ -656,10 +657,10 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
                         const uint4 u = src[(c + row) & 7];  // rotated start: conflict-free across the warp
-                        const __half2 *h = reinterpret_cast<const __half2 *>(&u);
+                        const uint32_t *h = reinterpret_cast<const uint32_t *>(&u);
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            const float2 f = __half22float2(h[e]);
+                            const float2 f = unpack2<kBf16>(h[e]);
                             n2 = fmaf(f.x, f.x, n2);
                             n2 = fmaf(f.y, f.y, n2);
                         }
@@ -706,7 +707,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     uint32_t o[16];
 #pragma unroll
                     for (int e = 0; e < 16; ++e)
-                        o[e] = pack_half2(__uint_as_float(pv[c * 32 + 2 * e]) * __uint_as_float(dp[2 * e]),
+                        o[e] = pack2<kBf16>(__uint_as_float(pv[c * 32 + 2 * e]) * __uint_as_float(dp[2 * e]),
                                           __uint_as_float(pv[c * 32 + 2 * e + 1]) * __uint_as_float(dp[2 * e + 1]));
 #pragma unroll
                     for (int v4 = 0; v4 < 4; ++v4)
@@ -879,10 +880,10 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #pragma unroll
                         for (int v8 = 0; v8 < 4; ++v8) {
                             uint4 o;
-                            o.x = pack_half2(__uint_as_float(r[8 * v8 + 0]) * mult, __uint_as_float(r[8 * v8 + 1]) * mult);
-                            o.y = pack_half2(__uint_as_float(r[8 * v8 + 2]) * mult, __uint_as_float(r[8 * v8 + 3]) * mult);
-                            o.z = pack_half2(__uint_as_float(r[8 * v8 + 4]) * mult, __uint_as_float(r[8 * v8 + 5]) * mult);
-                            o.w = pack_half2(__uint_as_float(r[8 * v8 + 6]) * mult, __uint_as_float(r[8 * v8 + 7]) * mult);
+                            o.x = pack2<kBf16>(__uint_as_float(r[8 * v8 + 0]) * mult, __uint_as_float(r[8 * v8 + 1]) * mult);
+                            o.y = pack2<kBf16>(__uint_as_float(r[8 * v8 + 2]) * mult, __uint_as_float(r[8 * v8 + 3]) * mult);
+                            o.z = pack2<kBf16>(__uint_as_float(r[8 * v8 + 4]) * mult, __uint_as_float(r[8 * v8 + 5]) * mult);
+                            o.w = pack2<kBf16>(__uint_as_float(r[8 * v8 + 6]) * mult, __uint_as_float(r[8 * v8 + 7]) * mult);
                             if (s_row < p.S) reinterpret_cast<uint4 *>(dst + c * 32)[v8] = o;
                         }
                     }
@@ -925,7 +926,7 @@ extern "C" int lt_dbg_bwd_trace(unsigned long long *out, int reset) {
 }
 #endif
 
-template <int D>
+template <int D, bool kBf16>
 static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, const lt_half *O, const lt_half *dO,
                       const float *LSE, lt_half *dQ, lt_half *dK, lt_half *dV, const lt_attn_layout &lay, int B,
                       int Hq, int Hkv, int S, int causal, float scale, void *workspace, cudaStream_t stream,
@@ -948,10 +949,10 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
 
     CUtensorMap mq, mk, mv, mdo;
     int rc;
-    if ((rc = make_bhsd_map(&mq, Q, B, Hq, S, D, lay.q, 128)) != LT_OK) return rc;
-    if ((rc = make_bhsd_map(&mdo, dO, B, Hq, S, D, lay.d_o, 128)) != LT_OK) return rc;
-    if ((rc = make_bhsd_map(&mk, K, B, Hkv, S, D, lay.k, 128)) != LT_OK) return rc;
-    if ((rc = make_bhsd_map(&mv, V, B, Hkv, S, D, lay.v, 128)) != LT_OK) return rc;
+    if ((rc = make_bhsd_map(&mq, Q, B, Hq, S, D, lay.q, 128, kBf16)) != LT_OK) return rc;
+    if ((rc = make_bhsd_map(&mdo, dO, B, Hq, S, D, lay.d_o, 128, kBf16)) != LT_OK) return rc;
+    if ((rc = make_bhsd_map(&mk, K, B, Hkv, S, D, lay.k, 128, kBf16)) != LT_OK) return rc;
+    if ((rc = make_bhsd_map(&mv, V, B, Hkv, S, D, lay.v, 128, kBf16)) != LT_OK) return rc;
 
     cudaError_t e = cudaMemsetAsync(status, 0, kStatusBytes, stream);
     if (e != cudaSuccess) return record_cuda_error("cudaMemsetAsync(status)", e);
@@ -965,7 +966,7 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
     constexpr int kRowsPerBlock = 8 * (32 / (D / 8)) * kPreUnroll;
     const long long want = (n_rows + kRowsPerBlock - 1) / kRowsPerBlock;
     const int pre_blocks = static_cast<int>(want < static_cast<long long>(sms) * 16 ? want : sms * 16);
-    bwd_preprocess_kernel<D><<<pre_blocks, 256, 0, stream>>>(reinterpret_cast<const __half *>(dO),
+    bwd_preprocess_kernel<D, kBf16><<<pre_blocks, 256, 0, stream>>>(reinterpret_cast<const __half *>(dO),
                                                              reinterpret_cast<const __half *>(O), LSE, delta_ext,
                                                              lse_ext, dq_acc, n_rows, S, S_pad, Hq, lay.d_o, lay.o, plain_pre,
                                                              1.f / scale, status);
@@ -984,13 +985,13 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
     prm.dk_st = lay.dk;
     prm.dv_st = lay.dv;
     const size_t smem = sizeof(BwdSmem<D>);
-    e = cudaFuncSetAttribute(bwd_main_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    e = cudaFuncSetAttribute(bwd_main_kernel<D, kBf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return record_cuda_error("cudaFuncSetAttribute(bwd_main)", e);
     const int n_items = B * Hkv * (S_pad / kTileRows);
     const int grid = n_items < sms ? n_items : sms;  // persistent: one CTA per SM walks the item list
     if (ev_main_begin && (e = cudaEventRecord(ev_main_begin, stream)) != cudaSuccess)
         return record_cuda_error("cudaEventRecord", e);
-    bwd_main_kernel<D><<<grid, kBwdThreads, smem, stream>>>(mq, mk, mv, mdo, prm);
+    bwd_main_kernel<D, kBf16><<<grid, kBwdThreads, smem, stream>>>(mq, mk, mv, mdo, prm);
     e = cudaGetLastError();
     if (e != cudaSuccess) return record_cuda_error("bwd_main_kernel launch", e);
     if (ev_main_end && (e = cudaEventRecord(ev_main_end, stream)) != cudaSuccess)
@@ -999,7 +1000,7 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
     const long long n_vec8 = static_cast<long long>(B) * Hq * S * D / 8;
     const long long fwant = (n_vec8 + 255) / 256;
     const int fin_blocks = static_cast<int>(fwant < static_cast<long long>(sms) * 16 ? fwant : sms * 16);
-    bwd_finalize_kernel<<<fin_blocks, 256, 0, stream>>>(dq_acc, reinterpret_cast<__half *>(dQ), n_vec8, S * (D / 8),
+    bwd_finalize_kernel<kBf16><<<fin_blocks, 256, 0, stream>>>(dq_acc, reinterpret_cast<__half *>(dQ), n_vec8, S * (D / 8),
                                                         S_pad * (D / 8), D / 8, Hq, lay.dq, plain_fin);
     e = cudaGetLastError();
     if (e != cudaSuccess) return record_cuda_error("bwd_finalize_kernel launch", e);
@@ -1021,7 +1022,7 @@ int lt_attn_bwd_num_launches(void) { return 3; }
 static int bwd_entry(const lt_half *Q, const lt_half *K, const lt_half *V, const lt_half *O, const lt_half *dO,
                      const float *LSE, lt_half *dQ, lt_half *dK, lt_half *dV, const lt_attn_layout *layout, int B,
                      int Hq, int Hkv, int S, int D, int causal, float scale, void *workspace, size_t workspace_bytes,
-                     lt_stream_t stream, lt_event_t main_begin, lt_event_t main_end) {
+                     lt_stream_t stream, lt_event_t main_begin, lt_event_t main_end, bool bf16 = false) {
     using namespace lt;
     if (!Q || !K || !V || !O || !dO || !LSE || !dQ || !dK || !dV) return LT_ERR_INVALID_ARG;
     int rc = check_shape(B, Hq, Hkv, S, D, scale);
@@ -1034,11 +1035,18 @@ static int bwd_entry(const lt_half *Q, const lt_half *K, const lt_half *V, const
     if (!workspace || !aligned256(workspace) || workspace_bytes < lt_attn_bwd_workspace_bytes(B, Hq, Hkv, S, D))
         return LT_ERR_WORKSPACE;
     if ((rc = check_device()) != LT_OK) return rc;
+    if (bf16) {
+        if (D == 64)
+            return launch_bwd<64, true>(Q, K, V, O, dO, LSE, dQ, dK, dV, lay, B, Hq, Hkv, S, causal, scale, workspace,
+                                        stream, main_begin, main_end);
+        return launch_bwd<128, true>(Q, K, V, O, dO, LSE, dQ, dK, dV, lay, B, Hq, Hkv, S, causal, scale, workspace,
+                                     stream, main_begin, main_end);
+    }
     if (D == 64)
-        return launch_bwd<64>(Q, K, V, O, dO, LSE, dQ, dK, dV, lay, B, Hq, Hkv, S, causal, scale, workspace, stream,
-                              main_begin, main_end);
-    return launch_bwd<128>(Q, K, V, O, dO, LSE, dQ, dK, dV, lay, B, Hq, Hkv, S, causal, scale, workspace, stream,
-                           main_begin, main_end);
+        return launch_bwd<64, false>(Q, K, V, O, dO, LSE, dQ, dK, dV, lay, B, Hq, Hkv, S, causal, scale, workspace,
+                                     stream, main_begin, main_end);
+    return launch_bwd<128, false>(Q, K, V, O, dO, LSE, dQ, dK, dV, lay, B, Hq, Hkv, S, causal, scale, workspace,
+                                  stream, main_begin, main_end);
 }
 
 int lt_attn_bwd_profiled(const lt_half *Q, const lt_half *K, const lt_half *V, const lt_half *O, const lt_half *dO,
@@ -1055,6 +1063,14 @@ int lt_attn_bwd_strided(const lt_half *Q, const lt_half *K, const lt_half *V, co
                         size_t workspace_bytes, lt_stream_t stream) {
     return bwd_entry(Q, K, V, O, dO, LSE, dQ, dK, dV, layout, B, Hq, Hkv, S, D, causal, scale, workspace,
                      workspace_bytes, stream, nullptr, nullptr);
+}
+
+int lt_attn_bwd_bf16(const lt_bf16 *Q, const lt_bf16 *K, const lt_bf16 *V, const lt_bf16 *O, const lt_bf16 *dO,
+                     const float *LSE, lt_bf16 *dQ, lt_bf16 *dK, lt_bf16 *dV, const lt_attn_layout *layout, int B,
+                     int Hq, int Hkv, int S, int D, int causal, float scale, void *workspace,
+                     size_t workspace_bytes, lt_stream_t stream) {
+    return bwd_entry(Q, K, V, O, dO, LSE, dQ, dK, dV, layout, B, Hq, Hkv, S, D, causal, scale, workspace,
+                     workspace_bytes, stream, nullptr, nullptr, true);
 }
 
 int lt_attn_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, const lt_half *O, const lt_half *dO,

@@ -68,7 +68,7 @@ __device__ unsigned long long g_fwd_trace[32];
 #endif
 
 // Registers are handed out per four warps, so ten warps get the 168-register cap of twelve.
-template <int D>
+template <int D, bool kBf16>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
            const __grid_constant__ CUtensorMap map_v, const FwdParams p) {
@@ -181,8 +181,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
             constexpr uint64_t kSlotStep = static_cast<uint64_t>(kTileBytes) >> 4;
             auto koff = [](int kk) -> uint64_t { return static_cast<uint64_t>((kk >> 2) * (kFwdBoxBytes >> 4) + (kk & 3) * 2); };
             auto roff = [](int kk) -> uint64_t { return static_cast<uint64_t>(kk * (2048 >> 4)); };
-            constexpr uint32_t idesc_s = make_idesc(128, 128, false, false);
-            constexpr uint32_t idesc_o = make_idesc(128, D, false, true);
+            constexpr uint32_t idesc_s = make_idesc(128, 128, false, false, kBf16);
+            constexpr uint32_t idesc_o = make_idesc(128, D, false, true, kBf16);
             auto issue_s = [&](int t, int s) {  // S_t = Q_t K^T with the key tile in ring slot s
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk)
@@ -359,7 +359,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
                     uint32_t out[16];
 #pragma unroll
                     for (int e = 0; e < 32; e += 2)
-                        out[e / 2] = pack_half2(__uint_as_float(sc[c * 32 + e]), __uint_as_float(sc[c * 32 + e + 1]));
+                        out[e / 2] = pack2<kBf16>(__uint_as_float(sc[c * 32 + e]), __uint_as_float(sc[c * 32 + e + 1]));
                     tmem_st16(tS + c * 16, out);
                 }
             };
@@ -399,10 +399,10 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
 #pragma unroll
                 for (int v8 = 0; v8 < 4; ++v8) {
                     uint4 o;
-                    o.x = pack_half2(__uint_as_float(r[8 * v8 + 0]) * inv_l, __uint_as_float(r[8 * v8 + 1]) * inv_l);
-                    o.y = pack_half2(__uint_as_float(r[8 * v8 + 2]) * inv_l, __uint_as_float(r[8 * v8 + 3]) * inv_l);
-                    o.z = pack_half2(__uint_as_float(r[8 * v8 + 4]) * inv_l, __uint_as_float(r[8 * v8 + 5]) * inv_l);
-                    o.w = pack_half2(__uint_as_float(r[8 * v8 + 6]) * inv_l, __uint_as_float(r[8 * v8 + 7]) * inv_l);
+                    o.x = pack2<kBf16>(__uint_as_float(r[8 * v8 + 0]) * inv_l, __uint_as_float(r[8 * v8 + 1]) * inv_l);
+                    o.y = pack2<kBf16>(__uint_as_float(r[8 * v8 + 2]) * inv_l, __uint_as_float(r[8 * v8 + 3]) * inv_l);
+                    o.z = pack2<kBf16>(__uint_as_float(r[8 * v8 + 4]) * inv_l, __uint_as_float(r[8 * v8 + 5]) * inv_l);
+                    o.w = pack2<kBf16>(__uint_as_float(r[8 * v8 + 6]) * inv_l, __uint_as_float(r[8 * v8 + 7]) * inv_l);
                     if (s_row < p.S) reinterpret_cast<uint4 *>(o_row + c * 32)[v8] = o;
                 }
             }
@@ -426,15 +426,15 @@ extern "C" int lt_dbg_fwd_trace(unsigned long long *out, int reset) {
 }
 #endif
 
-template <int D>
+template <int D, bool kBf16>
 static int launch_fwd(const lt_half *Q, const lt_half *K, const lt_half *V, lt_half *O, float *LSE,
                       const lt_attn_layout &lay, int B, int Hq, int Hkv, int S, int causal, float scale,
                       void *workspace, cudaStream_t stream) {
     CUtensorMap mq, mk, mv;
     int rc;
-    if ((rc = make_bhsd_map(&mq, Q, B, Hq, S, D, lay.q, 128)) != LT_OK) return rc;
-    if ((rc = make_bhsd_map(&mk, K, B, Hkv, S, D, lay.k, 128)) != LT_OK) return rc;
-    if ((rc = make_bhsd_map(&mv, V, B, Hkv, S, D, lay.v, 128)) != LT_OK) return rc;
+    if ((rc = make_bhsd_map(&mq, Q, B, Hq, S, D, lay.q, 128, kBf16)) != LT_OK) return rc;
+    if ((rc = make_bhsd_map(&mk, K, B, Hkv, S, D, lay.k, 128, kBf16)) != LT_OK) return rc;
+    if ((rc = make_bhsd_map(&mv, V, B, Hkv, S, D, lay.v, 128, kBf16)) != LT_OK) return rc;
     cudaError_t e = cudaMemsetAsync(workspace, 0, kStatusBytes, stream);
     if (e != cudaSuccess) return record_cuda_error("cudaMemsetAsync(status)", e);
     FwdParams prm;
@@ -446,11 +446,11 @@ static int launch_fwd(const lt_half *Q, const lt_half *K, const lt_half *V, lt_h
     prm.scale = scale;
     // at least 120 KB, so that one CTA (which takes all 512 tensor-memory columns) lives on an SM
     const size_t smem = std::max<size_t>(sizeof(FwdSmem<D>) + 1024, 120 * 1024);
-    e = cudaFuncSetAttribute(fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    e = cudaFuncSetAttribute(fwd_kernel<D, kBf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return record_cuda_error("cudaFuncSetAttribute(fwd)", e);
     const int n_tiles = (S + kFwdTileRows - 1) / kFwdTileRows;
     const int grid = B * Hq * ((n_tiles + 1) / 2);
-    fwd_kernel<D><<<grid, kFwdThreads, smem, stream>>>(mq, mk, mv, prm);
+    fwd_kernel<D, kBf16><<<grid, kFwdThreads, smem, stream>>>(mq, mk, mv, prm);
     e = cudaGetLastError();
     if (e != cudaSuccess) return record_cuda_error("fwd_kernel launch", e);
     return LT_OK;
@@ -473,9 +473,9 @@ int lt_attn_fwd(const lt_half *Q, const lt_half *K, const lt_half *V, lt_half *O
                                stream);
 }
 
-int lt_attn_fwd_strided(const lt_half *Q, const lt_half *K, const lt_half *V, lt_half *O, float *LSE,
-                        const lt_attn_layout *layout, int B, int Hq, int Hkv, int S, int D, int causal, float scale,
-                        void *workspace, size_t workspace_bytes, lt_stream_t stream) {
+static int fwd_entry(const lt_half *Q, const lt_half *K, const lt_half *V, lt_half *O, float *LSE,
+                     const lt_attn_layout *layout, int B, int Hq, int Hkv, int S, int D, int causal, float scale,
+                     void *workspace, size_t workspace_bytes, lt_stream_t stream, bool bf16) {
     using namespace lt;
     if (!Q || !K || !V || !O || !LSE) return LT_ERR_INVALID_ARG;
     int rc = check_shape(B, Hq, Hkv, S, D, scale);
@@ -492,8 +492,26 @@ int lt_attn_fwd_strided(const lt_half *Q, const lt_half *K, const lt_half *V, lt
     if (!workspace || !aligned256(workspace) || workspace_bytes < lt_attn_fwd_workspace_bytes(B, Hq, Hkv, S, D))
         return LT_ERR_WORKSPACE;
     if ((rc = check_device()) != LT_OK) return rc;
-    if (D == 64) return launch_fwd<64>(Q, K, V, O, LSE, lay, B, Hq, Hkv, S, causal, scale, workspace, stream);
-    return launch_fwd<128>(Q, K, V, O, LSE, lay, B, Hq, Hkv, S, causal, scale, workspace, stream);
+    if (bf16) {
+        if (D == 64) return launch_fwd<64, true>(Q, K, V, O, LSE, lay, B, Hq, Hkv, S, causal, scale, workspace, stream);
+        return launch_fwd<128, true>(Q, K, V, O, LSE, lay, B, Hq, Hkv, S, causal, scale, workspace, stream);
+    }
+    if (D == 64) return launch_fwd<64, false>(Q, K, V, O, LSE, lay, B, Hq, Hkv, S, causal, scale, workspace, stream);
+    return launch_fwd<128, false>(Q, K, V, O, LSE, lay, B, Hq, Hkv, S, causal, scale, workspace, stream);
+}
+
+int lt_attn_fwd_strided(const lt_half *Q, const lt_half *K, const lt_half *V, lt_half *O, float *LSE,
+                        const lt_attn_layout *layout, int B, int Hq, int Hkv, int S, int D, int causal, float scale,
+                        void *workspace, size_t workspace_bytes, lt_stream_t stream) {
+    return fwd_entry(Q, K, V, O, LSE, layout, B, Hq, Hkv, S, D, causal, scale, workspace, workspace_bytes, stream,
+                     false);
+}
+
+int lt_attn_fwd_bf16(const lt_bf16 *Q, const lt_bf16 *K, const lt_bf16 *V, lt_bf16 *O, float *LSE,
+                     const lt_attn_layout *layout, int B, int Hq, int Hkv, int S, int D, int causal, float scale,
+                     void *workspace, size_t workspace_bytes, lt_stream_t stream) {
+    return fwd_entry(Q, K, V, O, LSE, layout, B, Hq, Hkv, S, D, causal, scale, workspace, workspace_bytes, stream,
+                     true);
 }
 
 size_t lt_attn_host_arena_bytes(int B, int Hq, int Hkv, int S, int D) {

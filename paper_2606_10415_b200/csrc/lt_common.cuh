@@ -4,6 +4,7 @@
 #pragma once
 
 #include <cuda.h>
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -224,19 +225,55 @@ __device__ __forceinline__ uint64_t desc_kmajor_noswz(uint32_t smem_addr, uint32
            (static_cast<uint64_t>((sbo >> 4) & 0x3FFF) << 32) | static_cast<uint64_t>((smem_addr & 0x3FFFF) >> 4);
 }
 
-// x = 256 * hi + lo with both parts fp16: about 22 significant bits and a range of 1.6e7.
-// Used to add a per-row fp32 value inside a tensor-core product: one extra contraction step
-// whose other operand holds (256, 1, 0, ..., 0).
-__device__ __forceinline__ uint32_t split_hi_lo(float x) {
-    const __half hi = __float2half_rn(x * (1.f / 256.f));
-    const __half lo = __float2half_rn(x - 256.f * __half2float(hi));
-    return static_cast<uint32_t>(__half_as_ushort(hi)) | (static_cast<uint32_t>(__half_as_ushort(lo)) << 16);
+// Two fp32 values rounded to a pair of 16-bit floats (fp16, or bf16 when kBf16), first value in
+// the low half, and back.
+template <bool kBf16>
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+    if constexpr (kBf16) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+        return *reinterpret_cast<uint32_t *>(&h);
+    } else {
+        __half2 h = __floats2half2_rn(lo, hi);
+        return *reinterpret_cast<uint32_t *>(&h);
+    }
+}
+template <bool kBf16>
+__device__ __forceinline__ float2 unpack2(uint32_t w) {
+    if constexpr (kBf16) return __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&w));
+    else return __half22float2(*reinterpret_cast<const __half2 *>(&w));
 }
 
-// Instruction descriptor, kind::f16: fp16 A and B, fp32 accumulator, dense.
-constexpr uint32_t make_idesc(int M, int N, bool a_mn_major, bool b_mn_major) {
+// A per-row fp32 value x is added inside a tensor-core product by one extra contraction step whose
+// other operand holds the multipliers kExtMult = (256, 1, 1/256, 0, ...).  The row stored for x holds
+// 16-bit floats (hi, mid, lo, 0, ...) with 256*hi + mid + lo/256 = x: two terms for fp16 (about 22
+// significant bits, lo = 0), three for bf16 (24 bits).  Returned as the 16-byte row.
+template <bool kBf16>
+__device__ __forceinline__ uint4 split_ext(float x) {
+    if constexpr (kBf16) {
+        const __nv_bfloat16 hi = __float2bfloat16_rn(x * (1.f / 256.f));
+        const float r1 = x - 256.f * __bfloat162float(hi);
+        const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+        const __nv_bfloat16 lo = __float2bfloat16_rn((r1 - __bfloat162float(mid)) * 256.f);
+        return make_uint4(static_cast<uint32_t>(__bfloat16_as_ushort(hi)) |
+                              (static_cast<uint32_t>(__bfloat16_as_ushort(mid)) << 16),
+                          static_cast<uint32_t>(__bfloat16_as_ushort(lo)), 0u, 0u);
+    } else {
+        const __half hi = __float2half_rn(x * (1.f / 256.f));
+        const __half mid = __float2half_rn(x - 256.f * __half2float(hi));
+        return make_uint4(static_cast<uint32_t>(__half_as_ushort(hi)) | (static_cast<uint32_t>(__half_as_ushort(mid)) << 16),
+                          0u, 0u, 0u);
+    }
+}
+// the first two words of the multiplier row (256, 1 | 1/256, 0)
+template <bool kBf16>
+__device__ __forceinline__ uint2 ext_multipliers() {
+    return make_uint2(pack2<kBf16>(256.f, 1.f), pack2<kBf16>(1.f / 256.f, 0.f));
+}
+
+// Instruction descriptor, kind::f16: fp16 (or bf16) A and B, fp32 accumulator, dense.
+constexpr uint32_t make_idesc(int M, int N, bool a_mn_major, bool b_mn_major, bool bf16 = false) {
     return (1u << 4)                                   // accumulator format: f32
-           | (0u << 7) | (0u << 10)                    // A, B format: f16
+           | ((bf16 ? 1u : 0u) << 7) | ((bf16 ? 1u : 0u) << 10)   // A, B format: f16 = 0, bf16 = 1
            | (static_cast<uint32_t>(a_mn_major) << 15) | (static_cast<uint32_t>(b_mn_major) << 16) |
            (static_cast<uint32_t>(N >> 3) << 17) | (static_cast<uint32_t>(M >> 4) << 24);
 }
@@ -350,10 +387,7 @@ __device__ __forceinline__ void red_add_v4(float *addr, float a, float b, float 
     asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d)
                  : "memory");
 }
-__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
-    __half2 h = __floats2half2_rn(lo, hi);  // .x = lo (low 16 bits), .y = hi
-    return *reinterpret_cast<uint32_t *>(&h);
-}
+__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) { return pack2<false>(lo, hi); }
 
 // Byte offset of element (row, col) inside one swizzled tile of 64 fp16 columns
 // (rows of 128 bytes, 16-byte chunks XORed with row % 8), the layout TMA's 128B swizzle

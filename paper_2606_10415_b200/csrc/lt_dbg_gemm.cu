@@ -76,7 +76,7 @@ dbg_tile_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         const float x = 1000.f * __half2float(reinterpret_cast<const __half *>(b_gmem)[static_cast<size_t>(tid) * kTile]);
         const __half2 ones = __halves2half2(__float2half_rn(256.f), __float2half_rn(1.f));
         reinterpret_cast<uint4 *>(sm.ext_a)[tid] = make_uint4(*reinterpret_cast<const uint32_t *>(&ones), 0u, 0u, 0u);
-        reinterpret_cast<uint4 *>(sm.ext_b)[tid] = make_uint4(split_hi_lo(x), 0u, 0u, 0u);
+        reinterpret_cast<uint4 *>(sm.ext_b)[tid] = split_ext<false>(x);
         reinterpret_cast<uint4 *>(sm.ext_zero)[tid] = make_uint4(0u, 0u, 0u, 0u);
         fence_proxy_async_smem();
     }

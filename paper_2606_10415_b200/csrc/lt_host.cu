@@ -81,7 +81,7 @@ int make_tile_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t co
 }
 
 int make_bhsd_map(CUtensorMap *map, const void *base, uint64_t B, uint64_t H, uint64_t S, uint64_t D,
-                  const lt_tensor_strides &st, uint32_t box_rows) {
+                  const lt_tensor_strides &st, uint32_t box_rows, bool bf16) {
     EncodeTiledFn enc = get_encoder();
     if (!enc) return LT_ERR_CUDA;
     cuuint64_t dims[4] = {D, S, H, B};
@@ -90,7 +90,8 @@ int make_bhsd_map(CUtensorMap *map, const void *base, uint64_t B, uint64_t H, ui
                              static_cast<cuuint64_t>(st.batch) * sizeof(__half)};
     cuuint32_t box[4] = {64u, box_rows, 1u, 1u};
     cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
-    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
+    CUresult r = enc(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4,
+                     const_cast<void *>(base), dims, strides, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {

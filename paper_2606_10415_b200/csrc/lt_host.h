@@ -29,10 +29,10 @@ inline size_t round256(size_t n) { return (n + 255u) & ~static_cast<size_t>(255u
 // fp16 matrix [rows, cols] row-major viewed as a 2-D tensor; tiles of box_rows x 64
 // columns are fetched with the 128-byte swizzle.  Returns LT_OK or LT_ERR_CUDA.
 int make_tile_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows);
-// 4-D view [batch][head][row][element] of an fp16 tensor with the given element strides (boxes of
+// 4-D view [batch][head][row][element] of an fp16 (or bf16) tensor with the given element strides (boxes of
 // 64 elements x box_rows rows of one head, 128-byte swizzle, zero fill past the last row).
 int make_bhsd_map(CUtensorMap *map, const void *base, uint64_t B, uint64_t H, uint64_t S, uint64_t D,
-                  const lt_tensor_strides &st, uint32_t box_rows);
+                  const lt_tensor_strides &st, uint32_t box_rows, bool bf16 = false);
 // strides of a contiguous [B,H,S,D] tensor
 inline lt_tensor_strides contiguous_strides(int H, int S, int D) {
     lt_tensor_strides st;

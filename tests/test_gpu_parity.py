@@ -348,6 +348,44 @@ def test_fused_qkv_buffer_matches_oracle(lt, oracle):
     assert torch.all(views.grad[..., width:] == 7.0)
 
 
+# ------------------------------------------------------------------ bfloat16
+
+# bf16 keeps 8 significant bits: outputs, P and dS each carry about 2^-9 relative rounding
+BF16_REL_FRO_TOL = 5e-3
+BF16_FWD_O_REL_FRO_TOL = 4e-3
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,S,D,causal", [
+    (1, 2, 2, 128, 64, True), (2, 4, 2, 384, 128, True), (1, 6, 2, 333, 128, True), (1, 2, 1, 256, 64, False),
+    (1, 8, 2, 1024, 128, True),
+])
+def test_bf16_matches_oracle(lt, oracle, B, Hq, Hkv, S, D, causal):
+    """bfloat16 inputs and outputs; the oracle works in fp64 on the bf16-rounded inputs."""
+    cfg = workloads.custom(B, Hq, Hkv, S, D, causal, seed=41 + S)
+    Q, K, V, dO = (t.float().bfloat16() for t in workloads.make_inputs(cfg))
+    Qd, Kd, Vd, dOd = (t.cuda() for t in (Q, K, V, dO))
+    O = torch.empty_like(Qd)
+    LSE = torch.empty(Q.shape[:3], dtype=torch.float32, device="cuda")
+    fws = lt.alloc_workspace(lt.lt_attn_fwd_workspace_bytes(B, Hq, Hkv, S, D))
+    lt.lt_attn_fwd_bf16(Qd, Kd, Vd, O, LSE, causal, cfg.scale, fws)
+    assert lt.lt_attn_check_status(fws) == lt.LT_OK, lt.last_cuda_error()
+    Qn, Kn, Vn, dOn = (t.double().numpy() for t in (Q, K, V, dO))
+    O_ref, LSE_ref = oracle.attn_fwd(Qn, Kn, Vn, causal, cfg.scale)
+    assert rel_fro(O.cpu().double().numpy(), O_ref) <= BF16_FWD_O_REL_FRO_TOL
+    assert max_abs(LSE.cpu().double().numpy(), LSE_ref) <= FWD_LSE_ABS_TOL
+    dQ, dK, dV = (torch.full_like(t, float("nan")) for t in (Qd, Kd, Vd))
+    ws = lt.alloc_workspace(lt.lt_attn_bwd_workspace_bytes(B, Hq, Hkv, S, D))
+    ws.fill_(0xFF)
+    lt.lt_attn_bwd_bf16(Qd, Kd, Vd, O, dOd, LSE, dQ, dK, dV, causal, cfg.scale, ws)
+    assert lt.lt_attn_check_status(ws) == lt.LT_OK, lt.last_cuda_error()
+    ref = oracle.attn_bwd(Qn, Kn, Vn, dOn, causal, cfg.scale)
+    for name, g, r in zip(("dQ", "dK", "dV"), (dQ, dK, dV), ref):
+        g = g.cpu().double().numpy()
+        assert np.all(np.isfinite(g)), name
+        assert rel_fro(g, r) <= BF16_REL_FRO_TOL, f"bf16 {name}: {rel_fro(g, r):.3e}"
+        assert max_abs(g, r) <= MAX_ABS_TOL, f"bf16 {name}: max abs {max_abs(g, r):.3e}"
+
+
 # ------------------------------------------------------------------ benchmark configurations, full size
 
 def _full_size_check(lt, oracle, name, units):
