@@ -125,3 +125,15 @@ def delta(dO, O):
     if rc != 0:
         raise RuntimeError(f"lt_oracle_delta_f64 failed with code {rc}")
     return out
+
+
+def gemm_nt(A, W):
+    """C = A W^T in float64: A is [M, K] (activations), W is [N, K] (the weight matrix of a linear
+    layer as it is stored), C is [M, N].  This is the product the paper's FP16 GEMM backend computes
+    for the QKV, output and FFN projections (Section 4.1: C[M,N] accumulates A[M,K] B[K,N]; here
+    B = W^T) and profiles in its table of GEMM shapes (Section 6.6).  numpy's matmul is the library
+    step; nothing is blocked or reordered here."""
+    A, W = _f64(A), _f64(W)
+    if A.ndim != 2 or W.ndim != 2 or A.shape[1] != W.shape[1]:
+        raise ValueError("expected A [M, K] and W [N, K]")
+    return A @ W.T

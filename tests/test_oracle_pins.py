@@ -361,3 +361,37 @@ def test_thread_count_does_not_change_results(oracle):
         outs.add(subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True,
                                 check=True).stdout.strip())
     assert len(outs) == 1
+
+
+# ------------------------------------------------------------------ GEMM oracle (C = A W^T)
+
+def test_gemm_oracle_hand_worked_example(oracle):
+    lines = [ln for ln in (Path(__file__).parent / "golden" / "gemm_worked_example.txt").read_text().splitlines()
+             if ln and not ln.startswith("#")]
+    rows = [list(map(float, ln.split())) for ln in lines]
+    A, W, C = np.array(rows[0:2]), np.array(rows[2:4]), np.array(rows[4:6])
+    assert np.array_equal(oracle.gemm_nt(A, W), C)
+
+
+def test_gemm_oracle_against_triple_loop_and_special_cases(oracle):
+    rng = np.random.default_rng(3)
+    M, N, K = 5, 7, 11
+    A, W = rng.standard_normal((M, K)), rng.standard_normal((N, K))
+    brute = np.zeros((M, N))
+    for m in range(M):
+        for n in range(N):
+            for k in range(K):
+                brute[m, n] += A[m, k] * W[n, k]
+    np.testing.assert_allclose(oracle.gemm_nt(A, W), brute, rtol=1e-13, atol=1e-13)
+    # identity weight returns A; a weight row that selects one input column returns that column
+    assert np.array_equal(oracle.gemm_nt(A, np.eye(K)), A)
+    sel = np.zeros((1, K)); sel[0, 4] = 1.0
+    assert np.array_equal(oracle.gemm_nt(A, sel)[:, 0], A[:, 4])
+    # not symmetric in its arguments (a swapped or untransposed operand changes the shape or the values)
+    assert oracle.gemm_nt(A, W).shape == (M, N) and oracle.gemm_nt(W, A).shape == (N, M)
+    np.testing.assert_allclose(oracle.gemm_nt(W, A), oracle.gemm_nt(A, W).T, rtol=1e-13)
+    # linear in each argument
+    A2 = rng.standard_normal((M, K))
+    np.testing.assert_allclose(oracle.gemm_nt(A + 2 * A2, W), oracle.gemm_nt(A, W) + 2 * oracle.gemm_nt(A2, W), rtol=1e-12)
+    with pytest.raises(ValueError):
+        oracle.gemm_nt(A, rng.standard_normal((N, K + 1)))
