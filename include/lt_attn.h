@@ -167,6 +167,18 @@ int lt_attn_bwd_bf16(const lt_bf16 *Q, const lt_bf16 *K, const lt_bf16 *V,
                      int B, int Hq, int Hkv, int S, int D, int causal, float scale,
                      void *workspace, size_t workspace_bytes, lt_stream_t stream);
 
+/* FP16 GEMM, the linear-layer primitive of the paper's backend (Section 4.1, "FP16 GEMM assembly
+ * pipeline"; its profiled shapes are in Section 6.6):  C[M,N] = A[M,K] W[N,K]^T.
+ *   in : A [M,K] fp16 row-major (activations), W [N,K] fp16 row-major (a linear layer's weight as stored)
+ *   out: C [M,N] fp16 row-major, fully overwritten; products accumulate in fp32
+ * Any M, N >= 1; K >= 8 and a multiple of 8 (16-byte row pitch for the tile loads); otherwise
+ * LT_ERR_UNSUPPORTED.  Device pointers, 16-byte aligned, owned by the caller.  `workspace` holds only
+ * the 256-byte status block (lt_gemm_f16_workspace_bytes()); read it with lt_attn_check_status.
+ * Enqueues one kernel on `stream`; allocates nothing; does not synchronise. */
+size_t lt_gemm_f16_workspace_bytes(void);
+int lt_gemm_f16(const lt_half *A, const lt_half *W, lt_half *C, int M, int N, int K,
+                void *workspace, size_t workspace_bytes, lt_stream_t stream);
+
 /* Same computation as lt_attn_fwd followed by lt_attn_bwd, but every tensor pointer is
  * a HOST pointer (pinned memory makes the copies asynchronous).  `arena` is a caller-
  * owned DEVICE buffer of at least lt_attn_host_arena_bytes() bytes, 256-byte aligned,

@@ -1,0 +1,243 @@
+// FP16 GEMM for sm_100a: C[M,N] = A[M,K] W[N,K]^T, fp16 operands, fp32 accumulation, fp16 result.
+// This is the linear-layer primitive of the paper's backend (Section 4.1, "FP16 GEMM assembly
+// pipeline"; shapes profiled in Section 6.6).  The MT-3000 dataflow of the paper (A staged through
+// GSM/SM, B broadcast to AM, C accumulated in AM) maps here to: A and W tiles staged in shared memory
+// by TMA, C accumulated in tensor memory, one CTA per SM walking the output tiles.
+//
+//   warp 0      : TMA producer - 64-wide contraction blocks of a 128-row A tile and a 256-row W
+//                 tile through a four-slot ring
+//   warp 1      : tcgen05 issuer - four 128x256x16 products per block into one of two 256-column
+//                 accumulators
+//   warps 2..5  : epilogue - tensor memory -> fp16 -> global, one accumulator while the other is
+//                 being filled
+#include "lt_common.cuh"
+#include "lt_host.h"
+
+namespace lt {
+
+constexpr int kGemmBM = 128, kGemmBN = 256, kGemmBK = 64, kGemmStages = 4;
+constexpr int kGemmThreads = 192;
+constexpr uint32_t kGemmABytes = kGemmBM * kGemmBK * 2;   // 16 KB
+constexpr uint32_t kGemmBBytes = kGemmBN * kGemmBK * 2;   // 32 KB
+
+enum { kWaitGemmFull = 401, kWaitGemmEmpty = 402, kWaitGemmAccFull = 403, kWaitGemmAccEmpty = 404 };
+
+struct __align__(1024) GemmSmem {
+    uint8_t a[kGemmStages][kGemmABytes];
+    uint8_t b[kGemmStages][kGemmBBytes];
+    uint64_t bar_full[kGemmStages], bar_empty[kGemmStages], bar_acc_full[2], bar_acc_empty[2];
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+struct GemmParams {
+    __half *C;
+    unsigned int *status;
+    int M, N, K;
+    int tiles_m, tiles_n;
+};
+
+// Output tiles are numbered so that consecutive numbers share the W tile (the larger operand tile)
+// and a wave of CTAs covers a compact block of C: tile -> (m, n) with m fastest inside groups of
+// eight tile rows.
+__device__ __forceinline__ void gemm_tile_coords(const GemmParams &p, int tile, int &tm, int &tn) {
+    constexpr int kGroup = 8;
+    const int per_group = kGroup * p.tiles_n;
+    const int g = tile / per_group;
+    const int first_m = g * kGroup;
+    const int rows = min(kGroup, p.tiles_m - first_m);
+    const int r = tile - g * per_group;
+    tm = first_m + r % rows;
+    tn = r / rows;
+}
+
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+            const GemmParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    GemmSmem &sm = *reinterpret_cast<GemmSmem *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+    const int n_tiles = p.tiles_m * p.tiles_n;
+    const int k_blocks = (p.K + kGemmBK - 1) / kGemmBK;  // a ragged last block reads zeros past K
+
+    if (tid == 0) {
+        sm.abort_flag = 0;
+        for (int s = 0; s < kGemmStages; ++s) {
+            mbar_init(&sm.bar_full[s], 1);
+            mbar_init(&sm.bar_empty[s], 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&sm.bar_acc_full[a], 1);
+            mbar_init(&sm.bar_acc_empty[a], 4);  // lane 0 of each epilogue warp
+        }
+        mbar_fence_init();
+        tma_prefetch_desc(&map_a);
+        tma_prefetch_desc(&map_b);
+    }
+    if (warp == 0) {
+        tmem_alloc(&sm.tmem_base, 512);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = sm.tmem_base;
+    volatile int *abort_flag = &sm.abort_flag;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            bool ok = true;
+            int kb_total = 0;  // contraction blocks loaded so far, over all tiles
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+                int tm, tn;
+                gemm_tile_coords(p, tile, tm, tn);
+                for (int kb = 0; kb < k_blocks; ++kb, ++kb_total) {
+                    const int s = kb_total % kGemmStages;
+                    const uint32_t use = kb_total / kGemmStages;
+                    if (use >= 1 && !(ok = mbar_wait(&sm.bar_empty[s], (use - 1) & 1, abort_flag, p.status, kWaitGemmEmpty)))
+                        break;
+                    mbar_arrive_expect_tx(&sm.bar_full[s], kGemmABytes + kGemmBBytes);
+                    tma_load_2d(sm.a[s], &map_a, &sm.bar_full[s], kb * kGemmBK, tm * kGemmBM);
+                    tma_load_2d(sm.b[s], &map_b, &sm.bar_full[s], kb * kGemmBK, tn * kGemmBN);
+                }
+            }
+            if (!ok || *abort_flag) {
+                // somebody gave up: wait (bounded) for the copies in flight before the CTA exits
+                for (int back = 0; back < kGemmStages && back < kb_total; ++back) {
+                    const int q = kb_total - 1 - back;
+                    for (int w = 0; w < (1 << 16) && !mbar_try_wait(&sm.bar_full[q % kGemmStages], (q / kGemmStages) & 1); ++w) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(kGemmBM, kGemmBN, false, false);
+            bool ok = true;
+            int kb_total = 0, t_local = 0;
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++t_local) {
+                const int acc = t_local & 1;
+                const uint32_t acc_use = t_local >> 1;
+                // the epilogue must have read this accumulator's previous tile
+                if (acc_use >= 1 && !(ok = mbar_wait(&sm.bar_acc_empty[acc], (acc_use - 1) & 1, abort_flag, p.status, kWaitGemmAccEmpty)))
+                    break;
+                tc_fence_after_sync();
+                for (int kb = 0; kb < k_blocks; ++kb, ++kb_total) {
+                    const int s = kb_total % kGemmStages;
+                    if (!(ok = mbar_wait(&sm.bar_full[s], (kb_total / kGemmStages) & 1, abort_flag, p.status, kWaitGemmFull))) break;
+                    tc_fence_after_sync();
+                    const uint64_t da = desc_kmajor(smem_u32(sm.a[s])), db = desc_kmajor(smem_u32(sm.b[s]));
+#pragma unroll
+                    for (int kk = 0; kk < kGemmBK / 16; ++kk)
+                        umma_ss(tmem + acc * kGemmBN, da + kk * 2, db + kk * 2, idesc, (kb > 0) | (kk > 0));
+                    umma_commit(&sm.bar_empty[s]);  // the slot is free once these products have read it
+                }
+                if (!ok) break;
+                umma_commit(&sm.bar_acc_full[acc]);
+            }
+        }
+    } else {
+        // epilogue: thread = row of the tile, 32 columns at a time
+        const int quad = warp & 3;  // tensor-memory lane quadrant this warp may read
+        const int row = quad * 32 + lane;
+        const uint32_t lane_base = static_cast<uint32_t>(quad * 32) << 16;
+        bool ok = true;
+        int t_local = 0;
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++t_local) {
+            const int acc = t_local & 1;
+            ok = mbar_wait(&sm.bar_acc_full[acc], (t_local >> 1) & 1, abort_flag, p.status, kWaitGemmAccFull);
+            if (!(ok = __all_sync(0xffffffffu, ok))) break;
+            tc_fence_after_sync();
+            int tm, tn;
+            gemm_tile_coords(p, tile, tm, tn);
+            const long long m = static_cast<long long>(tm) * kGemmBM + row;
+            const int n0 = tn * kGemmBN;
+            __half *c_row = p.C + m * p.N + n0;
+            const bool vec_ok = (p.N % 8) == 0;  // 16-byte stores need the row pitch to allow them
+#pragma unroll
+            for (int c = 0; c < kGemmBN / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld32(tmem + lane_base + acc * kGemmBN + c * 32, r);
+                tmem_wait_ld();
+                if (c == kGemmBN / 32 - 1) {
+                    // the whole accumulator is in registers or stored: the issuer may reuse it
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm.bar_acc_empty[acc]);
+                }
+                if (m < p.M) {
+                    const int nc = n0 + c * 32;
+                    if (vec_ok && nc + 32 <= p.N) {
+#pragma unroll
+                        for (int v8 = 0; v8 < 4; ++v8) {
+                            uint4 o;
+                            o.x = pack_half2(__uint_as_float(r[8 * v8 + 0]), __uint_as_float(r[8 * v8 + 1]));
+                            o.y = pack_half2(__uint_as_float(r[8 * v8 + 2]), __uint_as_float(r[8 * v8 + 3]));
+                            o.z = pack_half2(__uint_as_float(r[8 * v8 + 4]), __uint_as_float(r[8 * v8 + 5]));
+                            o.w = pack_half2(__uint_as_float(r[8 * v8 + 6]), __uint_as_float(r[8 * v8 + 7]));
+                            reinterpret_cast<uint4 *>(c_row + c * 32)[v8] = o;
+                        }
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            if (nc + e < p.N) c_row[c * 32 + e] = __float2half_rn(__uint_as_float(r[e]));
+                    }
+                }
+            }
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 512);
+}
+
+}  // namespace lt
+
+extern "C" {
+
+size_t lt_gemm_f16_workspace_bytes(void) { return lt::kStatusBytes; }
+
+int lt_gemm_f16(const lt_half *A, const lt_half *W, lt_half *C, int M, int N, int K, void *workspace,
+                size_t workspace_bytes, lt_stream_t stream) {
+    using namespace lt;
+    if (!A || !W || !C) return LT_ERR_INVALID_ARG;
+    if (M <= 0 || N <= 0 || K <= 0) return LT_ERR_INVALID_ARG;
+    // TMA needs 16-byte row pitches for the operands
+    if ((K % 8) != 0) return LT_ERR_UNSUPPORTED;
+    if (!aligned16(A) || !aligned16(W) || !aligned16(C)) return LT_ERR_UNSUPPORTED;
+    if (!workspace || !aligned256(workspace) || workspace_bytes < kStatusBytes) return LT_ERR_WORKSPACE;
+    int rc = check_device();
+    if (rc != LT_OK) return rc;
+
+    CUtensorMap ma, mb;
+    if ((rc = make_tile_map(&ma, A, M, K, kGemmBM)) != LT_OK) return rc;
+    if ((rc = make_tile_map(&mb, W, N, K, kGemmBN)) != LT_OK) return rc;
+    cudaError_t e = cudaMemsetAsync(workspace, 0, kStatusBytes, stream);
+    if (e != cudaSuccess) return record_cuda_error("cudaMemsetAsync(status)", e);
+
+    GemmParams prm;
+    prm.C = reinterpret_cast<__half *>(C);
+    prm.status = reinterpret_cast<unsigned int *>(workspace);
+    prm.M = M; prm.N = N; prm.K = K;
+    prm.tiles_m = (M + kGemmBM - 1) / kGemmBM;
+    prm.tiles_n = (N + kGemmBN - 1) / kGemmBN;
+    const size_t smem = sizeof(GemmSmem) + 1024;
+    e = cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return record_cuda_error("cudaFuncSetAttribute(gemm)", e);
+    int sms = 148;
+    {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    }
+    const long long n_tiles = static_cast<long long>(prm.tiles_m) * prm.tiles_n;
+    const int grid = static_cast<int>(n_tiles < sms ? n_tiles : sms);
+    gemm_kernel<<<grid, kGemmThreads, smem, stream>>>(ma, mb, prm);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return record_cuda_error("gemm_kernel launch", e);
+    return LT_OK;
+}
+
+}  // extern "C"

@@ -132,3 +132,20 @@ def test_strided_entry_points_reject_bad_strides(binding):
     assert fwd(layout(o=(2 * 128 * 64, 128 * 64, -64))) == b.LT_ERR_UNSUPPORTED
     # the forward ignores the gradient entries: it gets as far as the workspace check (nothing is launched)
     assert fwd(layout(dq=(1, 1, 1)), ws_bytes=16) == b.LT_ERR_WORKSPACE
+
+
+def test_gemm_rejects_bad_arguments_without_launching(binding):
+    b = binding
+    lib = b._lib
+
+    def call(A=0x1000, W=0x2000, C=0x3000, M=128, N=256, K=64, ws=0x10000, ws_bytes=256):
+        return lib.lt_gemm_f16(A, W, C, M, N, K, ws, ws_bytes, 0)
+
+    assert b.lt_gemm_f16_workspace_bytes() == 256
+    assert call(A=0) == b.LT_ERR_INVALID_ARG
+    assert call(M=0) == b.LT_ERR_INVALID_ARG
+    assert call(K=-8) == b.LT_ERR_INVALID_ARG
+    assert call(K=12) == b.LT_ERR_UNSUPPORTED        # row pitch of 24 bytes: no 16-byte tile loads
+    assert call(W=0x2002) == b.LT_ERR_UNSUPPORTED    # misaligned
+    assert call(ws=0) == b.LT_ERR_WORKSPACE
+    assert call(ws_bytes=16) == b.LT_ERR_WORKSPACE

@@ -1,0 +1,81 @@
+"""Parity of the FP16 GEMM (C = A W^T) against the fp64 oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+# fp16 output rounding (2^-11 per element) dominates; fp32 accumulation adds far less
+GEMM_REL_FRO_TOL = 1e-3
+
+
+@pytest.fixture(scope="module")
+def lt():
+    from paper_2606_10415_b200 import binding
+    return binding
+
+
+def rel_fro(a, b):
+    return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
+
+
+def make_operands(M, N, K, seed):
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(seed)
+    A = torch.randn((M, K), generator=gen, dtype=torch.float32).half()
+    W = (torch.randn((N, K), generator=gen, dtype=torch.float32) * K ** -0.5).half()
+    return A, W
+
+
+def run_gemm(lt, A, W):
+    Ad, Wd = A.cuda(), W.cuda()
+    C = torch.full((A.shape[0], W.shape[0]), float("nan"), dtype=torch.float16, device="cuda")
+    ws = lt.alloc_workspace(lt.lt_gemm_f16_workspace_bytes())
+    lt.lt_gemm_f16(Ad, Wd, C, ws)
+    assert lt.lt_attn_check_status(ws) == lt.LT_OK, lt.last_cuda_error()
+    return C.cpu()
+
+
+@pytest.mark.parametrize("M,N,K", [
+    (128, 256, 64), (128, 256, 256), (256, 512, 512),            # whole tiles
+    (1, 8, 8), (100, 200, 72), (129, 257, 136), (300, 1000, 520),  # ragged in every dimension
+    (384, 250, 64), (77, 36, 1024),                                # N not a multiple of 8: scalar stores
+    (2048, 1024, 768),                                             # more tiles than SMs would need twice
+])
+def test_gemm_matches_oracle(lt, oracle, M, N, K):
+    A, W = make_operands(M, N, K, seed=M + N + K)
+    C = run_gemm(lt, A, W)
+    ref = oracle.gemm_nt(A.double().numpy(), W.double().numpy())
+    got = C.double().numpy()
+    assert np.all(np.isfinite(got))
+    assert rel_fro(got, ref) <= GEMM_REL_FRO_TOL, f"{(M, N, K)}: {rel_fro(got, ref):.3e}"
+    # element-wise: within fp16 rounding of the exact value plus accumulation slack
+    assert np.max(np.abs(got - ref) - 2.0 ** -10 * np.abs(ref)) <= 1e-3
+
+
+def test_gemm_integer_operands_are_exact(lt, oracle):
+    """Small integers: every product and partial sum is exact in fp32 and fp16, so the result must
+    equal the oracle bit for bit."""
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(1)
+    A = torch.randint(-3, 4, (200, 136), generator=gen).half()
+    W = torch.randint(-2, 3, (300, 136), generator=gen).half()
+    C = run_gemm(lt, A, W)
+    ref = oracle.gemm_nt(A.double().numpy(), W.double().numpy())
+    assert np.array_equal(C.double().numpy(), ref)
+
+
+@pytest.mark.parametrize("N,K", [(4096, 4096), (11008, 4096), (4096, 11008), (6656, 6656), (8192, 8192)])
+def test_gemm_paper_shapes_sampled_rows(lt, oracle, N, K):
+    """The five weight shapes of the paper's GEMM profile (Section 6.6) at its sequence length of 2048
+    rows; the launch the benchmark times, compared on sampled rows and columns."""
+    M = 2048
+    A, W = make_operands(M, N, K, seed=N + K)
+    C = run_gemm(lt, A, W)
+    assert torch.isfinite(C.float()).all()
+    rows = [0, 1, 127, 128, 1000, 2047]
+    ref = oracle.gemm_nt(A[rows].double().numpy(), W.double().numpy())
+    assert rel_fro(C[rows].double().numpy(), ref) <= GEMM_REL_FRO_TOL
+    cols = [0, 255, 256, N // 2 + 3, N - 1]
+    ref_c = oracle.gemm_nt(A.double().numpy(), W[cols].double().numpy())
+    assert rel_fro(C[:, cols].double().numpy(), ref_c) <= GEMM_REL_FRO_TOL
