@@ -37,6 +37,8 @@ NOMINAL_FP16_TFLOPS = 2250.0  # datasheet dense figure, context only
 # dram__bytes_read.sum + dram__bytes_write.sum of one bwd_main_kernel launch, from the ncu capture
 # summarised in profiles/bwd_main_kernel_llama2_7b.md (taken on the full configuration itself)
 MAIN_KERNEL_DRAM_BYTES = {"llama2_7b": 688.0e6}
+# (rows, weight rows, weight columns): the paper's GEMM profile shapes at sequence length 2048
+GEMM_SHAPES = [(2048, 4096, 4096), (2048, 11008, 4096), (2048, 4096, 11008), (2048, 6656, 6656), (2048, 8192, 8192)]
 FALLBACK_PEAK_TFLOPS = 1590.0
 FALLBACK_SUSTAINED_TFLOPS = 1400.0
 
@@ -49,6 +51,7 @@ def parse_args():
     ap.add_argument("--config", default="llama2_7b", choices=sorted(workloads.ALL_CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the timed oracle leg (profiling runs)")
+    ap.add_argument("--no-gemm", action="store_true", help="skip the side measurement of the FP16 GEMM primitive")
     ap.add_argument("--clock-sample-ms", type=int, default=600,
                     help="untimed busy period before the timed steps so nvidia-smi samples clocks under load "
                          "(0 for profiler runs)")
@@ -249,6 +252,33 @@ def run_ours(args, cfg):
     f1.record()
     torch.cuda.synchronize()
     fwd_ms = f0.elapsed_time(f1) / fwd_iters
+
+    # the FP16 GEMM primitive on the weight shapes of the paper's GEMM profile (Section 6.6) at its
+    # 2048 rows; a side measurement like the forward, not part of the metric
+    gemm_lines = []
+    if rank == 0 and not args.no_gemm:
+        gws = lt.alloc_workspace(lt.lt_gemm_f16_workspace_bytes())
+        ggen = torch.Generator(device="cuda")
+        ggen.manual_seed(0)
+        for (gm, gn, gk) in GEMM_SHAPES:
+            ga = torch.randn((gm, gk), generator=ggen, device="cuda", dtype=torch.float32).half()
+            gw = (torch.randn((gn, gk), generator=ggen, device="cuda", dtype=torch.float32) * gk ** -0.5).half()
+            gc = torch.empty((gm, gn), device="cuda", dtype=torch.float16)
+            for _ in range(5):
+                lt.lt_gemm_f16(ga, gw, gc, gws, stream)
+            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            g_iters = 30
+            g0.record()
+            for _ in range(g_iters):
+                lt.lt_gemm_f16(ga, gw, gc, gws, stream)
+            g1.record()
+            torch.cuda.synchronize()
+            if lt.lt_attn_check_status(gws) != lt.LT_OK:
+                raise SystemExit("GEMM kernel reported: " + lt.last_cuda_error())
+            g_ms = g0.elapsed_time(g1) / g_iters
+            gemm_lines.append({"M": gm, "N": gn, "K": gk, "ms": g_ms,
+                               "tflops": 2.0 * gm * gn * gk / (g_ms * 1e-3) / 1e12})
+            del ga, gw, gc
     fwd_flops = cfg.flops * 2.0 / 5.0
 
     def step(ev0=None, ev1=None):
@@ -374,6 +404,10 @@ def run_ours(args, cfg):
                                                 + peak_kind + " bf16 burst peak"}},
             "fwd": {"value": fwd_flops / (fwd_ms * 1e-3) / 1e12, "unit": UNIT, "ms": fwd_ms},
         }
+        if gemm_lines:
+            line["gemm"] = {"unit": UNIT, "what": "lt_gemm_f16, C[M,N] = A[M,K] W[N,K]^T, 30 back-to-back launches",
+                            "peak": peak, "peak_source": peak_kind + " bf16 burst (short loops of one kernel)",
+                            "shapes": [dict(g, frac=g["tflops"] / peak) for g in gemm_lines]}
         if not args.no_cpu_baseline and world == 1:
             import oracle
             n_heads = max(1, min(cfg.Hq, 2 * oracle.num_threads()))
