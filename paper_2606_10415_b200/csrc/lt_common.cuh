@@ -377,10 +377,6 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 __device__ __forceinline__ void red_add_v2(float *addr, float a, float b) {
-#ifdef LT_EXP_NO_RED
-    if (a == 1234.5f) asm volatile("red.global.add.v2.f32 [%0], {%1, %2};" ::"l"(addr), "f"(a), "f"(b) : "memory");
-    return;
-#endif
     asm volatile("red.global.add.v2.f32 [%0], {%1, %2};" ::"l"(addr), "f"(a), "f"(b) : "memory");
 }
 __device__ __forceinline__ void red_add_v4(float *addr, float a, float b, float c, float d) {
