@@ -178,6 +178,9 @@ int lt_attn_bwd_bf16(const lt_bf16 *Q, const lt_bf16 *K, const lt_bf16 *V,
 size_t lt_gemm_f16_workspace_bytes(void);
 int lt_gemm_f16(const lt_half *A, const lt_half *W, lt_half *C, int M, int N, int K,
                 void *workspace, size_t workspace_bytes, lt_stream_t stream);
+/* The same product with bfloat16 A, W and C (fp32 accumulation); everything else as lt_gemm_f16. */
+int lt_gemm_bf16(const lt_bf16 *A, const lt_bf16 *W, lt_bf16 *C, int M, int N, int K,
+                 void *workspace, size_t workspace_bytes, lt_stream_t stream);
 
 /* Same computation as lt_attn_fwd followed by lt_attn_bwd, but every tensor pointer is
  * a HOST pointer (pinned memory makes the copies asynchronous).  `arena` is a caller-

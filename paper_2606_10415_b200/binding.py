@@ -24,7 +24,7 @@ LT_ERR_DEVICE_TIMEOUT = 5
 EXPORTS = (
     "lt_attn_fwd_workspace_bytes", "lt_attn_bwd_workspace_bytes", "lt_attn_fwd", "lt_attn_bwd",
     "lt_attn_bwd_profiled", "lt_attn_bwd_noalloc", "lt_attn_fwd_strided", "lt_attn_bwd_strided",
-    "lt_attn_fwd_bf16", "lt_attn_bwd_bf16", "lt_gemm_f16", "lt_gemm_f16_workspace_bytes",
+    "lt_attn_fwd_bf16", "lt_attn_bwd_bf16", "lt_gemm_f16", "lt_gemm_bf16", "lt_gemm_f16_workspace_bytes",
     "lt_attn_host_arena_bytes", "lt_attn_fwd_bwd_host", "lt_attn_check_status", "lt_status_string",
     "lt_last_cuda_error", "lt_attn_bwd_num_launches", "lt_attn_fwd_num_launches", "lt_dbg_tile_gemm",
     "lt_dbg_wait_timeout",
@@ -79,6 +79,8 @@ def _load() -> ctypes.CDLL:
     lib.lt_gemm_f16_workspace_bytes.restype = sz
     lib.lt_gemm_f16.argtypes = [vp] * 3 + [i] * 3 + [vp, sz, vp]
     lib.lt_gemm_f16.restype = i
+    lib.lt_gemm_bf16.argtypes = lib.lt_gemm_f16.argtypes
+    lib.lt_gemm_bf16.restype = i
     lib.lt_attn_bwd_noalloc.argtypes = [vp] * 9 + [i] * 6 + [f, vp]
     lib.lt_attn_bwd_noalloc.restype = i
     lib.lt_attn_fwd_bwd_host.argtypes = [vp] * 9 + [i] * 6 + [f, vp, sz, vp]
@@ -222,13 +224,16 @@ def lt_gemm_f16_workspace_bytes() -> int:
 
 
 def lt_gemm_f16(A, W, C, workspace, stream=None) -> None:
-    """C[M,N] = A[M,K] W[N,K]^T, fp16 device tensors, contiguous; asynchronous on ``stream``."""
+    """C[M,N] = A[M,K] W[N,K]^T, fp16 (or, all three, bfloat16) device tensors, contiguous; asynchronous
+    on ``stream``."""
     _check_layout(A, W, C)
+    fn = _lib.lt_gemm_bf16 if A.dtype == torch.bfloat16 else _lib.lt_gemm_f16
+    _require_dtype(A.dtype, W, C)
     M, K = (int(x) for x in A.shape)
     N = int(W.shape[0])
     if W.shape[1] != K or tuple(C.shape) != (M, N):
         raise ValueError("expected A [M, K], W [N, K], C [M, N]")
-    rc = _lib.lt_gemm_f16(_ptr(A), _ptr(W), _ptr(C), M, N, K, _ptr(workspace),
+    rc = fn(_ptr(A), _ptr(W), _ptr(C), M, N, K, _ptr(workspace),
                           workspace.numel() * workspace.element_size(), _stream_ptr(stream))
     if rc != LT_OK:
         raise LtError("lt_gemm_f16", rc)

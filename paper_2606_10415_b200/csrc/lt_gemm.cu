@@ -51,6 +51,7 @@ __device__ __forceinline__ void gemm_tile_coords(const GemmParams &p, int tile, 
     tn = r / rows;
 }
 
+template <bool kBf16>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
             const GemmParams p) {
@@ -113,7 +114,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc(kGemmBM, kGemmBN, false, false);
+            constexpr uint32_t idesc = make_idesc(kGemmBM, kGemmBN, false, false, kBf16);
             bool ok = true;
             int kb_total = 0, t_local = 0;
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++t_local) {
@@ -172,16 +173,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 #pragma unroll
                         for (int v8 = 0; v8 < 4; ++v8) {
                             uint4 o;
-                            o.x = pack_half2(__uint_as_float(r[8 * v8 + 0]), __uint_as_float(r[8 * v8 + 1]));
-                            o.y = pack_half2(__uint_as_float(r[8 * v8 + 2]), __uint_as_float(r[8 * v8 + 3]));
-                            o.z = pack_half2(__uint_as_float(r[8 * v8 + 4]), __uint_as_float(r[8 * v8 + 5]));
-                            o.w = pack_half2(__uint_as_float(r[8 * v8 + 6]), __uint_as_float(r[8 * v8 + 7]));
+                            o.x = pack2<kBf16>(__uint_as_float(r[8 * v8 + 0]), __uint_as_float(r[8 * v8 + 1]));
+                            o.y = pack2<kBf16>(__uint_as_float(r[8 * v8 + 2]), __uint_as_float(r[8 * v8 + 3]));
+                            o.z = pack2<kBf16>(__uint_as_float(r[8 * v8 + 4]), __uint_as_float(r[8 * v8 + 5]));
+                            o.w = pack2<kBf16>(__uint_as_float(r[8 * v8 + 6]), __uint_as_float(r[8 * v8 + 7]));
                             reinterpret_cast<uint4 *>(c_row + c * 32)[v8] = o;
                         }
                     } else {
 #pragma unroll
                         for (int e = 0; e < 32; ++e)
-                            if (nc + e < p.N) c_row[c * 32 + e] = __float2half_rn(__uint_as_float(r[e]));
+                            if (nc + e < p.N)
+                                reinterpret_cast<uint16_t *>(c_row)[c * 32 + e] =
+                                    static_cast<uint16_t>(pack2<kBf16>(__uint_as_float(r[e]), 0.f) & 0xFFFFu);
                     }
                 }
             }
@@ -199,8 +202,8 @@ extern "C" {
 
 size_t lt_gemm_f16_workspace_bytes(void) { return lt::kStatusBytes; }
 
-int lt_gemm_f16(const lt_half *A, const lt_half *W, lt_half *C, int M, int N, int K, void *workspace,
-                size_t workspace_bytes, lt_stream_t stream) {
+static int gemm_entry(const void *A, const void *W, void *C, int M, int N, int K, void *workspace,
+                      size_t workspace_bytes, lt_stream_t stream, bool bf16) {
     using namespace lt;
     if (!A || !W || !C) return LT_ERR_INVALID_ARG;
     if (M <= 0 || N <= 0 || K <= 0) return LT_ERR_INVALID_ARG;
@@ -224,7 +227,8 @@ int lt_gemm_f16(const lt_half *A, const lt_half *W, lt_half *C, int M, int N, in
     prm.tiles_m = (M + kGemmBM - 1) / kGemmBM;
     prm.tiles_n = (N + kGemmBN - 1) / kGemmBN;
     const size_t smem = sizeof(GemmSmem) + 1024;
-    e = cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    auto kernel = bf16 ? gemm_kernel<true> : gemm_kernel<false>;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return record_cuda_error("cudaFuncSetAttribute(gemm)", e);
     int sms = 148;
     {
@@ -234,10 +238,20 @@ int lt_gemm_f16(const lt_half *A, const lt_half *W, lt_half *C, int M, int N, in
     }
     const long long n_tiles = static_cast<long long>(prm.tiles_m) * prm.tiles_n;
     const int grid = static_cast<int>(n_tiles < sms ? n_tiles : sms);
-    gemm_kernel<<<grid, kGemmThreads, smem, stream>>>(ma, mb, prm);
+    kernel<<<grid, kGemmThreads, smem, stream>>>(ma, mb, prm);
     e = cudaGetLastError();
     if (e != cudaSuccess) return record_cuda_error("gemm_kernel launch", e);
     return LT_OK;
+}
+
+int lt_gemm_f16(const lt_half *A, const lt_half *W, lt_half *C, int M, int N, int K, void *workspace,
+                size_t workspace_bytes, lt_stream_t stream) {
+    return gemm_entry(A, W, C, M, N, K, workspace, workspace_bytes, stream, false);
+}
+
+int lt_gemm_bf16(const lt_bf16 *A, const lt_bf16 *W, lt_bf16 *C, int M, int N, int K, void *workspace,
+                 size_t workspace_bytes, lt_stream_t stream) {
+    return gemm_entry(A, W, C, M, N, K, workspace, workspace_bytes, stream, true);
 }
 
 }  // extern "C"

@@ -79,3 +79,15 @@ def test_gemm_paper_shapes_sampled_rows(lt, oracle, N, K):
     cols = [0, 255, 256, N // 2 + 3, N - 1]
     ref_c = oracle.gemm_nt(A.double().numpy(), W[cols].double().numpy())
     assert rel_fro(C[:, cols].double().numpy(), ref_c) <= GEMM_REL_FRO_TOL
+
+
+@pytest.mark.parametrize("M,N,K", [(129, 257, 136), (512, 768, 1024)])
+def test_gemm_bf16_matches_oracle(lt, oracle, M, N, K):
+    A, W = (t.float().bfloat16() for t in make_operands(M, N, K, seed=7 + M))
+    C = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    ws = lt.alloc_workspace(lt.lt_gemm_f16_workspace_bytes())
+    lt.lt_gemm_f16(A.cuda(), W.cuda(), C, ws)
+    assert lt.lt_attn_check_status(ws) == lt.LT_OK, lt.last_cuda_error()
+    ref = oracle.gemm_nt(A.double().numpy(), W.double().numpy())
+    # bf16 output rounding: 2^-9 per element
+    assert rel_fro(C.cpu().double().numpy(), ref) <= 4e-3
