@@ -63,6 +63,7 @@ bwd_preprocess_kernel(const __half *__restrict__ dO, const __half *__restrict__ 
                       int plain, float inv_scale, unsigned int *status) {
     // `n_rows` counts rows of the padded row space (every head rounded up to S_pad rows), the
     // indexing of delta_ext, lse_ext and dq_acc; padding rows get zeros everywhere.
+    grid_launch_dependents();  // the main kernel sets itself up while this kernel's last blocks run
     constexpr int kLanesPerRow = D / 8;
     constexpr int kRowsPerWarp = 32 / kLanesPerRow;
     constexpr int kRowsPerTrip = kRowsPerWarp * kPreUnroll;
@@ -165,6 +166,7 @@ bwd_finalize_kernel(const float *__restrict__ dq_acc, __half *__restrict__ dQ, l
                     int vec_per_padded_head, int vec_per_row, int Hq, lt_tensor_strides dq_st, int plain) {
     // n_vec8 groups of eight output elements, numbered over the logical [B,Hq,S,D]; the accumulator
     // is indexed in the padded row space (`plain`: contiguous dQ and no padding, so both are group v)
+    grid_dependency_wait();  // launched while the main kernel drains: its reductions must have landed
     const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
     for (long long v = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; v < n_vec8; v += stride) {
         long long src = v, dst = v * 8;
@@ -387,6 +389,9 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    // everything above ran while the preprocess kernel was finishing; its results (row operands, zeroed
+    // accumulator, running maxima, item counter) are read only from here on
+    grid_dependency_wait();
     const uint32_t tmem = sm.tmem_base;
     volatile int *abort_flag = &sm.abort_flag;
 #ifdef LT_BWD_TRACE
@@ -901,6 +906,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #ifdef LT_BWD_TRACE
     const long long trace_teardown_begin = clock64();
 #endif
+    grid_launch_dependents();  // the dQ conversion kernel may be scheduled while the last CTAs finish
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
@@ -991,8 +997,20 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
     const int grid = n_items < sms ? n_items : sms;  // persistent: one CTA per SM walks the item list
     if (ev_main_begin && (e = cudaEventRecord(ev_main_begin, stream)) != cudaSuccess)
         return record_cuda_error("cudaEventRecord", e);
-    bwd_main_kernel<D, kBf16><<<grid, kBwdThreads, smem, stream>>>(mq, mk, mv, mdo, prm);
-    e = cudaGetLastError();
+    // programmatic stream serialisation: the kernel may start before its predecessor has finished and
+    // waits inside for it (grid_dependency_wait)
+    cudaLaunchAttribute pdl;
+    pdl.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    pdl.val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg_main = {};
+    cfg_main.gridDim = dim3(grid);
+    cfg_main.blockDim = dim3(kBwdThreads);
+    cfg_main.dynamicSmemBytes = smem;
+    cfg_main.stream = stream;
+    cfg_main.attrs = &pdl;
+    cfg_main.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg_main, bwd_main_kernel<D, kBf16>, mq, mk, mv, mdo, prm);
+    if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return record_cuda_error("bwd_main_kernel launch", e);
     if (ev_main_end && (e = cudaEventRecord(ev_main_end, stream)) != cudaSuccess)
         return record_cuda_error("cudaEventRecord", e);
@@ -1000,9 +1018,16 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
     const long long n_vec8 = static_cast<long long>(B) * Hq * S * D / 8;
     const long long fwant = (n_vec8 + 255) / 256;
     const int fin_blocks = static_cast<int>(fwant < static_cast<long long>(sms) * 16 ? fwant : sms * 16);
-    bwd_finalize_kernel<kBf16><<<fin_blocks, 256, 0, stream>>>(dq_acc, reinterpret_cast<__half *>(dQ), n_vec8, S * (D / 8),
-                                                        S_pad * (D / 8), D / 8, Hq, lay.dq, plain_fin);
-    e = cudaGetLastError();
+    cudaLaunchConfig_t cfg_fin = {};
+    cfg_fin.gridDim = dim3(fin_blocks);
+    cfg_fin.blockDim = dim3(256);
+    cfg_fin.stream = stream;
+    cfg_fin.attrs = &pdl;
+    cfg_fin.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg_fin, bwd_finalize_kernel<kBf16>, static_cast<const float *>(dq_acc),
+                           reinterpret_cast<__half *>(dQ), n_vec8, S * (D / 8), S_pad * (D / 8), D / 8, Hq, lay.dq,
+                           plain_fin);
+    if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return record_cuda_error("bwd_finalize_kernel launch", e);
     return LT_OK;
 }

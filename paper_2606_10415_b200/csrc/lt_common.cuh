@@ -90,6 +90,14 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
     }
 }
 
+// ----------------------------------------------------------------------------- dependent launches
+// A kernel launched with programmatic stream serialisation may start while the previous kernel of
+// the stream is still running; it must not touch that kernel's results before grid_dependency_wait().
+// The previous kernel lets it start early with grid_launch_dependents() (which takes effect once every
+// CTA of that kernel has executed it or exited).  Without the launch attribute both are no-ops.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ----------------------------------------------------------------------------- fences
 __device__ __forceinline__ void fence_proxy_async_smem() {
     // generic-proxy writes to shared memory become visible to the async proxy (TMA, UMMA)
