@@ -242,6 +242,7 @@ constexpr int kExtBytes = 2048;            // 128 rows x 16 bytes: one operand o
 constexpr float kPScaleLog2Max = 14.f;     // P is kept as P * 2^c with c <= 14 so that fp16(P') <= 16384
 constexpr int kBarComputeWarps = 2, kBarReduceWarps = 1;  // named barrier ids
 constexpr int kItemRing = 4;  // roles are never more than two items apart
+constexpr double kL2BatchBytes = 80.0e6;  // working set of one batch of work items (L2 holds 126 MB)
 
 template <int D>
 struct BwdSmem {
@@ -284,6 +285,7 @@ struct BwdParams {
     __half *dV;
     unsigned int *status;
     int B, Hq, Hkv, S, S_pad, causal;  // S_pad: S rounded up to whole 128-row tiles
+    int units_per_batch;               // (batch, kv head) units per L2-sized batch of work items
     float scale;
     lt_tensor_strides dk_st, dv_st;  // element strides of dK and dV
 };
@@ -297,8 +299,16 @@ __device__ __forceinline__ BwdItem bwd_item(const BwdParams &p, int item) {
     BwdItem w;
     const int n_tiles = (p.S + kTileRows - 1) / kTileRows;  // the last tile may be ragged
     const int n_bg = p.B * p.Hkv;
-    w.j = item / n_bg;
-    const int bg = item - w.j * n_bg;
+    // Items are numbered batch of (batch, kv head) units by batch; inside a batch key tile by key tile
+    // (heavy tiles first), all units of the batch per key tile.  A batch is sized so that everything its
+    // items touch (K, V, the group's Q and dO, the fp32 dQ rows) stays in L2 while the CTAs work
+    // through it; with one batch this is the plain heavy-first order.
+    const int batch = item / (p.units_per_batch * n_tiles);
+    const int first_unit = batch * p.units_per_batch;
+    const int units = min(p.units_per_batch, n_bg - first_unit);
+    const int within = item - first_unit * n_tiles;
+    w.j = within / units;
+    const int bg = first_unit + (within - w.j * units);
     w.b = bg / p.Hkv;
     w.g = bg - w.b * p.Hkv;
     w.i_first = p.causal ? w.j : 0;
@@ -990,6 +1000,18 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
     prm.scale = scale;
     prm.dk_st = lay.dk;
     prm.dv_st = lay.dv;
+    {
+        // bytes one (batch, kv head) unit keeps live: K, V, the group's Q, dO (fp16) and dQ rows (fp32)
+        const int G = Hq / Hkv;
+        const double unit_bytes = static_cast<double>(S_pad) * D * (2.0 * 2 + 2.0 * 2 * G + 4.0 * G);
+        const int n_units = B * Hkv;
+        int n_batches = static_cast<int>(unit_bytes * n_units / kL2BatchBytes) + 1;
+        // CTAs flow from one batch into the next, but the last batch should still offer every SM two items
+        const int max_batches = (n_units * (S_pad / kTileRows)) / (2 * sms);
+        if (n_batches > max_batches) n_batches = max_batches;
+        if (n_batches < 1) n_batches = 1;
+        prm.units_per_batch = (n_units + n_batches - 1) / n_batches;
+    }
     const size_t smem = sizeof(BwdSmem<D>);
     e = cudaFuncSetAttribute(bwd_main_kernel<D, kBf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return record_cuda_error("cudaFuncSetAttribute(bwd_main)", e);
