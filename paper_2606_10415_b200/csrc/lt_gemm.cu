@@ -35,13 +35,15 @@ struct GemmParams {
     unsigned int *status;
     int M, N, K;
     int tiles_m, tiles_n;
+    int group_rows;  // tile rows of A kept hot in L2 while the W column blocks stream past them
 };
 
 // Output tiles are numbered so that consecutive numbers share the W tile (the larger operand tile)
 // and a wave of CTAs covers a compact block of C: tile -> (m, n) with m fastest inside groups of
-// eight tile rows.
+// `group_rows` tile rows (as many rows of A as stay resident in L2, so that W is read from DRAM once
+// per group).
 __device__ __forceinline__ void gemm_tile_coords(const GemmParams &p, int tile, int &tm, int &tn) {
-    constexpr int kGroup = 8;
+    const int kGroup = p.group_rows;
     const int per_group = kGroup * p.tiles_n;
     const int g = tile / per_group;
     const int first_m = g * kGroup;
@@ -226,6 +228,11 @@ static int gemm_entry(const void *A, const void *W, void *C, int M, int N, int K
     prm.M = M; prm.N = N; prm.K = K;
     prm.tiles_m = (M + kGemmBM - 1) / kGemmBM;
     prm.tiles_n = (N + kGemmBN - 1) / kGemmBN;
+    {
+        // about 48 MB of A rows per group (L2 holds 126 MB; the rest is for the W blocks in flight and C)
+        const long long rows = static_cast<long long>(48.0e6 / (static_cast<double>(kGemmBM) * K * 2.0));
+        prm.group_rows = static_cast<int>(rows < 1 ? 1 : (rows > prm.tiles_m ? prm.tiles_m : rows));
+    }
     const size_t smem = sizeof(GemmSmem) + 1024;
     auto kernel = bf16 ? gemm_kernel<true> : gemm_kernel<false>;
     e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
