@@ -154,7 +154,7 @@ BWD_SHAPES = [
 @pytest.mark.parametrize("stds", [(1.0, 1.0), (None, 1e-2)])
 def test_backward_matches_oracle_small(lt, oracle, B, Hq, Hkv, S, D, causal, stds):
     """Several tiles, GQA groups, both head dims; forward state taken from the oracle
-    (O rounded to fp16, LSE to fp32) so the backward is judged on its own."""
+    (O rounded to fp16, LSE to fp32) so the backward is checked on its own."""
     cfg = workloads.custom(B, Hq, Hkv, S, D, causal, qkv_std=stds[0], do_std=stds[1], seed=B * 1000 + S + D)
     Q, K, V, dO = workloads.make_inputs(cfg)
     Qn, Kn, Vn, dOn = (t.double().numpy() for t in (Q, K, V, dO))
