@@ -17,7 +17,7 @@
  *   - Supported shapes: D in {64, 128}, any S >= 1 (a last tile of fewer than 128 rows is
  *     handled inside the kernels; workspace arrays are sized for S rounded up to 128), Hq % Hkv == 0.
  *     Anything else returns LT_ERR_UNSUPPORTED and launches nothing.
- *   - Unless a function says otherwise pointers are DEVICE pointers, 16-byte aligned,
+ *   - Unless a function says otherwise pointers are DEVICE pointers, 16-byte aligned (LSE: 4-byte),
  *     owned by the caller, and must stay valid until the stream reaches the end of the
  *     call's work.  Inputs are never written.  Outputs are fully overwritten.
  *   - Calls only enqueue work on `stream` and return; they do not synchronise and
@@ -188,7 +188,12 @@ int lt_gemm_bf16(const lt_bf16 *A, const lt_bf16 *W, lt_bf16 *C, int M, int N, i
  * that holds the device copies and the workspace.  The call enqueues the host-to-device
  * copies of Q, K, V, dO, the two kernels' work and the device-to-host copies of
  * O, LSE, dQ, dK, dV on `stream`; the host outputs are valid once the stream is
- * synchronised.  O and LSE may be NULL if the caller does not want them back. */
+ * synchronised.  O and LSE may be NULL if the caller does not want them back.
+ * Large problems are cut into chunks of (batch, kv head) units so that the copy in of one chunk, the
+ * kernels of the previous one and the copy back of the one before overlap; the copies run on two
+ * streams the library creates once per device (no device memory is allocated), forked from and
+ * joined back into `stream` with events, so the ordering guarantees above are unchanged.  The status
+ * blocks inside the arena are those of the last chunk. */
 size_t lt_attn_host_arena_bytes(int B, int Hq, int Hkv, int S, int D);
 int lt_attn_fwd_bwd_host(const lt_half *Q, const lt_half *K, const lt_half *V, const lt_half *dO,
                          lt_half *O, float *LSE, lt_half *dQ, lt_half *dK, lt_half *dV,

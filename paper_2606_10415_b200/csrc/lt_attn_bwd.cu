@@ -1076,9 +1076,10 @@ static int bwd_entry(const lt_half *Q, const lt_half *K, const lt_half *V, const
     if (rc != LT_OK) return rc;
     const lt_attn_layout lay = layout ? *layout : contiguous_layout(Hq, Hkv, S, D);
     if (layout && (rc = check_layout(lay, D)) != LT_OK) return rc;
-    const void *ptrs[] = {Q, K, V, O, dO, LSE, dQ, dK, dV};
+    const void *ptrs[] = {Q, K, V, O, dO, dQ, dK, dV};
     for (const void *ptr : ptrs)
         if (!aligned16(ptr)) return LT_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(LSE) & 3u) != 0) return LT_ERR_UNSUPPORTED;  // fp32, read one at a time
     if (!workspace || !aligned256(workspace) || workspace_bytes < lt_attn_bwd_workspace_bytes(B, Hq, Hkv, S, D))
         return LT_ERR_WORKSPACE;
     if ((rc = check_device()) != LT_OK) return rc;

@@ -10,6 +10,7 @@
 // The running row maximum is only raised when it grew by more than 2^8 since the output
 // was last rescaled, so most key tiles need no pass over O.
 #include <algorithm>
+#include <mutex>
 #include <type_traits>
 
 #include "lt_common.cuh"
@@ -456,6 +457,16 @@ static int launch_fwd(const lt_half *Q, const lt_half *K, const lt_half *V, lt_h
     return LT_OK;
 }
 
+// Internal streams and events of the host-buffer entry point, created on first use per device.
+constexpr int kHostMaxChunks = 8, kHostMaxDevices = 64;
+struct HostPipe {
+    bool ready = false;
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    cudaEvent_t ev_start = nullptr, ev_out = nullptr, ev_in[kHostMaxChunks] = {}, ev_comp[kHostMaxChunks] = {};
+};
+static HostPipe g_host_pipe[kHostMaxDevices];
+static std::mutex g_host_pipe_mu;
+
 }  // namespace lt
 
 extern "C" {
@@ -486,9 +497,10 @@ static int fwd_entry(const lt_half *Q, const lt_half *K, const lt_half *V, lt_ha
         lay.q = layout->q; lay.k = layout->k; lay.v = layout->v; lay.o = layout->o;
         if ((rc = check_layout(lay, D)) != LT_OK) return rc;
     }
-    const void *ptrs[] = {Q, K, V, O, LSE};
+    const void *ptrs[] = {Q, K, V, O};
     for (const void *ptr : ptrs)
         if (!aligned16(ptr)) return LT_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(LSE) & 3u) != 0) return LT_ERR_UNSUPPORTED;  // fp32, read and written one at a time
     if (!workspace || !aligned256(workspace) || workspace_bytes < lt_attn_fwd_workspace_bytes(B, Hq, Hkv, S, D))
         return LT_ERR_WORKSPACE;
     if ((rc = check_device()) != LT_OK) return rc;
@@ -551,25 +563,85 @@ int lt_attn_fwd_bwd_host(const lt_half *Q, const lt_half *K, const lt_half *V, c
     void *ws = kbase + 4 * nk + nl + kStatusBytes;
     const size_t ws_bytes = arena_bytes - (4 * nq + 4 * nk + nl + kStatusBytes);
 
-    cudaError_t e;
-#define LT_COPY(dst, src, n, kind)                                                       \
-    if ((e = cudaMemcpyAsync(dst, src, n, kind, stream)) != cudaSuccess)                 \
-        return record_cuda_error("cudaMemcpyAsync", e)
-    LT_COPY(d_Q, Q, bq, cudaMemcpyHostToDevice);
-    LT_COPY(d_K, K, bk, cudaMemcpyHostToDevice);
-    LT_COPY(d_V, V, bk, cudaMemcpyHostToDevice);
-    LT_COPY(d_dO, dO, bq, cudaMemcpyHostToDevice);
-    rc = lt_attn_fwd(d_Q, d_K, d_V, d_O, d_lse, B, Hq, Hkv, S, D, causal, scale, fwd_ws, kStatusBytes, stream);
-    if (rc != LT_OK) return rc;
-    rc = lt_attn_bwd(d_Q, d_K, d_V, d_O, d_dO, d_lse, d_dQ, d_dK, d_dV, B, Hq, Hkv, S, D, causal, scale, ws,
-                     ws_bytes, stream);
-    if (rc != LT_OK) return rc;
-    if (O) LT_COPY(O, d_O, bq, cudaMemcpyDeviceToHost);
-    if (LSE) LT_COPY(LSE, d_lse, bl, cudaMemcpyDeviceToHost);
-    LT_COPY(dQ, d_dQ, bq, cudaMemcpyDeviceToHost);
-    LT_COPY(dK, d_dK, bk, cudaMemcpyDeviceToHost);
-    LT_COPY(dV, d_dV, bk, cudaMemcpyDeviceToHost);
-#undef LT_COPY
+    // ---- chunks of (batch, kv head) units: the host-to-device copy of one chunk, the kernels of the
+    // previous one and the device-to-host copy of the one before run at the same time (two copy engines
+    // and the SMs), on two internal streams beside the caller's.  A chunk is a contiguous slice of every
+    // tensor and a problem of its own with B = 1.
+    const int G = Hq / Hkv;
+    const int n_units = B * Hkv;
+    const long long n_tiles = padded_rows(S) / 128;
+    const long long unit_iters = static_cast<long long>(G) * (causal ? n_tiles * (n_tiles + 1) / 2 : n_tiles * n_tiles);
+    long long want = unit_iters * n_units / 3000;  // a chunk should still fill the GPU
+    int n_chunks = static_cast<int>(want < 1 ? 1 : (want > kHostMaxChunks ? kHostMaxChunks : want));
+    if (n_chunks > n_units) n_chunks = n_units;
+
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return record_cuda_error("cudaGetDevice", e);
+    if (dev < 0 || dev >= kHostMaxDevices) n_chunks = 1;
+    std::lock_guard<std::mutex> lock(g_host_pipe_mu);
+    HostPipe *pipe = nullptr;
+    if (n_chunks > 1) {
+        pipe = &g_host_pipe[dev];
+        if (!pipe->ready) {
+            bool ok = cudaStreamCreateWithFlags(&pipe->s_in, cudaStreamNonBlocking) == cudaSuccess &&
+                      cudaStreamCreateWithFlags(&pipe->s_out, cudaStreamNonBlocking) == cudaSuccess &&
+                      cudaEventCreateWithFlags(&pipe->ev_start, cudaEventDisableTiming) == cudaSuccess &&
+                      cudaEventCreateWithFlags(&pipe->ev_out, cudaEventDisableTiming) == cudaSuccess;
+            for (int c = 0; c < kHostMaxChunks && ok; ++c)
+                ok = cudaEventCreateWithFlags(&pipe->ev_in[c], cudaEventDisableTiming) == cudaSuccess &&
+                     cudaEventCreateWithFlags(&pipe->ev_comp[c], cudaEventDisableTiming) == cudaSuccess;
+            if (!ok) return record_cuda_error("stream/event creation for the host pipeline", cudaGetLastError());
+            pipe->ready = true;
+        }
+    }
+    cudaStream_t s_in = pipe ? pipe->s_in : stream, s_out = pipe ? pipe->s_out : stream;
+#define LT_CUDA(call, what)                      \
+    if ((e = (call)) != cudaSuccess) return record_cuda_error(what, e)
+    if (pipe) {
+        // nothing of this call may start before the work already queued on the caller's stream
+        LT_CUDA(cudaEventRecord(pipe->ev_start, stream), "cudaEventRecord");
+        LT_CUDA(cudaStreamWaitEvent(s_in, pipe->ev_start, 0), "cudaStreamWaitEvent");
+        LT_CUDA(cudaStreamWaitEvent(s_out, pipe->ev_start, 0), "cudaStreamWaitEvent");
+    }
+    for (int c = 0; c < n_chunks; ++c) {
+        const int u0 = static_cast<int>(static_cast<long long>(n_units) * c / n_chunks);
+        const int u1 = static_cast<int>(static_cast<long long>(n_units) * (c + 1) / n_chunks);
+        const int hkv = u1 - u0, hq = hkv * G;
+        const size_t oq = static_cast<size_t>(u0) * G * S * D, ok_ = static_cast<size_t>(u0) * S * D;  // elements
+        const size_t ol = static_cast<size_t>(u0) * G * S;
+        const size_t cq = static_cast<size_t>(hq) * S * D * 2, ck = static_cast<size_t>(hkv) * S * D * 2;
+        const size_t cl = static_cast<size_t>(hq) * S * 4;
+        LT_CUDA(cudaMemcpyAsync(d_Q + oq, Q + oq, cq, cudaMemcpyHostToDevice, s_in), "cudaMemcpyAsync");
+        LT_CUDA(cudaMemcpyAsync(d_K + ok_, K + ok_, ck, cudaMemcpyHostToDevice, s_in), "cudaMemcpyAsync");
+        LT_CUDA(cudaMemcpyAsync(d_V + ok_, V + ok_, ck, cudaMemcpyHostToDevice, s_in), "cudaMemcpyAsync");
+        LT_CUDA(cudaMemcpyAsync(d_dO + oq, dO + oq, cq, cudaMemcpyHostToDevice, s_in), "cudaMemcpyAsync");
+        if (pipe) {
+            LT_CUDA(cudaEventRecord(pipe->ev_in[c], s_in), "cudaEventRecord");
+            LT_CUDA(cudaStreamWaitEvent(stream, pipe->ev_in[c], 0), "cudaStreamWaitEvent");
+        }
+        rc = lt_attn_fwd(d_Q + oq, d_K + ok_, d_V + ok_, d_O + oq, d_lse + ol, 1, hq, hkv, S, D, causal, scale, fwd_ws,
+                         kStatusBytes, stream);
+        if (rc != LT_OK) return rc;
+        rc = lt_attn_bwd(d_Q + oq, d_K + ok_, d_V + ok_, d_O + oq, d_dO + oq, d_lse + ol, d_dQ + oq, d_dK + ok_,
+                         d_dV + ok_, 1, hq, hkv, S, D, causal, scale, ws, ws_bytes, stream);
+        if (rc != LT_OK) return rc;
+        if (pipe) {
+            LT_CUDA(cudaEventRecord(pipe->ev_comp[c], stream), "cudaEventRecord");
+            LT_CUDA(cudaStreamWaitEvent(s_out, pipe->ev_comp[c], 0), "cudaStreamWaitEvent");
+        }
+        if (O) LT_CUDA(cudaMemcpyAsync(O + oq, d_O + oq, cq, cudaMemcpyDeviceToHost, s_out), "cudaMemcpyAsync");
+        if (LSE) LT_CUDA(cudaMemcpyAsync(LSE + ol, d_lse + ol, cl, cudaMemcpyDeviceToHost, s_out), "cudaMemcpyAsync");
+        LT_CUDA(cudaMemcpyAsync(dQ + oq, d_dQ + oq, cq, cudaMemcpyDeviceToHost, s_out), "cudaMemcpyAsync");
+        LT_CUDA(cudaMemcpyAsync(dK + ok_, d_dK + ok_, ck, cudaMemcpyDeviceToHost, s_out), "cudaMemcpyAsync");
+        LT_CUDA(cudaMemcpyAsync(dV + ok_, d_dV + ok_, ck, cudaMemcpyDeviceToHost, s_out), "cudaMemcpyAsync");
+    }
+    if (pipe) {
+        // the caller's stream is done when the last copy back is
+        LT_CUDA(cudaEventRecord(pipe->ev_out, s_out), "cudaEventRecord");
+        LT_CUDA(cudaStreamWaitEvent(stream, pipe->ev_out, 0), "cudaStreamWaitEvent");
+    }
+#undef LT_CUDA
     return LT_OK;
 }
 
