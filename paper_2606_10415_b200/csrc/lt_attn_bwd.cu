@@ -60,10 +60,15 @@ __global__ void __launch_bounds__(256)
 bwd_preprocess_kernel(const __half *__restrict__ dO, const __half *__restrict__ O, const float *__restrict__ lse,
                       uint4 *__restrict__ delta_ext, uint4 *__restrict__ lse_ext, float *__restrict__ dq_acc,
                       long long n_rows, int S, int S_pad, int Hq, lt_tensor_strides do_st, lt_tensor_strides o_st,
-                      int plain, float inv_scale, unsigned int *status) {
+                      int plain, float inv_scale, unsigned int *status, float4 *__restrict__ kv_acc,
+                      long long kv_acc_vec4) {
     // `n_rows` counts rows of the padded row space (every head rounded up to S_pad rows), the
     // indexing of delta_ext, lse_ext and dq_acc; padding rows get zeros everywhere.
     grid_launch_dependents();  // the main kernel sets itself up while this kernel's last blocks run
+    // fp32 dK/dV sums (only when key tiles are split over several work items): zero them
+    for (long long v = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; v < kv_acc_vec4;
+         v += static_cast<long long>(gridDim.x) * blockDim.x)
+        kv_acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
     constexpr int kLanesPerRow = D / 8;
     constexpr int kRowsPerWarp = 32 / kLanesPerRow;
     constexpr int kRowsPerTrip = kRowsPerWarp * kPreUnroll;
@@ -189,6 +194,36 @@ bwd_finalize_kernel(const float *__restrict__ dq_acc, __half *__restrict__ dQ, l
     }
 }
 
+// fp32 dK / dV sums [B,Hkv,S_pad,D] -> 16-bit outputs (only when key tiles were split over work items)
+template <bool kBf16>
+__global__ void __launch_bounds__(256)
+bwd_finalize_kv_kernel(const float *__restrict__ dk_acc, const float *__restrict__ dv_acc, __half *__restrict__ dK,
+                       __half *__restrict__ dV, long long n_vec8, int vec_per_head, int vec_per_padded_head,
+                       int vec_per_row, int Hkv, lt_tensor_strides dk_st, lt_tensor_strides dv_st) {
+    grid_dependency_wait();  // every share of the main kernel must have landed
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    for (long long v = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; v < 2 * n_vec8; v += stride) {
+        const bool second = v >= n_vec8;
+        const long long u = second ? v - n_vec8 : v;
+        const int bh = static_cast<int>(u / vec_per_head);
+        const int rem = static_cast<int>(u - static_cast<long long>(bh) * vec_per_head);
+        const int s_in = rem / vec_per_row, c = rem - s_in * vec_per_row;
+        const int bb = bh / Hkv, hh = bh - bb * Hkv;
+        const long long src = static_cast<long long>(bh) * vec_per_padded_head + rem;
+        const lt_tensor_strides &st = second ? dv_st : dk_st;
+        const long long dst = bb * st.batch + hh * st.head + s_in * st.row + c * 8;
+        const float *acc = second ? dv_acc : dk_acc;
+        const float4 a = __ldcs(reinterpret_cast<const float4 *>(acc) + 2 * src);
+        const float4 b = __ldcs(reinterpret_cast<const float4 *>(acc) + 2 * src + 1);
+        uint4 o;
+        o.x = pack2<kBf16>(a.x, a.y);
+        o.y = pack2<kBf16>(a.z, a.w);
+        o.z = pack2<kBf16>(b.x, b.y);
+        o.w = pack2<kBf16>(b.z, b.w);
+        *reinterpret_cast<uint4 *>((second ? dV : dK) + dst) = o;
+    }
+}
+
 // ----------------------------------------------------------------------------- optional cycle trace
 // Built only with -DLT_BWD_TRACE (development aid): per-role cycle totals, summed over all CTAs.
 // Slot = 16 * role + (wait code - 200); slot 16 * role + 15 = the role's whole loop.
@@ -285,7 +320,12 @@ struct BwdParams {
     __half *dV;
     unsigned int *status;
     int B, Hq, Hkv, S, S_pad, causal;  // S_pad: S rounded up to whole 128-row tiles
-    int units_per_batch;               // (batch, kv head) units per L2-sized batch of work items
+    // (batch, kv head) units per L2-sized batch of work items.  In the variant that splits a group of
+    // query heads over several items the word also carries, above bit 16, the items per (unit, key
+    // tile) and, above bit 24, the query heads per item; dK and dV then point at the fp32 sums
+    // [B,Hkv,S_pad,D] of the parts.  (The structure keeps its size: the main kernel's register
+    // allocation is sensitive to it.)
+    int units_per_batch;
     float scale;
     lt_tensor_strides dk_st, dv_st;  // element strides of dK and dV
 };
@@ -294,26 +334,42 @@ struct BwdParams {
 // ones (small j under a causal mask) come first; CTA c takes items c, c + gridDim.x, ...
 struct BwdItem {
     int j, b, g, i_first, tiles_per_head, n_iter;
+    int h_first;  // first query head of the group this item covers (0 unless the group is split)
 };
+template <bool kSplit>
 __device__ __forceinline__ BwdItem bwd_item(const BwdParams &p, int item) {
     BwdItem w;
+    const int parts = kSplit ? ((p.units_per_batch >> 16) & 0xFF) : 1;
+    const int units_per_batch = kSplit ? (p.units_per_batch & 0xFFFF) : p.units_per_batch;
+    const int heads_per_item = kSplit ? ((p.units_per_batch >> 24) & 0xFF) : 0;
     const int n_tiles = (p.S + kTileRows - 1) / kTileRows;  // the last tile may be ragged
     const int n_bg = p.B * p.Hkv;
     // Items are numbered batch of (batch, kv head) units by batch; inside a batch key tile by key tile
     // (heavy tiles first), all units of the batch per key tile.  A batch is sized so that everything its
     // items touch (K, V, the group's Q and dO, the fp32 dQ rows) stays in L2 while the CTAs work
     // through it; with one batch this is the plain heavy-first order.
-    const int batch = item / (p.units_per_batch * n_tiles);
-    const int first_unit = batch * p.units_per_batch;
-    const int units = min(p.units_per_batch, n_bg - first_unit);
-    const int within = item - first_unit * n_tiles;
-    w.j = within / units;
-    const int bg = first_unit + (within - w.j * units);
+    const int batch = item / (units_per_batch * n_tiles * parts);
+    const int first_unit = batch * units_per_batch;
+    const int units = min(units_per_batch, n_bg - first_unit);
+    // A group of query heads may be split into `parts` items per key tile (shapes with few, heavy
+    // items); the parts of one key tile are neighbours in the numbering.
+    const int within = item - first_unit * n_tiles * parts;
+    w.j = within / (units * parts);
+    const int rem = within - w.j * units * parts;
+    const int unit_local = rem / parts;
+    const int part = rem - unit_local * parts;
+    const int bg = first_unit + unit_local;
     w.b = bg / p.Hkv;
     w.g = bg - w.b * p.Hkv;
     w.i_first = p.causal ? w.j : 0;
     w.tiles_per_head = n_tiles - w.i_first;
-    w.n_iter = (p.Hq / p.Hkv) * w.tiles_per_head;  // flattened (query head of the group, query tile) loop
+    if constexpr (kSplit) {
+        w.h_first = part * heads_per_item;
+        w.n_iter = min(heads_per_item, p.Hq / p.Hkv - w.h_first) * w.tiles_per_head;
+    } else {
+        w.h_first = 0;
+        w.n_iter = (p.Hq / p.Hkv) * w.tiles_per_head;  // flattened (query head of the group, query tile) loop
+    }
     return w;
 }
 // Iteration n of an item -> its query tile: batch, query head, first row inside the head, and the tile's first row in the padded row space of the workspace arrays
@@ -327,13 +383,13 @@ __device__ __forceinline__ BwdQTile bwd_q_tile(const BwdParams &p, const BwdItem
     const int i = w.i_first + (n - hh * w.tiles_per_head);
     BwdQTile q;
     q.b = w.b;
-    q.h = w.g * (p.Hq / p.Hkv) + hh;
+    q.h = w.g * (p.Hq / p.Hkv) + w.h_first + hh;
     q.s0 = i * kTileRows;
     q.padded_row0 = (static_cast<long long>(w.b) * p.Hq + q.h) * p.S_pad + q.s0;
     return q;
 }
 
-template <int D, bool kBf16>
+template <int D, bool kBf16, bool kSplit>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
@@ -352,7 +408,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
     const int lane = tid & 31;
-    const int n_items = (p.S_pad / kTileRows) * p.B * p.Hkv;
+    const int n_items = (p.S_pad / kTileRows) * p.B * p.Hkv * (kSplit ? ((p.units_per_batch >> 16) & 0xFF) : 1);
 
     // the swizzled tiles need 1024-byte alignment; the shared window is expected to give it
     const bool smem_ok = (smem_u32(smem_raw) & 1023u) == 0u;
@@ -430,7 +486,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             };
             int item = claim(0);
             while (item >= 0 && ok) {
-                const BwdItem w = bwd_item(p, item);
+                const BwdItem w = bwd_item<kSplit>(p, item);
                 int next_item = -1;
                 for (int n = 0; n < w.n_iter && ok; ++n, ++it) {
                     const int s = it & 1, k = it >> 1;
@@ -466,7 +522,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         // its K/V tiles to be brought into L2 while this item finishes
                         next_item = claim(ic + 1);
                         if (next_item >= 0) {
-                            const BwdItem wn = bwd_item(p, next_item);
+                            const BwdItem wn = bwd_item<kSplit>(p, next_item);
 #pragma unroll
                             for (int x = 0; x < kBoxes; ++x) {
                                 tma_prefetch_l2_4d(&map_k, x * 64, wn.j * kTileRows, wn.g, wn.b);
@@ -531,7 +587,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 if (!(ok = LT_WAIT(&sm.bar_item[ic % kItemRing], (ic / kItemRing) & 1, kWaitItem))) break;
                 const int item = sm.item_ring[ic % kItemRing];
                 if (item < 0) break;
-                const BwdItem w = bwd_item(p, item);
+                const BwdItem w = bwd_item<kSplit>(p, item);
                 ok = LT_WAIT(&sm.bar_kv, ic & 1, kWaitKV) &&
                      LT_WAIT(&sm.bar_q_full[it & 1], (it >> 1) & 1, kWaitStageFull);
                 if (!ok) break;
@@ -658,7 +714,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             // (after an abandoned wait the loop still comes here, so that the vote below is never short of a warp)
             ok = ok && LT_WAIT(&sm.bar_item[ic % kItemRing], (ic / kItemRing) & 1, kWaitItem);
             const int item = ok ? sm.item_ring[ic % kItemRing] : -1;
-            const BwdItem w = bwd_item(p, item < 0 ? 0 : item);
+            const BwdItem w = bwd_item<kSplit>(p, item < 0 ? 0 : item);
             // ---- per item: a power-of-two factor 2^c carried by dS before it is rounded to fp16, chosen
             // from a bound on |dS| <= |dP| + |delta| <= max||dO_row|| * max||V_row|| + max|delta| so that
             // the scaled values use fp16's normal range without overflow.  The factor rides on P
@@ -757,7 +813,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             if (!ok) break;
             const int item = sm.item_ring[ic % kItemRing];
             if (item < 0) break;
-            const BwdItem w = bwd_item(p, item);
+            const BwdItem w = bwd_item<kSplit>(p, item);
             float dq_mult = 0.f, inv_p_scale = 0.f;
             for (int n = 0; n < w.n_iter; ++n, ++it) {
                 ok = LT_WAIT(&sm.bar_dq_full, it & 1, kWaitDqFull);
@@ -892,6 +948,20 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                             __syncwarp();
                             if (lane == 0) mbar_arrive(&sm.bar_acc_free);
                         }
+                        if constexpr (kSplit) {
+                            // the group's heads are spread over several items: add this item's share to
+                            // the fp32 sums; a separate pass rounds them once all shares are in
+                            float *acc = reinterpret_cast<float *>(which == 0 ? p.dK : p.dV) +
+                                         ((static_cast<long long>(w.b) * p.Hkv + w.g) * p.S_pad + s_row) * D + c * 32;
+                            if (s_row < p.S) {
+#pragma unroll
+                                for (int v4 = 0; v4 < 8; ++v4)
+                                    red_add_v4(acc + 4 * v4, __uint_as_float(r[4 * v4 + 0]) * mult,
+                                               __uint_as_float(r[4 * v4 + 1]) * mult, __uint_as_float(r[4 * v4 + 2]) * mult,
+                                               __uint_as_float(r[4 * v4 + 3]) * mult);
+                            }
+                            continue;
+                        }
 #pragma unroll
                         for (int v8 = 0; v8 < 4; ++v8) {
                             uint4 o;
@@ -942,6 +1012,24 @@ extern "C" int lt_dbg_bwd_trace(unsigned long long *out, int reset) {
 }
 #endif
 
+// Query heads of a group per work item.  A (batch, kv head, key tile) item normally covers the whole
+// group (dK_j, dV_j of all its heads accumulate in one CTA's tensor memory).  Shapes that would give
+// the 148 SMs only a few, heavy items get the group split over several items instead; their shares of
+// dK_j, dV_j are then summed in fp32 in the workspace and rounded by a small extra kernel.
+constexpr int kSplitBelowItems = 148 + 148 / 2;  // split when there are fewer than 1.5 whole-group items per SM
+constexpr int kSplitTargetItems = 2 * 148;       // and then aim at two items per SM (every item pays a pipeline fill)
+constexpr long long kSplitMinIterations = 20 * 148;  // problems below this are launch-bound anyway
+static int heads_per_item(int B, int Hq, int Hkv, int S, int causal) {
+    const int G = Hq / Hkv;
+    const long long n_tiles = padded_rows(S) / kTileRows;
+    const long long n_base = static_cast<long long>(B) * Hkv * n_tiles;
+    const long long iters = static_cast<long long>(B) * Hq * (causal ? n_tiles * (n_tiles + 1) / 2 : n_tiles * n_tiles);
+    if (G == 1 || n_base >= kSplitBelowItems || iters < kSplitMinIterations) return G;
+    const long long split = (kSplitTargetItems + n_base - 1) / n_base;
+    const int hs = static_cast<int>(split < G ? split : G);
+    return (G + hs - 1) / hs;
+}
+
 template <int D, bool kBf16>
 static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, const lt_half *O, const lt_half *dO,
                       const float *LSE, lt_half *dQ, lt_half *dK, lt_half *dV, const lt_attn_layout &lay, int B,
@@ -962,6 +1050,14 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
     uint4 *delta_ext = reinterpret_cast<uint4 *>(ws + kStatusBytes);
     uint4 *lse_ext = reinterpret_cast<uint4 *>(ws + kStatusBytes + ext_bytes);
     float *dq_acc = reinterpret_cast<float *>(ws + kStatusBytes + 2 * ext_bytes);
+    const int hpi = heads_per_item(B, Hq, Hkv, S, causal);
+    const int parts = (Hq / Hkv + hpi - 1) / hpi;
+    const size_t kv_floats = static_cast<size_t>(B) * Hkv * S_pad * D;
+    float *dk_acc = nullptr, *dv_acc = nullptr;
+    if (parts > 1) {
+        dk_acc = reinterpret_cast<float *>(ws + kStatusBytes + 2 * ext_bytes + round256(static_cast<size_t>(n_rows) * D * 4));
+        dv_acc = dk_acc + kv_floats;  // kv_floats * 4 is a multiple of 256 bytes
+    }
 
     CUtensorMap mq, mk, mv, mdo;
     int rc;
@@ -985,7 +1081,8 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
     bwd_preprocess_kernel<D, kBf16><<<pre_blocks, 256, 0, stream>>>(reinterpret_cast<const __half *>(dO),
                                                              reinterpret_cast<const __half *>(O), LSE, delta_ext,
                                                              lse_ext, dq_acc, n_rows, S, S_pad, Hq, lay.d_o, lay.o, plain_pre,
-                                                             1.f / scale, status);
+                                                             1.f / scale, status, reinterpret_cast<float4 *>(dk_acc),
+                                                             parts > 1 ? static_cast<long long>(kv_floats / 2) : 0LL);
     e = cudaGetLastError();
     if (e != cudaSuccess) return record_cuda_error("bwd_preprocess_kernel launch", e);
 
@@ -1007,15 +1104,25 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
         const int n_units = B * Hkv;
         int n_batches = static_cast<int>(unit_bytes * n_units / kL2BatchBytes) + 1;
         // CTAs flow from one batch into the next, but the last batch should still offer every SM two items
-        const int max_batches = (n_units * (S_pad / kTileRows)) / (2 * sms);
+        const int max_batches = (n_units * (S_pad / kTileRows) * parts) / (2 * sms);
         if (n_batches > max_batches) n_batches = max_batches;
         if (n_batches < 1) n_batches = 1;
         prm.units_per_batch = (n_units + n_batches - 1) / n_batches;
+        if (parts > 1) {
+            if (prm.units_per_batch > 0xFFFF || parts > 0xFF || hpi > 0x7F) {
+                set_last_error("lt_attn_bwd", "shape too large for the split-group variant");
+                return LT_ERR_UNSUPPORTED;
+            }
+            prm.units_per_batch |= (parts << 16) | (hpi << 24);
+            prm.dK = reinterpret_cast<__half *>(dk_acc);
+            prm.dV = reinterpret_cast<__half *>(dv_acc);
+        }
     }
     const size_t smem = sizeof(BwdSmem<D>);
-    e = cudaFuncSetAttribute(bwd_main_kernel<D, kBf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    auto main_kernel = parts > 1 ? bwd_main_kernel<D, kBf16, true> : bwd_main_kernel<D, kBf16, false>;
+    e = cudaFuncSetAttribute(main_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return record_cuda_error("cudaFuncSetAttribute(bwd_main)", e);
-    const int n_items = B * Hkv * (S_pad / kTileRows);
+    const int n_items = B * Hkv * (S_pad / kTileRows) * parts;
     const int grid = n_items < sms ? n_items : sms;  // persistent: one CTA per SM walks the item list
     if (ev_main_begin && (e = cudaEventRecord(ev_main_begin, stream)) != cudaSuccess)
         return record_cuda_error("cudaEventRecord", e);
@@ -1031,7 +1138,7 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
     cfg_main.stream = stream;
     cfg_main.attrs = &pdl;
     cfg_main.numAttrs = 1;
-    e = cudaLaunchKernelEx(&cfg_main, bwd_main_kernel<D, kBf16>, mq, mk, mv, mdo, prm);
+    e = cudaLaunchKernelEx(&cfg_main, main_kernel, mq, mk, mv, mdo, prm);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return record_cuda_error("bwd_main_kernel launch", e);
     if (ev_main_end && (e = cudaEventRecord(ev_main_end, stream)) != cudaSuccess)
@@ -1051,6 +1158,17 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
                            plain_fin);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return record_cuda_error("bwd_finalize_kernel launch", e);
+    if (parts > 1) {
+        const long long kv_vec8 = static_cast<long long>(B) * Hkv * S * D / 8;
+        const long long kwant = (2 * kv_vec8 + 255) / 256;
+        cfg_fin.gridDim = dim3(static_cast<int>(kwant < static_cast<long long>(sms) * 16 ? kwant : sms * 16));
+        e = cudaLaunchKernelEx(&cfg_fin, bwd_finalize_kv_kernel<kBf16>, static_cast<const float *>(dk_acc),
+                               static_cast<const float *>(dv_acc), reinterpret_cast<__half *>(dK),
+                               reinterpret_cast<__half *>(dV), kv_vec8, S * (D / 8), S_pad * (D / 8), D / 8, Hkv, lay.dk,
+                               lay.dv);
+        if (e == cudaSuccess) e = cudaGetLastError();
+        if (e != cudaSuccess) return record_cuda_error("bwd_finalize_kv_kernel launch", e);
+    }
     return LT_OK;
 }
 
@@ -1061,7 +1179,12 @@ extern "C" {
 size_t lt_attn_bwd_workspace_bytes(int B, int Hq, int Hkv, int S, int D) {
     if (lt::check_shape(B, Hq, Hkv, S, D, 1.0f) != LT_OK) return 0;
     const size_t n_rows = static_cast<size_t>(B) * Hq * static_cast<size_t>(lt::padded_rows(S));
-    return lt::kStatusBytes + 2 * lt::round256(n_rows * 16) + lt::round256(n_rows * D * 4);
+    size_t bytes = lt::kStatusBytes + 2 * lt::round256(n_rows * 16) + lt::round256(n_rows * D * 4);
+    // fp32 dK / dV sums for shapes whose groups are split over work items (either mask; sized for the
+    // unmasked case, which splits no less often)
+    if (lt::heads_per_item(B, Hq, Hkv, S, 1) < Hq / Hkv || lt::heads_per_item(B, Hq, Hkv, S, 0) < Hq / Hkv)
+        bytes += 2 * lt::round256(static_cast<size_t>(B) * Hkv * static_cast<size_t>(lt::padded_rows(S)) * D * 4);
+    return bytes;
 }
 
 int lt_attn_bwd_num_launches(void) { return 3; }
