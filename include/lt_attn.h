@@ -224,7 +224,11 @@ int lt_attn_fwd_num_launches(void);
  *   mode 4: as mode 0, with the accumulator read back in the 16-lane x 256-bit
  *           arrangement that the dQ reduction uses
  *   mode 5: C = A B^T + 1000 * B[n][0] added to column n through one extra, unswizzled
- *           contraction step (the way the kernels subtract LSE and delta) */
+ *           contraction step (the way the kernels subtract LSE and delta)
+ *   mode 6: no product is read back: the first 96 columns of C receive 1000 * row + column, written
+ *           to tensor memory with the two 16-lane store arrangements (64 columns as 32-bit values,
+ *           32 columns in the arrangement used for packed 16-bit pairs) and read back with the
+ *           32-lane arrangement; checks the register-to-element maps the forward relies on */
 int lt_dbg_tile_gemm(const lt_half *A, const lt_half *B, float *C, int mode,
                      void *workspace, size_t workspace_bytes, lt_stream_t stream);
 

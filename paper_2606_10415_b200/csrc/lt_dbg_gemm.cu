@@ -92,7 +92,7 @@ dbg_tile_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             const uint32_t koff = (kk >> 2) * kBoxBytes + (kk & 3) * 32;  // contraction-contiguous operand
             const uint32_t roff = kk * 16 * 128;                          // contraction index = row
             const uint32_t acc = kk > 0;
-            if (mode == 0 || mode == 4 || mode == 5) {
+            if (mode == 0 || mode == 4 || mode == 5 || mode == 6) {
                 umma_ss(tmem, desc_kmajor(a0 + koff), desc_kmajor(b0 + koff), make_idesc(128, 128, false, false), acc);
             } else if (mode == 1) {
                 umma_ss(tmem, desc_kmajor(a0 + koff), desc_mnmajor(b0 + roff, kBoxBytes),
@@ -153,6 +153,45 @@ dbg_tile_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                         make_float2(__uint_as_float(r[4 * k + 2]), __uint_as_float(r[4 * k + 3]));
                 }
             }
+        }
+    } else if (ok && mode == 6) {
+        // store-arrangement probe: no product is needed; every thread writes the value
+        // 1000 * row + column it believes it owns with the two 16-lane store shapes, the tile is read back
+        // with the plain 32-lane shape and the host checks C[row][col] = 1000 * row + col for col < 96
+        const int lane = tid & 31;
+#pragma unroll
+        for (int lh = 0; lh < 2; ++lh) {
+            const int row0 = warp * 32 + lh * 16 + (lane >> 2);
+            uint32_t r[32];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int col = 8 * k + 2 * (lane & 3);
+                r[4 * k + 0] = __float_as_uint(1000.f * row0 + col);
+                r[4 * k + 1] = __float_as_uint(1000.f * row0 + col + 1);
+                r[4 * k + 2] = __float_as_uint(1000.f * (row0 + 8) + col);
+                r[4 * k + 3] = __float_as_uint(1000.f * (row0 + 8) + col + 1);
+            }
+            tmem_st_16x256b_x8(tmem + (static_cast<uint32_t>(warp * 32 + lh * 16) << 16), r);
+            uint32_t q[16];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int col = 64 + 4 * k + (lane & 3);
+                q[2 * k + 0] = __float_as_uint(1000.f * row0 + col);
+                q[2 * k + 1] = __float_as_uint(1000.f * (row0 + 8) + col);
+            }
+            tmem_st_16x128b_x8(tmem + (static_cast<uint32_t>(warp * 32 + lh * 16) << 16) + 64, q);
+        }
+        tmem_wait_st();
+#pragma unroll
+        for (int c = 0; c < 3; ++c) {
+            uint32_t r[32];
+            tmem_ld32(tmem + lane_base + c * 32, r);
+            tmem_wait_ld();
+            float4 *dst = reinterpret_cast<float4 *>(c_gmem + static_cast<size_t>(tid) * kTile + c * 32);
+#pragma unroll
+            for (int v = 0; v < 8; ++v)
+                dst[v] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                     __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
         }
     } else if (ok) {
 #pragma unroll
@@ -218,7 +257,7 @@ extern "C" int lt_dbg_wait_timeout(void *workspace, size_t workspace_bytes, lt_s
 extern "C" int lt_dbg_tile_gemm(const lt_half *A, const lt_half *B, float *C, int mode, void *workspace,
                                 size_t workspace_bytes, lt_stream_t stream) {
     using namespace lt;
-    if (!A || !B || !C || mode < 0 || mode > 5) return LT_ERR_INVALID_ARG;
+    if (!A || !B || !C || mode < 0 || mode > 6) return LT_ERR_INVALID_ARG;
     if (!aligned16(A) || !aligned16(B) || !aligned16(C)) return LT_ERR_UNSUPPORTED;
     if (!workspace || !aligned256(workspace) || workspace_bytes < static_cast<size_t>(kStatusBytes))
         return LT_ERR_WORKSPACE;

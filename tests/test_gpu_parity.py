@@ -81,6 +81,19 @@ def test_tile_gemm_operand_conventions(lt, mode):
     assert err < (2e-2 if mode == 5 else 1e-3), f"mode {mode}: max abs error {err}"
 
 
+def test_tensor_memory_store_arrangements(lt):
+    """The two 16-lane store shapes put every register where the kernels assume (mode 6 writes
+    1000 * row + column through them and reads the tile back with the 32-lane shape)."""
+    A = torch.zeros(128, 128).half().cuda()
+    C = torch.full((128, 128), float("nan"), dtype=torch.float32, device="cuda")
+    ws = lt.alloc_workspace(256)
+    lt.lt_dbg_tile_gemm(A, A, C, 6, ws)
+    assert lt.lt_attn_check_status(ws) == lt.LT_OK, lt.last_cuda_error()
+    rows = torch.arange(128, dtype=torch.float32)[:, None]
+    cols = torch.arange(96, dtype=torch.float32)[None, :]
+    assert torch.equal(C.cpu()[:, :96], 1000.0 * rows + cols)
+
+
 def test_bounded_wait_reports_timeout_and_context_survives(lt):
     """A wait that nothing satisfies gives up, records its code, and the next call still works."""
     ws = lt.alloc_workspace(256)
