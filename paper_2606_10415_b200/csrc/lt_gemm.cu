@@ -119,16 +119,25 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             constexpr uint32_t idesc = make_idesc(kGemmBM, kGemmBN, false, false, kBf16);
             bool ok = true;
             int kb_total = 0, t_local = 0;
+#ifdef LT_GEMM_TRACE
+            long long tr_full = 0, tr_acc = 0, tr_issue = 0, tr_t = clock64();
+#define LT_GT(var) do { const long long n_ = clock64(); var += n_ - tr_t; tr_t = n_; } while (0)
+#else
+#define LT_GT(var)
+#endif
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++t_local) {
                 const int acc = t_local & 1;
                 const uint32_t acc_use = t_local >> 1;
                 // the epilogue must have read this accumulator's previous tile
                 if (acc_use >= 1 && !(ok = mbar_wait(&sm.bar_acc_empty[acc], (acc_use - 1) & 1, abort_flag, p.status, kWaitGemmAccEmpty)))
                     break;
+                LT_GT(tr_acc);
                 tc_fence_after_sync();
                 for (int kb = 0; kb < k_blocks; ++kb, ++kb_total) {
                     const int s = kb_total % kGemmStages;
+                    LT_GT(tr_issue);
                     if (!(ok = mbar_wait(&sm.bar_full[s], (kb_total / kGemmStages) & 1, abort_flag, p.status, kWaitGemmFull))) break;
+                    LT_GT(tr_full);
                     tc_fence_after_sync();
                     const uint64_t da = desc_kmajor(smem_u32(sm.a[s])), db = desc_kmajor(smem_u32(sm.b[s]));
 #pragma unroll
@@ -138,7 +147,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 }
                 if (!ok) break;
                 umma_commit(&sm.bar_acc_full[acc]);
+                LT_GT(tr_issue);
             }
+#ifdef LT_GEMM_TRACE
+            if (blockIdx.x == 0) {
+                p.status[8] = static_cast<unsigned int>(tr_full >> 4);
+                p.status[9] = static_cast<unsigned int>(tr_acc >> 4);
+                p.status[10] = static_cast<unsigned int>(tr_issue >> 4);
+                p.status[11] = static_cast<unsigned int>(kb_total);
+            }
+#endif
         }
     } else {
         // epilogue: thread = row of the tile, 32 columns at a time
