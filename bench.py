@@ -211,7 +211,22 @@ def job_throughput(flops_per_rank, world, seconds_per_step):
 
 # ------------------------------------------------------------------ GPU arm
 
+def ensure_library():
+    """Build the CUDA library in-tree if it is not there yet (local rank 0 builds, the others wait)."""
+    lib = ROOT / "paper_2606_10415_b200" / "liblt_attn.so"
+    if lib.exists():
+        return
+    if int(os.environ.get("LOCAL_RANK", "0")) == 0:
+        from paper_2606_10415_b200 import build as lib_build
+        lib_build.build()
+        return
+    deadline = time.time() + 900
+    while not lib.exists() and time.time() < deadline:
+        time.sleep(2)
+
+
 def run_ours(args, cfg):
+    ensure_library()
     from paper_2606_10415_b200 import binding as lt
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
