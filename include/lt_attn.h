@@ -208,7 +208,10 @@ int lt_attn_check_status(const void *workspace, lt_stream_t stream);
 const char *lt_status_string(int status);
 const char *lt_last_cuda_error(void);
 
-/* Number of kernels one call enqueues (for launch accounting by benchmarks). */
+/* Number of kernels one call enqueues (for launch accounting by benchmarks): the backward's
+ * preprocess, main and dQ-conversion kernels (a fourth, the dK/dV conversion, only on grouped-query
+ * shapes with fewer than about 1.5 key-tile work items per SM, where a group's query heads are split
+ * over several items), the forward's single kernel. */
 int lt_attn_bwd_num_launches(void);
 int lt_attn_fwd_num_launches(void);
 
