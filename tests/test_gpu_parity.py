@@ -303,6 +303,20 @@ def test_two_streams_with_distinct_workspaces(lt, oracle):
         assert rel_fro(outs[0].cpu().double().numpy(), alone[0].double().numpy()) < 1e-3
 
 
+def test_very_long_sequence(lt, oracle):
+    """S = 16384: 128 key tiles per head, 8 256 tile pairs per head, dQ rows that receive up to 128
+    partial sums."""
+    cfg = workloads.custom(1, 2, 1, 16384, 128, True, seed=25)
+    Q, K, V, dO = workloads.make_inputs(cfg)
+    O, LSE = run_fwd(lt, Q, K, V, cfg)
+    got = run_bwd(lt, Q, K, V, O.cpu(), dO, LSE.cpu(), cfg)
+    Qn, Kn, Vn, dOn = (t.double().numpy() for t in (Q, K, V, dO))
+    O_ref, LSE_ref = oracle.attn_fwd(Qn, Kn, Vn, True, cfg.scale)
+    assert rel_fro(O.cpu().double().numpy(), O_ref) <= FWD_O_REL_FRO_TOL
+    assert max_abs(LSE.cpu().double().numpy(), LSE_ref) <= FWD_LSE_ABS_TOL
+    check_grads(got, oracle.attn_bwd(Qn, Kn, Vn, dOn, True, cfg.scale), "S=16384")
+
+
 def test_host_buffer_entry_point(lt, oracle):
     cfg = workloads.custom(1, 4, 2, 256, 128, True, seed=13)
     Q, K, V, dO = (t.pin_memory() for t in workloads.make_inputs(cfg))
