@@ -1,0 +1,89 @@
+"""Seeded random sweep over shapes, masks, dtypes, layouts, magnitudes and scales: forward and
+backward through the strided / bfloat16 entry points against the fp64 oracle."""
+import random
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2606_10415_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def lt():
+    from paper_2606_10415_b200 import binding
+    return binding
+
+
+def rel(a, b):
+    return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
+
+
+def draw_case(rnd, case):
+    D = rnd.choice([64, 128])
+    Hkv = rnd.choice([1, 2, 3])
+    G = rnd.choice([1, 1, 2, 4, 5])
+    B = rnd.choice([1, 2, 3])
+    S = rnd.choice([1, 7, 64, 127, 128, 129, 200, 255, 256, 257, 300, 384, 500, 640, 777, 1024])
+    causal = rnd.random() < 0.6
+    bf16 = rnd.random() < 0.3
+    layout = rnd.choice(["bhsd", "bshd", "padded_rows"])
+    std = rnd.choice([1.0, D ** -0.25, 0.5])
+    do_std = rnd.choice([1.0, 1e-2])
+    scale = rnd.choice([D ** -0.5, 0.3 * D ** -0.5, -(D ** -0.5)])
+    pad = 8 * rnd.choice([1, 2, 5])
+    cfg = workloads.custom(B, Hkv * G, Hkv, S, D, causal, qkv_std=std, do_std=do_std, seed=1000 + case)
+    return cfg, bf16, layout, scale, pad
+
+
+def place(t, layout, pad, fill=None):
+    """A device [B,H,S,D] view of `t` (or of a tensor filled with `fill`) in the given memory layout."""
+    if layout == "bhsd":
+        return t.clone().cuda() if fill is None else torch.full_like(t, fill).cuda()
+    if layout == "bshd":
+        base = t.permute(0, 2, 1, 3).contiguous()
+        base = (base if fill is None else torch.full_like(base, fill)).cuda()
+        return base.permute(0, 2, 1, 3)
+    Bb, H, S, D = t.shape  # rows padded to D + pad elements
+    buf = torch.full((Bb, H, S, D + pad), 3.0 if fill is None else fill, dtype=t.dtype, device="cuda")
+    view = buf[..., :D]
+    if fill is None:
+        view.copy_(t.cuda())
+    return view
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_random_sweep(lt, oracle, seed):
+    rnd = random.Random(seed)
+    for case in range(16):
+        cfg, bf16, layout, scale, pad = draw_case(rnd, 100 * seed + case)
+        dt = torch.bfloat16 if bf16 else torch.float16
+        Q, K, V, dO = (t.float().to(dt) for t in workloads.make_inputs(cfg))
+        Qd, Kd, Vd, dOd = (place(t, layout, pad) for t in (Q, K, V, dO))
+        O, dQ = place(Q, layout, pad, float("nan")), place(Q, layout, pad, float("nan"))
+        dK, dV = place(K, layout, pad, float("nan")), place(V, layout, pad, float("nan"))
+        LSE = torch.full(Q.shape[:3], float("nan"), dtype=torch.float32, device="cuda")
+        dims = (cfg.B, cfg.Hq, cfg.Hkv, cfg.S, cfg.D)
+        fws = lt.alloc_workspace(lt.lt_attn_fwd_workspace_bytes(*dims))
+        ws = lt.alloc_workspace(lt.lt_attn_bwd_workspace_bytes(*dims))
+        ws.fill_(0xFF)
+        fwd = lt.lt_attn_fwd_bf16 if bf16 else lt.lt_attn_fwd_strided
+        bwd = lt.lt_attn_bwd_bf16 if bf16 else lt.lt_attn_bwd_strided
+        fwd(Qd, Kd, Vd, O, LSE, cfg.causal, scale, fws)
+        bwd(Qd, Kd, Vd, O, dOd, LSE, dQ, dK, dV, cfg.causal, scale, ws)
+        what = f"seed {seed} case {case}: {cfg} bf16={bf16} {layout} scale={scale:.4f}"
+        assert lt.lt_attn_check_status(fws) == lt.LT_OK and lt.lt_attn_check_status(ws) == lt.LT_OK, what
+        n = [t.double().numpy() for t in (Q, K, V, dO)]
+        O_ref, LSE_ref = oracle.attn_fwd(*n[:3], cfg.causal, scale)
+        ref = oracle.attn_bwd(*n, cfg.causal, scale)
+        assert rel(O.cpu().double().numpy(), O_ref) <= (4e-3 if bf16 else 2e-3), what
+        assert np.abs(LSE.cpu().double().numpy() - LSE_ref).max() <= 2e-3 * max(1.0, np.abs(LSE_ref).max() / 10), what
+        for name, g, r in zip(("dQ", "dK", "dV"), (dQ, dK, dV), ref):
+            g = g.cpu().double().numpy()
+            assert np.all(np.isfinite(g)), f"{what} {name}"
+            if np.linalg.norm(r) > 1e-12:  # (a single visible key makes dQ and dK exactly zero)
+                assert rel(g, r) <= (6e-3 if bf16 else 5e-3), f"{what} {name}: {rel(g, r):.3e}"
+            else:
+                assert np.abs(g).max() <= 1e-6, f"{what} {name}"
