@@ -8,8 +8,9 @@
  * not stored by the forward: it is rebuilt tile by tile from the row log-sum-exp.
  *
  * Conventions shared by every entry point
- *   - Tensors are contiguous [B, H, S, D] with D innermost.  Q, O, dO, dQ have H = Hq;
- *     K, V, dK, dV have H = Hkv.  LSE is fp32 [B, Hq, S].  fp16 is IEEE binary16.
+ *   - Tensors are contiguous [B, H, S, D] with D innermost (strided views: the *_strided and
+ *     *_bf16 entry points).  Q, O, dO, dQ have H = Hq; K, V, dK, dV have H = Hkv.  LSE is fp32
+ *     [B, Hq, S].  fp16 is IEEE binary16.
  *   - Grouped-query attention: query head h reads key/value head h / (Hq / Hkv);
  *     dK and dV are summed over the Hq / Hkv query heads of a group.
  *   - scores = scale * Q K^T with a finite, non-zero scale; causal != 0 hides key j from query i when j > i.
@@ -56,9 +57,11 @@ typedef unsigned short lt_half;
 typedef unsigned short lt_bf16;
 
 /* Bytes of caller-owned device workspace the calls below need; 0 means the shape is
- * not supported.  The workspace must be 256-byte aligned.  Layout (backward): a
- * 256-byte status block, -delta and -LSE/scale as 16-byte rows of fp16 (hi, lo, 0 x 6)
- * with 256*hi + lo = value, [B,Hq,S] rows each, then an fp32 dQ accumulator [B,Hq,S,D]. */
+ * not supported.  The workspace must be 256-byte aligned.  Layout (backward), with S_pad = S
+ * rounded up to a multiple of 128: a 256-byte status block, -delta and -LSE/scale as 16-byte rows
+ * of fp16 (hi, lo, 0 x 6) with 256*hi + lo = value, [B,Hq,S_pad] rows each, an fp32 dQ accumulator
+ * [B,Hq,S_pad,D], and, for the grouped-query shapes whose groups are split over work items (see
+ * lt_attn_bwd_num_launches), fp32 dK and dV sums [B,Hkv,S_pad,D] each. */
 size_t lt_attn_fwd_workspace_bytes(int B, int Hq, int Hkv, int S, int D);
 size_t lt_attn_bwd_workspace_bytes(int B, int Hq, int Hkv, int S, int D);
 
@@ -80,7 +83,10 @@ int lt_attn_fwd(const lt_half *Q, const lt_half *K, const lt_half *V,
  *   in : Q, O, dO [B,Hq,S,D] fp16; K, V [B,Hkv,S,D] fp16; LSE [B,Hq,S] fp32
  *   out: dQ [B,Hq,S,D], dK, dV [B,Hkv,S,D] fp16 (overwritten, not accumulated into)
  * dQ is accumulated in fp32 in the workspace with atomic adds, so its last bits may
- * differ between runs; dK and dV are bitwise reproducible. */
+ * differ between runs; dK and dV are bitwise reproducible, except on the grouped-query shapes
+ * whose groups are split over work items (see lt_attn_bwd_num_launches), where they are summed
+ * the same way.  The main and conversion kernels are launched with programmatic stream
+ * serialisation (each starts under the tail of its predecessor and waits inside for it). */
 int lt_attn_bwd(const lt_half *Q, const lt_half *K, const lt_half *V,
                 const lt_half *O, const lt_half *dO, const float *LSE,
                 lt_half *dQ, lt_half *dK, lt_half *dV,
