@@ -137,3 +137,48 @@ def gemm_nt(A, W):
     if A.ndim != 2 or W.ndim != 2 or A.shape[1] != W.shape[1]:
         raise ValueError("expected A [M, K] and W [N, K]")
     return A @ W.T
+
+
+def attn_probabilities(Q, K, causal: bool, scale: float):
+    """P [B,Hq,S,S] in float64: the row softmax of the scaled, optionally causally masked scores,
+    P[b,h,q,:] = softmax_k(scale * Q[b,h,q] . K[b,g,k]) with keys k > q hidden under the mask.
+    This is the probability matrix the paper's forward pass saves tile by tile for Attention
+    Backward (Section 4.1: the backward loads the saved tile P_ij).  Plain numpy, no blocking."""
+    Q, K = _f64(Q), _f64(K)
+    B, Hq, Hkv, S, D = _dims(Q, K)
+    G = Hq // Hkv
+    P = np.empty((B, Hq, S, S), dtype=np.float64)
+    hidden = np.triu(np.ones((S, S), dtype=bool), k=1) if causal else None
+    for b in range(B):
+        for h in range(Hq):
+            s = scale * (Q[b, h] @ K[b, h // G].T)
+            if causal:
+                s = np.where(hidden, -np.inf, s)
+            s = s - s.max(axis=1, keepdims=True)
+            e = np.exp(s)
+            P[b, h] = e / e.sum(axis=1, keepdims=True)
+    return P
+
+
+def attn_bwd_from_p(P, Q, K, V, dO, scale: float):
+    """(dQ, dK, dV) in float64 from a given probability matrix P [B,Hq,S,S], step by step as the
+    paper's Attention Backward states them (Section 4.1, Algorithm 1): GV = P^T GO, GP = GO V^T,
+    GS = P * (GP - rowsum(P * GP)) (the softmax backward), GQ = scale * GS K, GK = scale * GS^T Q;
+    the kv head of a group receives the sum over the group's query heads.  P is used as given (a
+    mask is already inside it as zeros)."""
+    P, Q, K, V, dO = _f64(P), _f64(Q), _f64(K), _f64(V), _f64(dO)
+    B, Hq, Hkv, S, D = _dims(Q, K)
+    G = Hq // Hkv
+    dQ = np.zeros_like(Q)
+    dK = np.zeros_like(K)
+    dV = np.zeros_like(K)
+    for b in range(B):
+        for h in range(Hq):
+            g = h // G
+            p = P[b, h]
+            dV[b, g] += p.T @ dO[b, h]
+            dP = dO[b, h] @ V[b, g].T
+            dS = p * (dP - (p * dP).sum(axis=1, keepdims=True))
+            dQ[b, h] = scale * (dS @ K[b, g])
+            dK[b, g] += scale * (dS.T @ Q[b, h])
+    return dQ, dK, dV

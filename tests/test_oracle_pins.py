@@ -395,3 +395,70 @@ def test_gemm_oracle_against_triple_loop_and_special_cases(oracle):
     np.testing.assert_allclose(oracle.gemm_nt(A + 2 * A2, W), oracle.gemm_nt(A, W) + 2 * oracle.gemm_nt(A2, W), rtol=1e-12)
     with pytest.raises(ValueError):
         oracle.gemm_nt(A, rng.standard_normal((N, K + 1)))
+
+
+# ---------------------------------------------------------------- saved-P route (Section 4.1)
+
+def test_probabilities_hand_worked_example_and_invariants(oracle):
+    # the two-key worked example: row 0 sees key 0 only, row 1 has P = (1/4, 3/4)
+    Q = np.array([1.0, 1.0]).reshape(1, 1, 2, 1)
+    K = np.array([0.0, np.log(3.0)]).reshape(1, 1, 2, 1)
+    P = oracle.attn_probabilities(Q, K, True, 1.0)
+    np.testing.assert_allclose(P[0, 0], [[1.0, 0.0], [0.25, 0.75]], rtol=1e-15, atol=0)
+    # unmasked, the first row sees both keys: (1/4, 3/4) as well, since Q_0 = Q_1
+    P = oracle.attn_probabilities(Q, K, False, 1.0)
+    np.testing.assert_allclose(P[0, 0], [[0.25, 0.75], [0.25, 0.75]], rtol=1e-15, atol=0)
+    # random GQA case: rows sum to one, the mask is exact zeros, and P agrees with the C forward
+    # oracle through both of its outputs: P V = O and P = exp(scale * s - LSE)
+    Q, K, V = rnd((2, 4, 37, 8), 1), rnd((2, 2, 37, 8), 2), rnd((2, 2, 37, 8), 3)
+    for causal in (False, True):
+        P = oracle.attn_probabilities(Q, K, causal, 0.3)
+        O, LSE = oracle.attn_fwd(Q, K, V, causal, 0.3)
+        np.testing.assert_allclose(P.sum(-1), 1.0, rtol=1e-13)
+        if causal:
+            assert np.all(P[..., np.triu_indices(37, 1)[0], np.triu_indices(37, 1)[1]] == 0.0)
+        for h in range(4):
+            np.testing.assert_allclose(P[:, h] @ V[:, h // 2], O[:, h], rtol=1e-12, atol=1e-13)
+            s = 0.3 * np.einsum("bqd,bkd->bqk", Q[:, h], K[:, h // 2])
+            ref = np.exp(s - LSE[:, h][..., None])
+            if causal:
+                ref = np.tril(ref)
+            np.testing.assert_allclose(P[:, h], ref, rtol=1e-12, atol=1e-15)
+
+
+def test_backward_from_p_hand_worked_example(oracle):
+    vals = {}
+    for line in (GOLDEN / "two_key_worked_example.txt").read_text().splitlines():
+        if line and not line.startswith("#"):
+            name, *nums = line.split()
+            vals[name] = np.array([float(x) for x in nums])
+    Q = np.array([1.0, 1.0]).reshape(1, 1, 2, 1)
+    K = np.array([0.0, np.log(3.0)]).reshape(1, 1, 2, 1)
+    V = np.array([1.0, 5.0]).reshape(1, 1, 2, 1)
+    dO = np.ones((1, 1, 2, 1))
+    P = np.array([[1.0, 0.0], [0.25, 0.75]]).reshape(1, 1, 2, 2)  # typed in, not computed
+    dQ, dK, dV = oracle.attn_bwd_from_p(P, Q, K, V, dO, 1.0)
+    for name, got in (("dQ", dQ), ("dK", dK), ("dV", dV)):
+        np.testing.assert_allclose(got.reshape(-1), vals[name], rtol=1e-14, atol=1e-15, err_msg=name)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_backward_from_p_agrees_with_recompute_oracle_and_autograd(oracle, causal):
+    # with the exact P the saved-P route must give the gradients of the recompute route (the C
+    # oracle, pinned above by finite differences) and of torch's fp64 autograd through an explicit
+    # softmax; asymmetric shapes and distinct scale catch transposed operands and a dropped scale
+    B, Hq, Hkv, S, D, scale = 2, 6, 2, 29, 5, 0.37
+    Q, K, V, dO = rnd((B, Hq, S, D), 11), rnd((B, Hkv, S, D), 12), rnd((B, Hkv, S, D), 13), rnd((B, Hq, S, D), 14)
+    P = oracle.attn_probabilities(Q, K, causal, scale)
+    got = oracle.attn_bwd_from_p(P, Q, K, V, dO, scale)
+    ref = oracle.attn_bwd(Q, K, V, dO, causal, scale)
+    for name, g, r in zip(("dQ", "dK", "dV"), got, ref):
+        np.testing.assert_allclose(g, r, rtol=1e-10, atol=1e-12, err_msg=name)
+    tq, tk, tv = (torch.tensor(x, dtype=torch.float64, requires_grad=True) for x in (Q, K, V))
+    s = scale * torch.einsum("bhqd,bhkd->bhqk", tq, tk.repeat_interleave(Hq // Hkv, dim=1))
+    if causal:
+        s = s.masked_fill(torch.triu(torch.ones(S, S, dtype=torch.bool), 1), float("-inf"))
+    o = torch.softmax(s, -1) @ tv.repeat_interleave(Hq // Hkv, dim=1)
+    (o * torch.tensor(dO)).sum().backward()
+    for name, g, r in zip(("dQ", "dK", "dV"), got, (tq.grad, tk.grad, tv.grad)):
+        np.testing.assert_allclose(g, r.numpy(), rtol=1e-10, atol=1e-12, err_msg=name)
