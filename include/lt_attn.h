@@ -173,6 +173,36 @@ int lt_attn_bwd_bf16(const lt_bf16 *Q, const lt_bf16 *K, const lt_bf16 *V,
                      int B, int Hq, int Hkv, int S, int D, int causal, float scale,
                      void *workspace, size_t workspace_bytes, lt_stream_t stream);
 
+/* Attention Backward with the forward pass's saved probabilities (Section 4.1: the paper's backward
+ * loads the probability tile P_ij the forward saved, where lt_attn_bwd recomputes it from LSE).
+ *
+ * lt_attn_save_p writes that forward state from Q, K and the forward's LSE: P = exp(scale*Q K^T - LSE)
+ * rounded to fp16, stored as transposed tiles.  Tile (b, h, j, i) - key tile j, query tile i of query
+ * head h, tiles of 128 rows, nT = ceil(S/128) - is a 32 KB block at tile index ((b*Hq + h)*nT + j)*nT + i
+ * of `P`; inside it, element (key, query) sits at fp16 offset (query/8)*1024 + key*8 + query%8 (sixteen
+ * blocks of eight query columns, each [128 keys][8 queries], so that a warp holding consecutive key
+ * rows moves 512 contiguous bytes per access).  `P` holds lt_attn_p_store_bytes() bytes
+ * (B*Hq*nT*nT*32768; 0 for an unsupported shape) and is 256-byte aligned.  Entries hidden by the
+ * causal mask or past the end of the sequence are zero; with causal != 0, tiles with i < j are not
+ * written and never read.  Q, K, LSE as for lt_attn_bwd (contiguous [B,H,S,D], fp16); `workspace` needs
+ * only the 256-byte status block.  One kernel launch.
+ *
+ * lt_attn_bwd_saved_p computes dQ, dK, dV as lt_attn_bwd does, with `P` (the store above, same shape
+ * arguments and mask) in place of LSE: the main kernel issues no S = Q K^T product and no exponentials;
+ * it reads each tile of P once (32 KB per tile pair, B*Hq*nT*(nT+1)/2 tile pairs under a causal mask).
+ * Contiguous fp16 tensors only; workspace of lt_attn_bwd_workspace_bytes() bytes; three launches; status
+ * and error behaviour as lt_attn_bwd.  P carries fp16 rounding (and flushes probabilities below 2^-24
+ * to zero), which the recompute path does not, so its gradients are slightly less accurate. */
+size_t lt_attn_p_store_bytes(int B, int Hq, int Hkv, int S, int D);
+int lt_attn_save_p(const lt_half *Q, const lt_half *K, const float *LSE, lt_half *P,
+                   int B, int Hq, int Hkv, int S, int D, int causal, float scale,
+                   void *workspace, size_t workspace_bytes, lt_stream_t stream);
+int lt_attn_bwd_saved_p(const lt_half *Q, const lt_half *K, const lt_half *V,
+                        const lt_half *O, const lt_half *dO, const lt_half *P,
+                        lt_half *dQ, lt_half *dK, lt_half *dV,
+                        int B, int Hq, int Hkv, int S, int D, int causal, float scale,
+                        void *workspace, size_t workspace_bytes, lt_stream_t stream);
+
 /* FP16 GEMM, the linear-layer primitive of the paper's backend (Section 4.1, "FP16 GEMM assembly
  * pipeline"; its profiled shapes are in Section 6.6):  C[M,N] = A[M,K] W[N,K]^T.
  *   in : A [M,K] fp16 row-major (activations), W [N,K] fp16 row-major (a linear layer's weight as stored)

@@ -24,7 +24,8 @@ LT_ERR_DEVICE_TIMEOUT = 5
 EXPORTS = (
     "lt_attn_fwd_workspace_bytes", "lt_attn_bwd_workspace_bytes", "lt_attn_fwd", "lt_attn_bwd",
     "lt_attn_bwd_profiled", "lt_attn_bwd_noalloc", "lt_attn_fwd_strided", "lt_attn_bwd_strided",
-    "lt_attn_fwd_bf16", "lt_attn_bwd_bf16", "lt_gemm_f16", "lt_gemm_bf16", "lt_gemm_f16_workspace_bytes",
+    "lt_attn_fwd_bf16", "lt_attn_bwd_bf16", "lt_attn_p_store_bytes", "lt_attn_save_p", "lt_attn_bwd_saved_p",
+    "lt_gemm_f16", "lt_gemm_bf16", "lt_gemm_f16_workspace_bytes",
     "lt_attn_host_arena_bytes", "lt_attn_fwd_bwd_host", "lt_attn_check_status", "lt_status_string",
     "lt_last_cuda_error", "lt_attn_bwd_num_launches", "lt_attn_fwd_num_launches", "lt_dbg_tile_gemm",
     "lt_dbg_wait_timeout",
@@ -75,6 +76,12 @@ def _load() -> ctypes.CDLL:
     lib.lt_attn_fwd_bf16.restype = i
     lib.lt_attn_bwd_bf16.argtypes = lib.lt_attn_bwd_strided.argtypes
     lib.lt_attn_bwd_bf16.restype = i
+    lib.lt_attn_p_store_bytes.argtypes = [i] * 5
+    lib.lt_attn_p_store_bytes.restype = sz
+    lib.lt_attn_save_p.argtypes = [vp] * 4 + [i] * 6 + [f, vp, sz, vp]
+    lib.lt_attn_save_p.restype = i
+    lib.lt_attn_bwd_saved_p.argtypes = [vp] * 9 + [i] * 6 + [f, vp, sz, vp]
+    lib.lt_attn_bwd_saved_p.restype = i
     lib.lt_gemm_f16_workspace_bytes.argtypes = []
     lib.lt_gemm_f16_workspace_bytes.restype = sz
     lib.lt_gemm_f16.argtypes = [vp] * 3 + [i] * 3 + [vp, sz, vp]
@@ -181,6 +188,37 @@ def lt_attn_bwd(Q, K, V, O, dO, LSE, dQ, dK, dV, causal, scale, workspace, strea
                           workspace.numel() * workspace.element_size(), _stream_ptr(stream))
     if rc != LT_OK:
         raise LtError("lt_attn_bwd", rc)
+
+
+def lt_attn_p_store_bytes(B: int, Hq: int, Hkv: int, S: int, D: int) -> int:
+    """Bytes of the saved-probability store of lt_attn_save_p (0 for an unsupported shape)."""
+    return int(_lib.lt_attn_p_store_bytes(B, Hq, Hkv, S, D))
+
+
+def lt_attn_save_p(Q, K, LSE, P, causal, scale, workspace, stream=None) -> None:
+    """Write the forward's probability tiles (fp16, transposed 128 x 128 tiles) into ``P``, a device
+    buffer of at least lt_attn_p_store_bytes() bytes; asynchronous on ``stream``."""
+    _check_layout(Q, K, LSE, P)
+    B, Hq, Hkv, S, D = _dims(Q, K)
+    if P.numel() * P.element_size() < lt_attn_p_store_bytes(B, Hq, Hkv, S, D):
+        raise ValueError("P is smaller than lt_attn_p_store_bytes()")
+    rc = _lib.lt_attn_save_p(_ptr(Q), _ptr(K), _ptr(LSE), _ptr(P), B, Hq, Hkv, S, D, int(bool(causal)), float(scale),
+                             _ptr(workspace), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    if rc != LT_OK:
+        raise LtError("lt_attn_save_p", rc)
+
+
+def lt_attn_bwd_saved_p(Q, K, V, O, dO, P, dQ, dK, dV, causal, scale, workspace, stream=None) -> None:
+    """lt_attn_bwd with the saved probability tiles ``P`` of lt_attn_save_p in place of LSE."""
+    _check_layout(Q, K, V, O, dO, P, dQ, dK, dV)
+    B, Hq, Hkv, S, D = _dims(Q, K)
+    if P.numel() * P.element_size() < lt_attn_p_store_bytes(B, Hq, Hkv, S, D):
+        raise ValueError("P is smaller than lt_attn_p_store_bytes()")
+    rc = _lib.lt_attn_bwd_saved_p(_ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(dO), _ptr(P), _ptr(dQ), _ptr(dK),
+                                  _ptr(dV), B, Hq, Hkv, S, D, int(bool(causal)), float(scale), _ptr(workspace),
+                                  workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    if rc != LT_OK:
+        raise LtError("lt_attn_bwd_saved_p", rc)
 
 
 def _strides_of(t: torch.Tensor) -> TensorStrides:

@@ -101,7 +101,7 @@ bwd_preprocess_kernel(const __half *__restrict__ dO, const __half *__restrict__ 
             if (valid) {
                 a[u] = __ldcs(reinterpret_cast<const uint4 *>(dO + src_do) + sub);
                 b[u] = __ldcs(reinterpret_cast<const uint4 *>(O + src_o) + sub);
-                if (sub == 0) l[u] = __ldg(lse + src_lse);
+                if (sub == 0 && lse) l[u] = __ldg(lse + src_lse);  // (no LSE in the saved-P variant)
             }
             if (row < n_rows) {
                 // the zero fill does not depend on the loads: issue it while they are in flight
@@ -389,7 +389,19 @@ __device__ __forceinline__ BwdQTile bwd_q_tile(const BwdParams &p, const BwdItem
     return q;
 }
 
-template <int D, bool kBf16, bool kSplit>
+// The saved P^T tile (128 keys x 128 queries, fp16, 32 KB) of key tile w.j and query tile qt.
+__device__ __forceinline__ const __half *saved_p_tile(const BwdParams &p, const BwdItem &w, const BwdQTile &qt) {
+    const long long n_tiles = p.S_pad / kTileRows;
+    const long long tile = ((static_cast<long long>(qt.b) * p.Hq + qt.h) * n_tiles + w.j) * n_tiles + qt.s0 / kTileRows;
+    return reinterpret_cast<const __half *>(p.lse_ext) + tile * (kTileRows * kTileRows);
+}
+
+// kSavedP: the variant that loads the probability tiles a forward pass saved (lt_attn_save_p's store)
+// instead of recomputing them.  It issues no S product; the producer asks for each P^T tile to be
+// brought into L2 one iteration ahead and every softmax thread reads its own 128 bytes of the tile
+// straight into registers.  BwdParams::lse_ext, which this variant does not need, carries the
+// store's address (the parameter block keeps its size).
+template <int D, bool kBf16, bool kSplit, bool kSavedP = false>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
@@ -492,11 +504,14 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     const int s = it & 1, k = it >> 1;
                     const BwdQTile qt = bwd_q_tile(p, w, n);
                     if (k >= 1 && !(ok = LT_WAIT(&sm.bar_q_empty[s], (k - 1) & 1, kWaitStageEmpty))) break;
-                    mbar_arrive_expect_tx(&sm.bar_q_full[s], kTileBytes + kExtBytes);
+                    mbar_arrive_expect_tx(&sm.bar_q_full[s], kSavedP ? kTileBytes : kTileBytes + kExtBytes);
 #pragma unroll
                     for (int x = 0; x < kBoxes; ++x)
                         tma_load_4d(sm.q[s] + x * kBoxBytesBwd, &map_q, &sm.bar_q_full[s], x * 64, qt.s0, qt.h, qt.b);
-                    bulk_load_1d(sm.ext_q[s], p.lse_ext + qt.padded_row0, kExtBytes, &sm.bar_q_full[s]);
+                    if constexpr (kSavedP)
+                        bulk_prefetch_l2(saved_p_tile(p, w, qt), kTileRows * kTileRows * 2);
+                    else
+                        bulk_load_1d(sm.ext_q[s], p.lse_ext + qt.padded_row0, kExtBytes, &sm.bar_q_full[s]);
                     last_q = it;
                     if (it >= 1 && !(ok = LT_WAIT(&sm.bar_do_empty, (it - 1) & 1, kWaitDoEmpty))) break;
                     mbar_arrive_expect_tx(&sm.bar_do_full, kTileBytes + kExtBytes);
@@ -592,7 +607,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                      LT_WAIT(&sm.bar_q_full[it & 1], (it >> 1) & 1, kWaitStageFull);
                 if (!ok) break;
                 tc_fence_after_sync();
-                issue_s(it);
+                if constexpr (!kSavedP) issue_s(it);
                 for (int n = 0; n < w.n_iter && ok; ++n, ++it) {
                     const int s = it & 1;
                     const uint64_t dQ_mn = dQ_mn0 + s * kQStageStep;
@@ -620,7 +635,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     // the next S^T overwrites P'^T; the tensor pipe executes in issue order
                     if (n + 1 < w.n_iter) {
                         if (!(ok = LT_WAIT(&sm.bar_q_full[(it + 1) & 1], ((it + 1) >> 1) & 1, kWaitStageFull))) break;
-                        issue_s(it + 1);
+                        if constexpr (!kSavedP) issue_s(it + 1);
                     }
                     if (!(ok = LT_WAIT(&sm.bar_ds_ready, it & 1, kWaitDsReady))) break;
                     tc_fence_after_sync();
@@ -666,7 +681,38 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         int it = 0, ic = 0;
         LT_TRACE_BEGIN();
 
+        // saved-P variant: this thread's 64 saved probabilities of the current tile pair (ph) and of the
+        // next one (pn, in flight while dS of the current pair is formed), as packed fp16 pairs
+        uint32_t ph[32], pn[32];
+        auto load_saved_p = [&](const BwdItem &w, int n, uint32_t *dst) {
+            // the store keeps a tile as sixteen blocks of eight query columns, each [128 keys][8 queries]:
+            // the 32 lanes of a warp (consecutive key rows) read 512 contiguous bytes per load
+            const uint4 *src = reinterpret_cast<const uint4 *>(saved_p_tile(p, w, bwd_q_tile(p, w, n))) + (cbase / 8) * kTileRows + row;
+#pragma unroll
+            for (int v = 0; v < 8; ++v) {
+                const uint4 u = ld_nc_v4(src + v * kTileRows);
+                dst[4 * v] = u.x; dst[4 * v + 1] = u.y; dst[4 * v + 2] = u.z; dst[4 * v + 3] = u.w;
+            }
+        };
         auto compute_p = [&](const BwdItem &w, int n, int t) -> bool {
+            if constexpr (kSavedP) {
+                // P'^T of the previous pair must have been read by its dV product before it is replaced
+                if (t > 0 && !LT_WAIT(&sm.bar_do_empty, (t - 1) & 1, kWaitDoEmpty)) return false;
+                tc_fence_after_sync();
+                const uint32_t mult = pack_half2(exp2f(p_scale_log2), exp2f(p_scale_log2));  // 2^c <= 2^14
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t out[16];
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) out[e] = hmul2_bits(ph[c * 16 + e], mult);
+                    tmem_st16(tmem + lane_base + kColS + cbase + c * 16, out);
+                }
+                tmem_wait_st();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.bar_p_ready);
+                return true;
+            }
             if (!LT_WAIT(&sm.bar_s_full, t & 1, kWaitSFull)) return false;
             tc_fence_after_sync();
             LT_TRACE_MARK(tp0);
@@ -759,13 +805,17 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     mbar_arrive(&sm.bar_scale_ready);  // the reduction warps read it
                 }
             }
+            if constexpr (kSavedP) load_saved_p(w, 0, ph);
             ok = compute_p(w, 0, it);
             for (int n = 0; n < w.n_iter && ok; ++n, ++it) {
+                if constexpr (kSavedP)
+                    if (n + 1 < w.n_iter) load_saved_p(w, n + 1, pn);
                 if (!(ok = LT_WAIT(&sm.bar_dp_full, it & 1, kWaitDpFull))) break;
                 tc_fence_after_sync();
                 // the previous dS^T tile must have been consumed by the dQ product before it is overwritten
                 if (it > 0 && !(ok = LT_WAIT(&sm.bar_ds_free, (it - 1) & 1, kWaitDsFree))) break;
                 LT_TRACE_MARK(td0);
+                const float saved_mult = kSavedP ? exp2f(p_scale_log2) : 0.f;
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
                     uint32_t dp[32];
@@ -777,9 +827,16 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     // memory (operand of dK).
                     uint32_t o[16];
 #pragma unroll
-                    for (int e = 0; e < 16; ++e)
-                        o[e] = pack2<kBf16>(__uint_as_float(pv[c * 32 + 2 * e]) * __uint_as_float(dp[2 * e]),
-                                          __uint_as_float(pv[c * 32 + 2 * e + 1]) * __uint_as_float(dp[2 * e + 1]));
+                    for (int e = 0; e < 16; ++e) {
+                        if constexpr (kSavedP) {
+                            const float2 f = unpack2<false>(ph[c * 16 + e]);
+                            o[e] = pack2<kBf16>(f.x * saved_mult * __uint_as_float(dp[2 * e]),
+                                                f.y * saved_mult * __uint_as_float(dp[2 * e + 1]));
+                        } else {
+                            o[e] = pack2<kBf16>(__uint_as_float(pv[c * 32 + 2 * e]) * __uint_as_float(dp[2 * e]),
+                                                __uint_as_float(pv[c * 32 + 2 * e + 1]) * __uint_as_float(dp[2 * e + 1]));
+                        }
+                    }
 #pragma unroll
                     for (int v4 = 0; v4 < 4; ++v4)
                         *reinterpret_cast<uint4 *>(ds_tile + swz128_offset(row, c * 32 + v4 * 8)) =
@@ -794,6 +851,10 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sm.bar_ds_ready);
                 LT_TRACE_SINCE(14, td0);
+                if constexpr (kSavedP) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) ph[e] = pn[e];
+                }
                 if (n + 1 < w.n_iter) ok = compute_p(w, n + 1, it + 1);
             }
 
@@ -1034,7 +1095,8 @@ template <int D, bool kBf16>
 static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, const lt_half *O, const lt_half *dO,
                       const float *LSE, lt_half *dQ, lt_half *dK, lt_half *dV, const lt_attn_layout &lay, int B,
                       int Hq, int Hkv, int S, int causal, float scale, void *workspace, cudaStream_t stream,
-                      cudaEvent_t ev_main_begin, cudaEvent_t ev_main_end) {
+                      cudaEvent_t ev_main_begin, cudaEvent_t ev_main_end, const lt_half *saved_p = nullptr) {
+    // saved_p: the probability tiles of lt_attn_save_p; LSE is then not needed (fp16, whole groups only)
     const int S_pad = static_cast<int>(padded_rows(S));
     // fast addressing in the two streaming kernels when nothing is padded or strided
     auto is_contig = [&](const lt_tensor_strides &st, int H) {
@@ -1050,7 +1112,7 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
     uint4 *delta_ext = reinterpret_cast<uint4 *>(ws + kStatusBytes);
     uint4 *lse_ext = reinterpret_cast<uint4 *>(ws + kStatusBytes + ext_bytes);
     float *dq_acc = reinterpret_cast<float *>(ws + kStatusBytes + 2 * ext_bytes);
-    const int hpi = heads_per_item(B, Hq, Hkv, S, causal);
+    const int hpi = saved_p ? Hq / Hkv : heads_per_item(B, Hq, Hkv, S, causal);
     const int parts = (Hq / Hkv + hpi - 1) / hpi;
     const size_t kv_floats = static_cast<size_t>(B) * Hkv * S_pad * D;
     float *dk_acc = nullptr, *dv_acc = nullptr;
@@ -1087,7 +1149,7 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
     if (e != cudaSuccess) return record_cuda_error("bwd_preprocess_kernel launch", e);
 
     BwdParams prm;
-    prm.lse_ext = lse_ext;
+    prm.lse_ext = saved_p ? reinterpret_cast<const uint4 *>(saved_p) : lse_ext;
     prm.delta_ext = delta_ext;
     prm.dq_acc = dq_acc;
     prm.dK = reinterpret_cast<__half *>(dK);
@@ -1120,6 +1182,8 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
     }
     const size_t smem = sizeof(BwdSmem<D>);
     auto main_kernel = parts > 1 ? bwd_main_kernel<D, kBf16, true> : bwd_main_kernel<D, kBf16, false>;
+    if constexpr (!kBf16)
+        if (saved_p) main_kernel = bwd_main_kernel<D, false, false, true>;
     e = cudaFuncSetAttribute(main_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return record_cuda_error("cudaFuncSetAttribute(bwd_main)", e);
     const int n_items = B * Hkv * (S_pad / kTileRows) * parts;
@@ -1218,6 +1282,28 @@ static int bwd_entry(const lt_half *Q, const lt_half *K, const lt_half *V, const
                                      stream, main_begin, main_end);
     return launch_bwd<128, false>(Q, K, V, O, dO, LSE, dQ, dK, dV, lay, B, Hq, Hkv, S, causal, scale, workspace,
                                   stream, main_begin, main_end);
+}
+
+int lt_attn_bwd_saved_p(const lt_half *Q, const lt_half *K, const lt_half *V, const lt_half *O, const lt_half *dO,
+                        const lt_half *P, lt_half *dQ, lt_half *dK, lt_half *dV, int B, int Hq, int Hkv, int S, int D,
+                        int causal, float scale, void *workspace, size_t workspace_bytes, lt_stream_t stream) {
+    using namespace lt;
+    if (!Q || !K || !V || !O || !dO || !P || !dQ || !dK || !dV) return LT_ERR_INVALID_ARG;
+    int rc = check_shape(B, Hq, Hkv, S, D, scale);
+    if (rc != LT_OK) return rc;
+    const void *ptrs[] = {Q, K, V, O, dO, dQ, dK, dV};
+    for (const void *ptr : ptrs)
+        if (!aligned16(ptr)) return LT_ERR_UNSUPPORTED;
+    if (!aligned256(P)) return LT_ERR_UNSUPPORTED;
+    if (!workspace || !aligned256(workspace) || workspace_bytes < lt_attn_bwd_workspace_bytes(B, Hq, Hkv, S, D))
+        return LT_ERR_WORKSPACE;
+    if ((rc = check_device()) != LT_OK) return rc;
+    const lt_attn_layout lay = contiguous_layout(Hq, Hkv, S, D);
+    if (D == 64)
+        return launch_bwd<64, false>(Q, K, V, O, dO, nullptr, dQ, dK, dV, lay, B, Hq, Hkv, S, causal, scale, workspace,
+                                     static_cast<cudaStream_t>(stream), nullptr, nullptr, P);
+    return launch_bwd<128, false>(Q, K, V, O, dO, nullptr, dQ, dK, dV, lay, B, Hq, Hkv, S, causal, scale, workspace,
+                                  static_cast<cudaStream_t>(stream), nullptr, nullptr, P);
 }
 
 int lt_attn_bwd_profiled(const lt_half *Q, const lt_half *K, const lt_half *V, const lt_half *O, const lt_half *dO,

@@ -415,6 +415,23 @@ __device__ __forceinline__ void red_add_v4(float *addr, float a, float b, float 
                  : "memory");
 }
 __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) { return pack2<false>(lo, hi); }
+// product of two packed fp16 pairs, element by element
+__device__ __forceinline__ uint32_t hmul2_bits(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("mul.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+// 16-byte read-only global load that does not allocate in L1 (data read once)
+__device__ __forceinline__ uint4 ld_nc_v4(const uint4 *ptr) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(ptr));
+    return v;
+}
+// ask for `bytes` (a multiple of 16) of global memory at a 16-byte aligned address to be brought into L2
+__device__ __forceinline__ void bulk_prefetch_l2(const void *gptr, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(gptr), "r"(bytes) : "memory");
+}
 
 // Byte offset of element (row, col) inside one swizzled tile of 64 fp16 columns
 // (rows of 128 bytes, 16-byte chunks XORed with row % 8), the layout TMA's 128B swizzle

@@ -149,3 +149,32 @@ def test_gemm_rejects_bad_arguments_without_launching(binding):
     assert call(W=0x2002) == b.LT_ERR_UNSUPPORTED    # misaligned
     assert call(ws=0) == b.LT_ERR_WORKSPACE
     assert call(ws_bytes=16) == b.LT_ERR_WORKSPACE
+
+
+def test_saved_p_entry_points_reject_bad_arguments_without_launching(binding):
+    b = binding
+    lib = b._lib
+    assert b.lt_attn_p_store_bytes(2, 4, 2, 300, 128) == 2 * 4 * 3 * 3 * 128 * 128 * 2  # ceil(300/128) = 3 tiles
+    assert b.lt_attn_p_store_bytes(1, 1, 1, 128, 64) == 32768
+    assert b.lt_attn_p_store_bytes(1, 3, 2, 128, 64) == 0      # heads do not divide
+    assert b.lt_attn_p_store_bytes(1, 2, 2, 128, 96) == 0      # unsupported head dim
+
+    def save(Q=0x1000, K=0x2000, LSE=0x3000, P=0x4000, S=128, D=128, scale=0.1, ws=0x10000, ws_bytes=256):
+        return lib.lt_attn_save_p(Q, K, LSE, P, 1, 2, 2, S, D, 1, scale, ws, ws_bytes, 0)
+
+    assert save(P=0) == b.LT_ERR_INVALID_ARG
+    assert save(S=0) == b.LT_ERR_INVALID_ARG
+    assert save(scale=0.0) == b.LT_ERR_INVALID_ARG
+    assert save(D=96) == b.LT_ERR_UNSUPPORTED
+    assert save(P=0x4010) == b.LT_ERR_UNSUPPORTED     # the store must be 256-byte aligned
+    assert save(LSE=0x3002) == b.LT_ERR_UNSUPPORTED
+    assert save(ws_bytes=16) == b.LT_ERR_WORKSPACE
+
+    def bwd(P=0x4000, ptr=0x1000, S=128, ws=0x10000, ws_bytes=16):
+        return lib.lt_attn_bwd_saved_p(ptr, ptr, ptr, ptr, ptr, P, ptr, ptr, ptr, 1, 2, 2, S, 128, 1, 0.1, ws, ws_bytes, 0)
+
+    assert bwd(P=0) == b.LT_ERR_INVALID_ARG
+    assert bwd(S=-1) == b.LT_ERR_INVALID_ARG
+    assert bwd(P=0x4020) == b.LT_ERR_UNSUPPORTED
+    assert bwd(ptr=0x1004) == b.LT_ERR_UNSUPPORTED
+    assert bwd() == b.LT_ERR_WORKSPACE                # 16 bytes of workspace: stops before any launch
