@@ -52,6 +52,8 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the timed oracle leg (profiling runs)")
     ap.add_argument("--no-gemm", action="store_true", help="skip the side measurement of the FP16 GEMM primitive")
+    ap.add_argument("--no-saved-p", action="store_true",
+                    help="skip the side measurement of the saved-probability route (lt_attn_save_p + lt_attn_bwd_saved_p)")
     ap.add_argument("--clock-sample-ms", type=int, default=600,
                     help="untimed busy period before the timed steps so nvidia-smi samples clocks under load "
                          "(0 for profiler runs)")
@@ -401,6 +403,46 @@ def run_ours(args, cfg):
     d2h = sum(t.numel() * t.element_size() for t in (hdQ, hdK, hdV))
     del hO, hL
 
+    # the saved-probability route (Section 4.1: the backward loads the forward's saved P tiles) beside
+    # the recompute route, both as back-to-back whole calls at the same moment; a side measurement
+    saved_p = None
+    store_bytes = lt.lt_attn_p_store_bytes(*dims)
+    if rank == 0 and not args.no_saved_p and 0 < store_bytes <= 8 << 30:
+        del arena
+        Pst = torch.empty(store_bytes // 2, dtype=torch.float16, device="cuda")
+        g2 = [torch.empty_like(t) for t in (dQ, dK, dV)]
+        routes = {
+            "save_p": lambda: lt.lt_attn_save_p(Q, K, LSE, Pst, cfg.causal, cfg.scale, fws, stream),
+            "bwd_saved_p": lambda: lt.lt_attn_bwd_saved_p(Q, K, V, O, dO, Pst, *g2, cfg.causal, cfg.scale, ws, stream),
+            "bwd_recompute": lambda: lt.lt_attn_bwd(Q, K, V, O, dO, LSE, dQ, dK, dV, cfg.causal, cfg.scale, ws, stream),
+        }
+        ms = {}
+        for name, fn in routes.items():
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            if lt.lt_attn_check_status(fws if name == "save_p" else ws) != lt.LT_OK:
+                raise SystemExit(name + " reported: " + lt.last_cuda_error())
+            s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n_it = max(10, min(50, args.steps))
+            s0.record()
+            for _ in range(n_it):
+                fn()
+            s1.record()
+            torch.cuda.synchronize()
+            ms[name] = s0.elapsed_time(s1) / n_it
+        n_t = (cfg.S + 127) // 128
+        pairs = cfg.B * cfg.Hq * (n_t * (n_t + 1) // 2 if cfg.causal else n_t * n_t)
+        saved_p = {"store_bytes": store_bytes, "p_bytes_read_per_backward": pairs * 32768,
+                   "save_p_ms": ms["save_p"], "bwd_saved_p_ms": ms["bwd_saved_p"],
+                   "bwd_recompute_ms": ms["bwd_recompute"],
+                   "bwd_saved_p_tflops_equiv": cfg.flops / (ms["bwd_saved_p"] * 1e-3) / 1e12,
+                   "rel_diff_vs_recompute": {n: float((a.float() - b.float()).norm() / b.float().norm())
+                                             for n, a, b in zip(("dQ", "dK", "dV"), g2, (dQ, dK, dV))},
+                   "how": "whole calls back to back (3 launches each), same inputs; tflops_equiv uses the "
+                          "recompute route's FLOP count"}
+        del Pst, g2
+
     total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], dist, "cuda")
 
     if rank == 0:
@@ -451,6 +493,8 @@ def run_ours(args, cfg):
                             "peak": peak, "peak_source": peak_kind + " bf16 burst (short loops of one kernel)",
                             "shapes": [dict(g, frac=g["tflops"] / peak) for g in gemm_lines],
                             "torch_matmul_fp16_8192_best_of_10_tflops": live_matmul_tflops}
+        if saved_p:
+            line["saved_p"] = saved_p
         if not args.no_cpu_baseline and world == 1:
             import oracle
             n_heads = max(1, min(cfg.Hq, 2 * oracle.num_threads()))
