@@ -41,6 +41,8 @@ def run_gemm(lt, A, W):
     (1, 8, 8), (100, 200, 72), (129, 257, 136), (300, 1000, 520),  # ragged in every dimension
     (384, 250, 64), (77, 36, 1024),                                # N not a multiple of 8: scalar stores
     (2048, 1024, 768),                                             # more tiles than SMs would need twice
+    (128, 40000, 128),   # one tile row: the single-CTA kernel, 157 tiles over 148 CTAs (accumulator ring reused)
+    (520, 20000, 192),   # CTA pairs: 3 x 79 tiles of 256 x 256 over 74 pairs (both accumulators reused), ragged M and N
 ])
 def test_gemm_matches_oracle(lt, oracle, M, N, K):
     A, W = make_operands(M, N, K, seed=M + N + K)
