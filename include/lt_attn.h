@@ -210,7 +210,9 @@ int lt_attn_bwd_saved_p(const lt_half *Q, const lt_half *K, const lt_half *V,
  * Any M, N >= 1; K >= 8 and a multiple of 8 (16-byte row pitch for the tile loads); otherwise
  * LT_ERR_UNSUPPORTED.  Device pointers, 16-byte aligned, owned by the caller.  `workspace` holds only
  * the 256-byte status block (lt_gemm_f16_workspace_bytes()); read it with lt_attn_check_status.
- * Enqueues one kernel on `stream`; allocates nothing; does not synchronise. */
+ * Enqueues one kernel on `stream`; allocates nothing; does not synchronise.  With more than 128 rows in A the
+ * kernel runs as clusters of two CTAs that share 256x256 output tiles (pair products); LT_GEMM_SINGLE_CTA=1 in the
+ * environment, read at the first call, keeps the single-CTA kernel. */
 size_t lt_gemm_f16_workspace_bytes(void);
 int lt_gemm_f16(const lt_half *A, const lt_half *W, lt_half *C, int M, int N, int K,
                 void *workspace, size_t workspace_bytes, lt_stream_t stream);
