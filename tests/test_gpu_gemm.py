@@ -93,3 +93,42 @@ def test_gemm_bf16_matches_oracle(lt, oracle, M, N, K):
     ref = oracle.gemm_nt(A.double().numpy(), W.double().numpy())
     # bf16 output rounding: 2^-9 per element
     assert rel_fro(C.cpu().double().numpy(), ref) <= 4e-3
+
+
+@pytest.mark.parametrize("seed", [0, 1])
+def test_gemm_random_shapes(lt, oracle, seed):
+    """Seeded sweep over ragged shapes on both kernels (one tile row: single CTA; more: CTA pairs):
+    integer operands, so every result is exact and compared bit for bit."""
+    rng = np.random.default_rng(1000 + seed)
+    for case in range(12):
+        M = int(rng.choice([1, 64, 127, 128, 129, 255, 256, 257, 384, 513, 700, 1100]))
+        N = int(rng.integers(1, 1400))
+        K = 8 * int(rng.integers(1, 90))
+        gen = torch.Generator(device="cpu")
+        gen.manual_seed(seed * 100 + case)
+        A = torch.randint(-3, 4, (M, K), generator=gen).half()
+        W = torch.randint(-2, 3, (N, K), generator=gen).half()
+        C = run_gemm(lt, A, W)
+        ref = oracle.gemm_nt(A.double().numpy(), W.double().numpy())
+        assert np.array_equal(C.double().numpy(), ref), f"case {case}: M={M} N={N} K={K}"
+
+
+def test_gemm_pair_kernel_on_two_streams(lt, oracle):
+    """Two products on two streams at once (clusters of both launches share the SMs); each has its own
+    status block and result."""
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    A1, W1 = make_operands(1024, 2048, 512, seed=21)
+    A2, W2 = make_operands(768, 1536, 1024, seed=22)
+    d = [t.cuda() for t in (A1, W1, A2, W2)]
+    C1 = torch.full((1024, 2048), float("nan"), dtype=torch.float16, device="cuda")
+    C2 = torch.full((768, 1536), float("nan"), dtype=torch.float16, device="cuda")
+    w1, w2 = lt.alloc_workspace(256), lt.alloc_workspace(256)
+    torch.cuda.synchronize()
+    for _ in range(5):
+        lt.lt_gemm_f16(d[0], d[1], C1, w1, s1)
+        lt.lt_gemm_f16(d[2], d[3], C2, w2, s2)
+    torch.cuda.synchronize()
+    assert lt.lt_attn_check_status(w1) == lt.LT_OK and lt.lt_attn_check_status(w2) == lt.LT_OK, lt.last_cuda_error()
+    for C, A, W in ((C1, A1, W1), (C2, A2, W2)):
+        ref = oracle.gemm_nt(A.double().numpy(), W.double().numpy())
+        assert rel_fro(C.cpu().double().numpy(), ref) <= GEMM_REL_FRO_TOL
