@@ -163,3 +163,38 @@ def test_saved_p_route_agrees_with_recompute_route_at_several_tiles_per_cta(lt, 
         ref = oracle.attn_bwd(sl(Q), sl(K), sl(V), sl(dO), True, cfg.scale)
         got = tuple(t[bb:bb + 1, hh:hh + 1].cpu() for t in b)
         check_grads(got, ref, f"saved-P slice ({bb},{hh})")
+
+
+@pytest.mark.parametrize("name,units", [
+    ("llama2_7b", [(0, 0), (0, 13), (0, 31)]),            # the launch bench.py's saved_p leg times
+    ("qwen25_32b_gqa", [(0, 5)]),                          # groups of five query heads per kv head
+    ("llama2_7b_s3000_ragged", [(0, 20)]),                 # ragged last tile at full width
+])
+def test_saved_p_route_on_benchmark_configurations(lt, oracle, name, units):
+    """Forward, lt_attn_save_p and lt_attn_bwd_saved_p at full size on the GPU; the (batch, kv head)
+    units in `units` -- all query heads of the group -- against the oracle."""
+    cfg = workloads.ALL_CONFIGS[name]
+    Q, K, V, dO = workloads.make_inputs(cfg)
+    Qd, Kd, Vd, dOd = (t.cuda() for t in (Q, K, V, dO))
+    O = torch.empty_like(Qd)
+    LSE = torch.empty(Q.shape[:3], dtype=torch.float32, device="cuda")
+    dims = (cfg.B, cfg.Hq, cfg.Hkv, cfg.S, cfg.D)
+    ws = lt.alloc_workspace(lt.lt_attn_bwd_workspace_bytes(*dims))
+    lt.lt_attn_fwd(Qd, Kd, Vd, O, LSE, cfg.causal, cfg.scale, ws)
+    assert lt.lt_attn_check_status(ws) == lt.LT_OK, lt.last_cuda_error()
+    P = torch.empty(lt.lt_attn_p_store_bytes(*dims) // 2, dtype=torch.float16, device="cuda")
+    lt.lt_attn_save_p(Qd, Kd, LSE, P, cfg.causal, cfg.scale, ws)
+    assert lt.lt_attn_check_status(ws) == lt.LT_OK, lt.last_cuda_error()
+    got = [torch.full_like(t, float("nan")) for t in (Qd, Kd, Vd)]
+    lt.lt_attn_bwd_saved_p(Qd, Kd, Vd, O, dOd, P, *got, cfg.causal, cfg.scale, ws)
+    assert lt.lt_attn_check_status(ws) == lt.LT_OK, lt.last_cuda_error()
+    got = [t.cpu() for t in got]
+    for t in got:
+        assert torch.isfinite(t.float()).all()
+    G = cfg.Hq // cfg.Hkv
+    for (b, g) in units:
+        hs = slice(g * G, (g + 1) * G)
+        sub_n = [t.double().numpy() for t in (Q[b:b + 1, hs], K[b:b + 1, g:g + 1], V[b:b + 1, g:g + 1], dO[b:b + 1, hs])]
+        ref = oracle.attn_bwd(*sub_n, cfg.causal, cfg.scale)
+        sub_got = (got[0][b:b + 1, hs], got[1][b:b + 1, g:g + 1], got[2][b:b + 1, g:g + 1])
+        check_grads(sub_got, ref, f"saved-P {name} unit {(b, g)}")
