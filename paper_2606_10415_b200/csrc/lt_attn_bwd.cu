@@ -25,10 +25,15 @@
 //                accumulator) and the per-item dK/dV epilogue
 // Transposed scores are used (S^T = K Q^T, dP^T = V dO^T) so that P^T, written back to
 // tensor memory as fp16, is directly the A operand of dV += P^T dO; dS^T is written both to
-// tensor memory (A operand of dK += dS^T Q) and to shared memory (operand of the dQ product).  The row terms -LSE_i/scale and -delta_i are added inside
-// the S^T and dP^T products by one extra 16-element contraction step whose operands are
-// (256, 1, 0...) and the (hi, lo, 0...) split of the term, so the softmax warps never
-// touch LSE or delta.
+// tensor memory (A operand of dK += dS^T Q) and to shared memory (operand of the dQ product).
+// The row terms -LSE_i/scale and -delta_i are added inside the S^T and dP^T products by one
+// extra 16-element contraction step whose operands are (256, 1, 0...) and the (hi, lo, 0...)
+// split of the term, so the softmax warps never touch LSE or delta.
+//
+// Instantiations of the main kernel: fp16 or bf16 operands; a variant that splits a group's query
+// heads over several work items (few, heavy items) and sums dK/dV in fp32 in the workspace; and a
+// variant that loads the probability tiles a forward pass saved (Section 4.1's own forward state,
+// written by lt_attn_save_p) instead of recomputing them.
 #include <mutex>
 #include <stdio.h>
 
