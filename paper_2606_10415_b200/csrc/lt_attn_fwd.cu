@@ -39,7 +39,7 @@ struct __align__(1024) FwdSmem {
     uint8_t k[2][kTile];   // ring of key tiles
     uint8_t v[2][kTile];   // ring of value tiles
     uint64_t bar_q[2], bar_k_full[2], bar_k_empty[2], bar_v_full[2], bar_v_empty[2];
-    uint64_t bar_s_full[2], bar_p_ready[2], bar_o_done[2], bar_done;
+    uint64_t bar_s_full[2], bar_p_ready[2], bar_p_half[2], bar_o_done[2], bar_done;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -113,6 +113,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
             mbar_init(&sm.bar_v_empty[t], 1);
             mbar_init(&sm.bar_s_full[t], 1);
             mbar_init(&sm.bar_p_ready[t], 128);
+            mbar_init(&sm.bar_p_half[t], 128);
             mbar_init(&sm.bar_o_done[t], 1);
         }
         mbar_init(&sm.bar_done, 1);
@@ -190,12 +191,15 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
                     umma_ss(tmem + kColS + t * 128, dQ0 + t * kSlotStep + koff(kk), dK0 + s * kSlotStep + koff(kk), idesc_s, kk > 0);
                 umma_commit(&sm.bar_s_full[t]);
             };
-            auto issue_pv = [&](int t, int s, bool acc) {  // O_t (+)= P_t V, P_t read from tensor memory
+            // O_t (+)= P_t V, P_t read from tensor memory; the keys of a tile in two halves of 64, so that the
+            // first half's products run while the softmax warps exponentiate the second half (quarters were
+            // measured too and lost to the extra hand-offs)
+            auto issue_pv_half = [&](int t, int s, bool acc, int half) {
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
+                for (int kk = 4 * half; kk < 4 * half + 4; ++kk)
                     umma_ts(tmem + kColO + t * D, tmem + kColS + t * 128 + kk * 8, dV0 + s * kSlotStep + roff(kk), idesc_o,
                             acc | (kk > 0));
-                umma_commit(&sm.bar_o_done[t]);
+                if (half == 1) umma_commit(&sm.bar_o_done[t]);
             };
             bool ok = mbar_wait(&sm.bar_q[0], 0, abort_flag, p.status, kWaitFwdQ) &&
                       (!has_b || mbar_wait(&sm.bar_q[1], 0, abort_flag, p.status, kWaitFwdQ)) &&
@@ -218,11 +222,14 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
                     const int j_last_t = t == 0 ? j_last0 : j_last1;
                     if (j > j_last_t) continue;
                     LT_FT(0);
+                    if (!(ok = mbar_wait(&sm.bar_p_half[t], j & 1, abort_flag, p.status, kWaitFwdP))) break;
+                    tc_fence_after_sync();
+                    issue_pv_half(t, s, j > 0, 0);
                     if (!(ok = mbar_wait(&sm.bar_p_ready[t], j & 1, abort_flag, p.status, kWaitFwdP))) break;
                     LT_FT(2 + t);
                     tc_fence_after_sync();
                     LT_FT(0);
-                    issue_pv(t, s, j > 0);
+                    issue_pv_half(t, s, j > 0, 1);
                     LT_FT(5);
                     // the second tile of the pair, when it uses this key tile, uses it last
                     const int last_user = (j <= j_last1) ? 1 : 0;
@@ -348,20 +355,29 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
                 // P = exp2(score - m_used) as fp16 over the first 64 columns of the S region
                 const float neg_m = -m_used;
 #pragma unroll
-                for (int e = 0; e < 128; ++e) {
-                    const float x = fmaf(__uint_as_float(sc[e]), scale_log2, neg_m);
-                    float pe = fast_exp2(x);
-                    if (kMasked && e > last_key) pe = 0.f;
-                    rs[e & 3] += pe;
-                    sc[e] = __float_as_uint(pe);
-                }
+                for (int half = 0; half < 2; ++half) {
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t out[16];
+                    for (int e = 64 * half; e < 64 * half + 64; ++e) {
+                        const float x = fmaf(__uint_as_float(sc[e]), scale_log2, neg_m);
+                        float pe = fast_exp2(x);
+                        if (kMasked && e > last_key) pe = 0.f;
+                        rs[e & 3] += pe;
+                        sc[e] = __float_as_uint(pe);
+                    }
 #pragma unroll
-                    for (int e = 0; e < 32; e += 2)
-                        out[e / 2] = pack2<kBf16>(__uint_as_float(sc[c * 32 + e]), __uint_as_float(sc[c * 32 + e + 1]));
-                    tmem_st16(tS + c * 16, out);
+                    for (int c = 2 * half; c < 2 * half + 2; ++c) {
+                        uint32_t out[16];
+#pragma unroll
+                        for (int e = 0; e < 32; e += 2)
+                            out[e / 2] = pack2<kBf16>(__uint_as_float(sc[c * 32 + e]), __uint_as_float(sc[c * 32 + e + 1]));
+                        tmem_st16(tS + c * 16, out);
+                    }
+                    if (half == 0) {
+                        // the first 64 keys' probabilities are in place: their products may start
+                        tmem_wait_st();
+                        tc_fence_before_sync();
+                        mbar_arrive(&sm.bar_p_half[t]);
+                    }
                 }
             };
             if (p.causal ? (j == i) : (j == n_tiles - 1 && tail_keys < kFwdTileRows)) tile_softmax(std::true_type{});
