@@ -772,22 +772,31 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             // (P' = P * 2^c, c <= 14); dV and dQ/dK undo it exactly in their epilogues.
             ok = ok && (item < 0 || LT_WAIT(&sm.bar_kv, ic & 1, kWaitKV));
             if (ok && item >= 0 && half_sel == 0) {
-                float n2 = 0.f;
+                // squared row norm of V: only a bound is needed (it picks a power of two, with a factor of two
+                // to spare), so the squares are summed in the operands' own packed precision, four
+                // independent sums.  fp16 values are scaled by 2^-4 first, so that elements up to 4080 square
+                // without overflow (beyond that the sum is inf and the most cautious factor is taken).
+                constexpr uint32_t kPre = 0x2C002C00u;   // (2^-4, 2^-4) as fp16
+                uint32_t acc2[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
                 for (int x = 0; x < kBoxes; ++x) {
                     const uint4 *src = reinterpret_cast<const uint4 *>(sm.v + x * kBoxBytesBwd + row * 128);
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
                         const uint4 u = src[(c + row) & 7];  // rotated start: conflict-free across the warp
-                        const uint32_t *h = reinterpret_cast<const uint32_t *>(&u);
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const float2 f = unpack2<kBf16>(h[e]);
-                            n2 = fmaf(f.x, f.x, n2);
-                            n2 = fmaf(f.y, f.y, n2);
-                        }
+                        acc2[0] = sq_acc2<kBf16>(kBf16 ? u.x : hmul2_bits(u.x, kPre), acc2[0]);
+                        acc2[1] = sq_acc2<kBf16>(kBf16 ? u.y : hmul2_bits(u.y, kPre), acc2[1]);
+                        acc2[2] = sq_acc2<kBf16>(kBf16 ? u.z : hmul2_bits(u.z, kPre), acc2[2]);
+                        acc2[3] = sq_acc2<kBf16>(kBf16 ? u.w : hmul2_bits(u.w, kPre), acc2[3]);
                     }
                 }
+                float n2 = 0.f;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float2 f = unpack2<kBf16>(acc2[e]);
+                    n2 += f.x + f.y;
+                }
+                n2 *= (kBf16 ? 1.0625f : 256.f * 1.0625f);  // undo the pre-scaling; head room for the packed sums' rounding
 #pragma unroll
                 for (int off = 16; off > 0; off >>= 1) n2 = fmaxf(n2, __shfl_xor_sync(0xffffffffu, n2, off));
                 if (lane == 0) sm.red[ic & 1][quad] = n2;

@@ -480,6 +480,14 @@ __device__ __forceinline__ void red_add_v4(float *addr, float a, float b, float 
                  : "memory");
 }
 __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) { return pack2<false>(lo, hi); }
+// acc + a*a on a packed pair (fp16 or bf16), element by element
+template <bool kBf16>
+__device__ __forceinline__ uint32_t sq_acc2(uint32_t a, uint32_t acc) {
+    uint32_t d;
+    if constexpr (kBf16) asm("fma.rn.bf16x2 %0, %1, %1, %2;" : "=r"(d) : "r"(a), "r"(acc));
+    else asm("fma.rn.f16x2 %0, %1, %1, %2;" : "=r"(d) : "r"(a), "r"(acc));
+    return d;
+}
 // product of two packed fp16 pairs, element by element
 __device__ __forceinline__ uint32_t hmul2_bits(uint32_t a, uint32_t b) {
     uint32_t d;

@@ -227,6 +227,39 @@ def test_gradient_magnitude_extremes(lt, oracle, do_std):
         assert rel_fro(g, r) <= REL_FRO_TOL, f"{name} at dO std {do_std}: {rel_fro(g, r):.3e}"
 
 
+@pytest.mark.parametrize("v_scale,do_std", [(1e-3, 1.0), (40.0, 1e-2), (600.0, 1e-4), (600.0, 1e-2)])
+def test_value_magnitude_extremes(lt, oracle, v_scale, do_std):
+    """The bound behind that factor uses the row norms of V, summed in packed half precision after a
+    2^-4 pre-scaling: tiny values (squares below fp16's range), outlier-sized values (elements of several
+    hundred, whose plain squares would overflow fp16) and their combination with small upstream gradients
+    must keep the relative accuracy (the tiny values come with a large upstream gradient, so that the fp16
+    outputs themselves stay representable).  D = 128 and D = 64, fp16 and bf16."""
+    for D, bf16 in ((128, False), (64, False), (128, True)):
+        cfg = workloads.custom(1, 4, 2, 300, D, True, do_std=do_std, seed=77)
+        Q, K, V, dO = workloads.make_inputs(cfg)
+        V = (V.float() * v_scale).half()
+        if bf16:
+            Q, K, V, dO = (t.float().bfloat16() for t in (Q, K, V, dO))
+        Qn, Kn, Vn, dOn = (t.double().numpy() for t in (Q, K, V, dO))
+        O_ref, LSE_ref = oracle.attn_fwd(Qn, Kn, Vn, True, cfg.scale)
+        ref = oracle.attn_bwd(Qn, Kn, Vn, dOn, True, cfg.scale)
+        O = torch.from_numpy(O_ref).to(Q.dtype)
+        LSE = torch.from_numpy(LSE_ref).float()
+        Qd, Kd, Vd, Od, dOd, Ld = (t.cuda() for t in (Q, K, V, O, dO, LSE))
+        dQ, dK, dV = torch.empty_like(Qd), torch.empty_like(Kd), torch.empty_like(Vd)
+        ws = lt.alloc_workspace(lt.lt_attn_bwd_workspace_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.S, cfg.D))
+        if bf16:
+            lt.lt_attn_bwd_bf16(Qd, Kd, Vd, Od, dOd, Ld, dQ, dK, dV, True, cfg.scale, ws)
+        else:
+            lt.lt_attn_bwd(Qd, Kd, Vd, Od, dOd, Ld, dQ, dK, dV, True, cfg.scale, ws)
+        assert lt.lt_attn_check_status(ws) == lt.LT_OK, lt.last_cuda_error()
+        tol = 2e-2 if bf16 else REL_FRO_TOL
+        for name, g, r in zip(("dQ", "dK", "dV"), (dQ, dK, dV), ref):
+            g = g.cpu().double().numpy()
+            assert np.all(np.isfinite(g)), name
+            assert rel_fro(g, r) <= tol, f"{name} D={D} bf16={bf16} V x{v_scale}, dO std {do_std}: {rel_fro(g, r):.3e}"
+
+
 def test_sharp_softmax_and_large_scores(lt, oracle):
     """Large |scores| (std 4 after scaling): rows dominated by one key, LSE far from 0, probabilities
     spanning the whole fp16 range; also exercises the forward's running-maximum updates."""
