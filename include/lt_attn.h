@@ -4,8 +4,9 @@
  * The operation is the Attention Backward of a dense decoder layer as the paper's
  * execution backend states it (Section 4.1, "Memory-resident Attention Backward",
  * Algorithm 1):  GP = GO V^T,  GS = SoftmaxBackward(P, GP),  GV = P^T GO,
- * GQ = GS K,  GK = GS^T Q, with the probability tile P as forward state.  Here P is
- * not stored by the forward: it is rebuilt tile by tile from the row log-sum-exp.
+ * GQ = GS K,  GK = GS^T Q, with the probability tile P as forward state.  By default P is
+ * not stored by the forward: lt_attn_bwd rebuilds it tile by tile from the row log-sum-exp.
+ * lt_attn_save_p and lt_attn_bwd_saved_p are the stored-P route of the paper, for comparison.
  *
  * Conventions shared by every entry point
  *   - Tensors are contiguous [B, H, S, D] with D innermost (strided views: the *_strided and
@@ -24,6 +25,11 @@
  *   - Calls only enqueue work on `stream` and return; they do not synchronise and
  *     allocate no device memory.  Two calls may overlap on the GPU only if they use
  *     different workspaces.
+ *   - Value range of the backward: dS is rounded to fp16 (bf16) after multiplication by a power of two that
+ *     each work item picks from max ||dO_row||, max |delta| and the row norms of its V tile, so gradients keep
+ *     their relative accuracy for upstream gradients and values of any usual magnitude.  fp16 V elements beyond
+ *     4080 (or non-finite inputs) make that bound infinite; the most cautious factor is then used and accuracy
+ *     drops, results stay finite where the exact ones are.
  *   - Return value: LT_OK or an lt_status error.  Errors found on the host launch
  *     nothing.  A device-side wait that gave up (a bounded spin on a barrier ran out)
  *     is recorded in the workspace and read back with lt_attn_check_status.
