@@ -470,7 +470,7 @@ def run_ours(args, cfg):
             "e2e": {"value": job_throughput(cfg.flops, world, e2e_ms * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
                     "includes": "H2D copies, lt_attn_fwd, lt_attn_bwd, D2H copies"},
-            "gpu_launches": args.steps * lt.lt_attn_bwd_num_launches(),
+            "gpu_launches": args.steps * lt.lt_attn_bwd_num_launches(*dims, cfg.causal),
             # The average launch inside the timed loop runs at sustained, power-capped clocks, so it is
             # set against the sustained GEMM figure; the same average against the burst figure and a
             # launch timed alone against the burst figure are given beside it.

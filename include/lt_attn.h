@@ -25,11 +25,10 @@
  *   - Calls only enqueue work on `stream` and return; they do not synchronise and
  *     allocate no device memory.  Two calls may overlap on the GPU only if they use
  *     different workspaces.
- *   - Value range of the backward: dS is rounded to fp16 (bf16) after multiplication by a power of two that
- *     each work item picks from max ||dO_row||, max |delta| and the row norms of its V tile, so gradients keep
- *     their relative accuracy for upstream gradients and values of any usual magnitude.  fp16 V elements beyond
- *     4080 (or non-finite inputs) make that bound infinite; the most cautious factor is then used and accuracy
- *     drops, results stay finite where the exact ones are.
+ *   - Value range of the backward: dS is rounded to fp16 (bf16) after multiplication by a power of two
+ *     picked per call from max ||dO_row||, max |delta| and max ||V_row|| (their product bounds |dS|), so
+ *     gradients keep their relative accuracy for upstream gradients and values of any usual magnitude.
+ *     Non-finite inputs make that bound infinite; the most cautious factor is then used.
  *   - Return value: LT_OK or an lt_status error.  Errors found on the host launch
  *     nothing.  A device-side wait that gave up (a bounded spin on a barrier ran out)
  *     is recorded in the workspace and read back with lt_attn_check_status.
@@ -64,7 +63,8 @@ typedef unsigned short lt_bf16;
 
 /* Bytes of caller-owned device workspace the calls below need; 0 means the shape is
  * not supported.  The workspace must be 256-byte aligned.  Layout (backward), with S_pad = S
- * rounded up to a multiple of 128: a 256-byte status block, -delta and -LSE/scale as 16-byte rows
+ * rounded up to a multiple of 128: a 256-byte status block (word 0: code of a wait that gave up;
+ * words 1, 2, 4: the three maxima above as fp32 bits; word 3: work-item counter), -delta and -LSE/scale as 16-byte rows
  * of fp16 (hi, lo, 0 x 6) with 256*hi + lo = value, [B,Hq,S_pad] rows each, an fp32 dQ accumulator
  * [B,Hq,S_pad,D], and, for the grouped-query shapes whose groups are split over work items (see
  * lt_attn_bwd_num_launches), fp32 dK and dV sums [B,Hkv,S_pad,D] each. */
@@ -126,14 +126,17 @@ int lt_attn_bwd_profiled(const lt_half *Q, const lt_half *K, const lt_half *V,
  *   - All calls on a device share the one scratch array.  Each call clears what it needs at
  *     zero itself, so an earlier call's leftovers are harmless, but two calls that overlap
  *     on the GPU (different streams) race on it: serialise them.
- *   - A device-side wait that gave up cannot be read back through this entry point, since
- *     the caller has no pointer to the scratch for lt_attn_check_status. */
+ *   - The caller has no pointer to the scratch, so a device-side wait that gave up is read back
+ *     with lt_attn_bwd_noalloc_check_status(stream): it synchronises `stream`, copies the status word
+ *     of the current device's scratch to the host (4 bytes; nothing is allocated and no pointer is
+ *     handed out) and returns what lt_attn_check_status would. */
 #define LT_ATTN_BWD_NOALLOC_MAX_SCRATCH_BYTES (18u * 1024u * 1024u)
 int lt_attn_bwd_noalloc(const lt_half *Q, const lt_half *K, const lt_half *V,
                         const lt_half *O, const lt_half *dO, const float *LSE,
                         lt_half *dQ, lt_half *dK, lt_half *dV,
                         int B, int Hq, int Hkv, int S, int D, int causal, float scale,
                         lt_stream_t stream);
+int lt_attn_bwd_noalloc_check_status(lt_stream_t stream);
 
 /* Layouts other than contiguous [B,H,S,D].  Each tensor is described by the element strides of
  * its batch, head and row (sequence position) indices; the D elements of a row are always
@@ -252,40 +255,12 @@ int lt_attn_check_status(const void *workspace, lt_stream_t stream);
 const char *lt_status_string(int status);
 const char *lt_last_cuda_error(void);
 
-/* Number of kernels one call enqueues (for launch accounting by benchmarks): the backward's
- * preprocess, main and dQ-conversion kernels (a fourth, the dK/dV conversion, only on grouped-query
- * shapes with fewer than about 1.5 key-tile work items per SM, where a group's query heads are split
- * over several items), the forward's single kernel. */
-int lt_attn_bwd_num_launches(void);
+/* Number of kernels one call enqueues for this shape (for launch accounting by benchmarks): the
+ * backward's preprocess, main and dQ-conversion kernels, plus the dK/dV conversion on grouped-query shapes
+ * with fewer than about 1.5 key-tile work items per multiprocessor, where a group's query heads are split
+ * over several items (4 instead of 3); 0 for an unsupported shape.  The forward enqueues one kernel. */
+int lt_attn_bwd_num_launches(int B, int Hq, int Hkv, int S, int D, int causal);
 int lt_attn_fwd_num_launches(void);
-
-/* Bring-up check of one tensor-core tile product, used by the tests to pin the
- * shared-memory / tensor-memory operand conventions the attention kernels rely on
- * (no counterpart in the paper; its analogue is the GEMM primitive inside Attention BP,
- * Section 4.1).  Computes C[128,128] (fp32, row-major, device) from fp16 device
- * matrices, each 128 x 128 row-major:
- *   mode 0: C = A  B^T   (A rows = M, B rows = N; both contraction-contiguous)
- *   mode 1: C = A  B     (B rows = contraction index)
- *   mode 2: C = A^T B    (A and B rows = contraction index)
- *   mode 3: C = A  B     (A staged through tensor memory instead of shared memory)
- *   mode 4: as mode 0, with the accumulator read back in the 16-lane x 256-bit
- *           arrangement that the dQ reduction uses
- *   mode 5: C = A B^T + 1000 * B[n][0] added to column n through one extra, unswizzled
- *           contraction step (the way the kernels subtract LSE and delta)
- *   mode 6: no product is read back: the first 96 columns of C receive 1000 * row + column, written
- *           to tensor memory with the two 16-lane store arrangements (64 columns as 32-bit values,
- *           32 columns in the arrangement used for packed 16-bit pairs) and read back with the
- *           32-lane arrangement; checks the register-to-element maps the forward relies on */
-int lt_dbg_tile_gemm(const lt_half *A, const lt_half *B, float *C, int mode,
-                     void *workspace, size_t workspace_bytes, lt_stream_t stream);
-
-/* Failure-path check used by the tests (no counterpart in the paper): launches one small
- * kernel whose threads wait on a barrier that nothing ever completes.  The wait is bounded
- * (about 10 ms of cycles), after which the kernel records a code in the status block of
- * `workspace` and returns normally; lt_attn_check_status then reports
- * LT_ERR_DEVICE_TIMEOUT and the CUDA context stays usable.  This is the same give-up path
- * every wait inside the attention kernels takes. */
-int lt_dbg_wait_timeout(void *workspace, size_t workspace_bytes, lt_stream_t stream);
 
 #ifdef __cplusplus
 }

@@ -27,9 +27,10 @@ EXPORTS = (
     "lt_attn_fwd_bf16", "lt_attn_bwd_bf16", "lt_attn_p_store_bytes", "lt_attn_save_p", "lt_attn_bwd_saved_p",
     "lt_gemm_f16", "lt_gemm_bf16", "lt_gemm_f16_workspace_bytes",
     "lt_attn_host_arena_bytes", "lt_attn_fwd_bwd_host", "lt_attn_check_status", "lt_status_string",
-    "lt_last_cuda_error", "lt_attn_bwd_num_launches", "lt_attn_fwd_num_launches", "lt_dbg_tile_gemm",
-    "lt_dbg_wait_timeout",
+    "lt_last_cuda_error", "lt_attn_bwd_num_launches", "lt_attn_fwd_num_launches", "lt_attn_bwd_noalloc_check_status",
 )
+# test-support entry points (include/lt_attn_debug.h)
+DEBUG_EXPORTS = ("lt_dbg_tile_gemm", "lt_dbg_wait_timeout")
 
 
 class TensorStrides(ctypes.Structure):
@@ -98,7 +99,10 @@ def _load() -> ctypes.CDLL:
     lib.lt_status_string.restype = ctypes.c_char_p
     lib.lt_last_cuda_error.argtypes = []
     lib.lt_last_cuda_error.restype = ctypes.c_char_p
+    lib.lt_attn_bwd_num_launches.argtypes = [i] * 6
     lib.lt_attn_bwd_num_launches.restype = i
+    lib.lt_attn_bwd_noalloc_check_status.argtypes = [vp]
+    lib.lt_attn_bwd_noalloc_check_status.restype = i
     lib.lt_attn_fwd_num_launches.restype = i
     lib.lt_dbg_tile_gemm.argtypes = [vp, vp, vp, i, vp, sz, vp]
     lib.lt_dbg_tile_gemm.restype = i
@@ -151,8 +155,9 @@ def lt_attn_host_arena_bytes(B, Hq, Hkv, S, D) -> int:
     return int(_lib.lt_attn_host_arena_bytes(B, Hq, Hkv, S, D))
 
 
-def lt_attn_bwd_num_launches() -> int:
-    return int(_lib.lt_attn_bwd_num_launches())
+def lt_attn_bwd_num_launches(B, Hq, Hkv, S, D, causal) -> int:
+    """Kernels one backward call enqueues for this shape (3, or 4 when groups are split over work items)."""
+    return int(_lib.lt_attn_bwd_num_launches(B, Hq, Hkv, S, D, int(bool(causal))))
 
 
 def lt_attn_fwd_num_launches() -> int:
@@ -341,6 +346,11 @@ def lt_attn_bwd_noalloc(Q, K, V, O, dO, LSE, dQ, dK, dV, causal, scale, stream=N
                                   _ptr(dV), B, Hq, Hkv, S, D, int(bool(causal)), float(scale), _stream_ptr(stream))
     if rc != LT_OK:
         raise LtError("lt_attn_bwd_noalloc", rc)
+
+
+def lt_attn_bwd_noalloc_check_status(stream=None) -> int:
+    """Status of the last lt_attn_bwd_noalloc call on the current device (synchronises ``stream``)."""
+    return int(_lib.lt_attn_bwd_noalloc_check_status(_stream_ptr(stream)))
 
 
 def lt_attn_fwd_bwd_host(Q, K, V, dO, O, LSE, dQ, dK, dV, causal, scale, arena, stream=None) -> None:

@@ -3,7 +3,7 @@
 // Three kernels per call:
 //   bwd_preprocess_kernel : delta = rowsum(dO * O); writes -delta and -LSE/scale as fp16
 //                           (hi, lo) pairs, zeroes the fp32 dQ accumulator, records
-//                           max |delta| and max ||dO_row||^2 (with the V tile they bound |dS|)
+//                           max |delta|, max ||dO_row||^2 and max ||V_row||^2 (together they bound |dS|)
 //   bwd_main_kernel       : per (batch, kv head, key tile j): loop over the group's
 //                           query heads and the visible query tiles i, recompute
 //                           P^T from LSE, and run the five tile contractions on
@@ -15,13 +15,14 @@
 // tensor memory for the whole loop, and the cross-CTA reduction falls on dQ instead.
 //
 // The main kernel is persistent (one CTA per SM claims work items, heavy ones first, from a counter)
-// and warp specialised (14 warps):
+// and warp specialised: 16 warps in four warpgroups, so that each group can resize its share of the
+// register file (the control group hands most of its registers to the other three):
 //   warp 0       TMA producer (one thread): K_j, V_j once; then a two-stage ring of Q_i and a
 //                single-buffered dO_i; the warp also owns the tensor-memory allocation
-//   warp 1       tensor-core issuer (one thread)
-//   warps 2-9    softmax / dS warps: warps 2-5 take query columns 0-63 of a tile pair,
-//                warps 6-9 columns 64-127; each thread owns one key row
-//   warps 10-13  dQ reduction (tensor memory -> shared memory -> bulk add.f32 into the fp32
+//   warp 1       tensor-core issuer (one thread); warps 2-3 only fill up the control group
+//   warps 4-11   softmax / dS warps: warps 4-7 take query columns 0-63 of a tile pair,
+//                warps 8-11 columns 64-127; each thread owns one key row
+//   warps 12-15  dQ reduction (tensor memory -> shared memory -> bulk add.f32 into the fp32
 //                accumulator) and the per-item dK/dV epilogue
 // Transposed scores are used (S^T = K Q^T, dP^T = V dO^T) so that P^T, written back to
 // tensor memory as fp16, is directly the A operand of dV += P^T dO; dS^T is written both to
@@ -50,7 +51,7 @@ constexpr float kLog2e = 1.4426950408889634f;
 enum {
     kWaitKV = 201, kWaitStageEmpty = 202, kWaitStageFull = 203, kWaitSFull = 204, kWaitPReady = 205,
     kWaitDpFull = 206, kWaitDsReady = 207, kWaitDsFree = 208, kWaitDqFull = 209, kWaitDqEmpty = 210,
-    kWaitDkvFull = 211, kWaitDoFull = 212, kWaitDoEmpty = 213, kWaitAccFree = 214, kWaitScale = 215,
+    kWaitDkvFull = 211, kWaitDoFull = 212, kWaitDoEmpty = 213, kWaitAccFree = 214,
     kWaitItem = 200, kBadSmemAlign = 220
 };
 
@@ -66,7 +67,8 @@ bwd_preprocess_kernel(const __half *__restrict__ dO, const __half *__restrict__ 
                       uint4 *__restrict__ delta_ext, uint4 *__restrict__ lse_ext, float *__restrict__ dq_acc,
                       long long n_rows, int S, int S_pad, int Hq, lt_tensor_strides do_st, lt_tensor_strides o_st,
                       int plain, float inv_scale, unsigned int *status, float4 *__restrict__ kv_acc,
-                      long long kv_acc_vec4) {
+                      long long kv_acc_vec4, const __half *__restrict__ V, long long v_rows, int Hkv,
+                      lt_tensor_strides v_st, int v_plain) {
     // `n_rows` counts rows of the padded row space (every head rounded up to S_pad rows), the
     // indexing of delta_ext, lse_ext and dq_acc; padding rows get zeros everywhere.
     grid_launch_dependents();  // the main kernel sets itself up while this kernel's last blocks run
@@ -146,26 +148,65 @@ bwd_preprocess_kernel(const __half *__restrict__ dO, const __half *__restrict__ 
             }
         }
     }
+    // largest squared row norm of V (rows of the logical [B,Hkv,S]): with the two maxima above it bounds
+    // |dS|, from which the main kernel picks the power of two that dS carries into fp16
+    // (kept as bit patterns: non-negative floats order like them, with inf above every finite value and
+    // NaN above inf, so non-finite inputs saturate the bound)
+    unsigned int max_v2 = 0u;
+    for (long long row0 = warp_global * kRowsPerTrip; row0 < v_rows; row0 += n_warps * kRowsPerTrip) {
+        uint4 a[kPreUnroll];
+#pragma unroll
+        for (int u = 0; u < kPreUnroll; ++u) {
+            const long long row = row0 + u * kRowsPerWarp + lane / kLanesPerRow;
+            a[u] = make_uint4(0u, 0u, 0u, 0u);
+            if (row < v_rows) {
+                long long src = row * D;
+                if (!v_plain) {
+                    const int bg = static_cast<int>(row / S);
+                    const int s_in = static_cast<int>(row - static_cast<long long>(bg) * S);
+                    const int bb = bg / Hkv, gg = bg - bb * Hkv;
+                    src = bb * v_st.batch + gg * v_st.head + s_in * v_st.row;
+                }
+                a[u] = __ldg(reinterpret_cast<const uint4 *>(V + src) + sub);  // (the main kernel reads V again)
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kPreUnroll; ++u) {
+            const uint32_t *ah = reinterpret_cast<const uint32_t *>(&a[u]);
+            float n2 = 0.f;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float2 x = unpack2<kBf16>(ah[e]);
+                n2 = fmaf(x.x, x.x, n2);
+                n2 = fmaf(x.y, x.y, n2);
+            }
+#pragma unroll
+            for (int off = kLanesPerRow / 2; off > 0; off >>= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, off);
+            max_v2 = max(max_v2, __float_as_uint(n2) & 0x7fffffffu);
+        }
+    }
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
         max_abs_delta = fmaxf(max_abs_delta, __shfl_xor_sync(0xffffffffu, max_abs_delta, off));
         max_norm2 = fmaxf(max_norm2, __shfl_xor_sync(0xffffffffu, max_norm2, off));
+        max_v2 = max(max_v2, __shfl_xor_sync(0xffffffffu, max_v2, off));
     }
-    // one pair of atomics per block, and only when it would raise the stored maximum: thousands of
-    // atomics on the same two words would otherwise queue up behind one another in L2
-    __shared__ float block_max[2][8];
+    // one set of atomics per block, and only when it would raise the stored maximum: thousands of
+    // atomics on the same words would otherwise queue up behind one another in L2
+    __shared__ float block_max[3][8];
     if (lane == 0) {
         block_max[0][threadIdx.x >> 5] = max_abs_delta;
         block_max[1][threadIdx.x >> 5] = max_norm2;
+        block_max[2][threadIdx.x >> 5] = __uint_as_float(max_v2);
     }
     __syncthreads();
-    if (threadIdx.x < 2) {
-        float m = 0.f;
+    if (threadIdx.x < 3) {
+        unsigned int m = 0u;
 #pragma unroll
-        for (int w = 0; w < 8; ++w) m = fmaxf(m, block_max[threadIdx.x][w]);
-        // non-negative floats order like their bit patterns; NaN/inf inputs simply saturate the bound
-        unsigned int *word = status + (threadIdx.x == 0 ? kStatusWordMaxAbsDelta : kStatusWordMaxDoNorm2);
-        if (__float_as_uint(m) > *reinterpret_cast<volatile unsigned int *>(word)) atomicMax(word, __float_as_uint(m));
+        for (int w = 0; w < 8; ++w) m = max(m, __float_as_uint(block_max[threadIdx.x][w]) & 0x7fffffffu);
+        unsigned int *word = status + (threadIdx.x == 0 ? kStatusWordMaxAbsDelta
+                                       : threadIdx.x == 1 ? kStatusWordMaxDoNorm2 : kStatusWordMaxVNorm2);
+        if (m > *reinterpret_cast<volatile unsigned int *>(word)) atomicMax(word, m);
     }
 }
 
@@ -274,13 +315,17 @@ __device__ __forceinline__ bool traced_wait(Trace &tr, uint64_t *bar, uint32_t p
 
 // ----------------------------------------------------------------------------- main kernel
 constexpr int kQStages = 2;   // Q_i ring; dO_i is single-buffered (it is dead once dV has been issued)
-constexpr int kBwdThreads = 448;  // 14 warps; 128 registers per thread
-constexpr int kComputeWarp0 = 2, kNumComputeWarps = 8;
-constexpr int kReduceWarp0 = 10, kNumReduceWarps = 4;
+constexpr int kBwdThreads = 512;  // 16 warps; 128 registers per thread at launch
+constexpr int kComputeWarp0 = 4, kNumComputeWarps = 8;
+constexpr int kReduceWarp0 = 12, kNumReduceWarps = 4;
+// registers per thread once the warpgroups have resized their shares (the SM has 64 K)
+constexpr int kRegsControl = 96, kRegsCompute = 144, kRegsReduce = 128;
+static_assert(128 * kRegsControl + kNumComputeWarps * 32 * kRegsCompute + kNumReduceWarps * 32 * kRegsReduce <= 65536,
+              "register shares exceed the register file");
 constexpr int kDqStageBufs = 3, kDqStageRows = 16;
 constexpr int kExtBytes = 2048;            // 128 rows x 16 bytes: one operand of the extra contraction step
 constexpr float kPScaleLog2Max = 14.f;     // P is kept as P * 2^c with c <= 14 so that fp16(P') <= 16384
-constexpr int kBarComputeWarps = 2, kBarReduceWarps = 1;  // named barrier ids
+constexpr int kBarReduceWarps = 1;  // named barrier id
 constexpr int kItemRing = 4;  // roles are never more than two items apart
 constexpr double kL2BatchBytes = 80.0e6;  // working set of one batch of work items (L2 holds 126 MB)
 
@@ -301,16 +346,14 @@ struct BwdSmem {
     // staging of the dQ partial for bulk reduction into global memory (D = 128 only):
     // each buffer holds 16 accumulator rows (16 query rows x 128 floats)
     float dq_stage[D == 128 ? kDqStageBufs : 1][D == 128 ? kDqStageRows * 128 : 4];
-    // per work item: K/V landed; dK/dV accumulators complete; accumulators read out; scale published
-    uint64_t bar_kv, bar_dkv_full, bar_acc_free, bar_scale_ready;
+    // per work item: K/V landed; dK/dV accumulators complete; accumulators read out
+    uint64_t bar_kv, bar_dkv_full, bar_acc_free;
     // work items are claimed from a global counter by the producer and published to the other roles
     uint64_t bar_item[kItemRing];
     int item_ring[kItemRing];
     // per (query head, query tile) iteration
     uint64_t bar_q_full[kQStages], bar_q_empty[kQStages], bar_do_full, bar_do_empty;
     uint64_t bar_s_full, bar_p_ready, bar_dp_full, bar_ds_ready, bar_ds_free, bar_dq_full, bar_dq_empty;
-    float red[2][4];       // per item parity: max squared row norm of V_j seen by each of four warps
-    float p_scale[2];      // per item parity: the exponent c of P' = P * 2^c
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -401,6 +444,21 @@ __device__ __forceinline__ const __half *saved_p_tile(const BwdParams &p, const 
     return reinterpret_cast<const __half *>(p.lse_ext) + tile * (kTileRows * kTileRows);
 }
 
+// The exponent c of the power of two that P carries (P' = P * 2^c, c <= 14), and with it dS, so that
+// dS' uses fp16's normal range without overflow when it is rounded: chosen from a bound on
+// |dS| <= |dP| + |delta| <= max ||dO_row|| * max ||V_row|| + max |delta| over the whole call (the
+// three maxima come from the preprocess kernel).  dV and dQ / dK undo the factor exactly in their
+// epilogues.  Every thread that needs c computes it once per CTA from the status block.
+__device__ __forceinline__ int bwd_p_scale_log2(const unsigned int *status) {
+    const float do2 = __uint_as_float(__ldcg(status + kStatusWordMaxDoNorm2));
+    const float v2 = __uint_as_float(__ldcg(status + kStatusWordMaxVNorm2));
+    const float dmax = __uint_as_float(__ldcg(status + kStatusWordMaxAbsDelta));
+    const float bound = sqrtf(do2) * sqrtf(v2) + dmax;
+    if (!(bound < 3.0e38f)) return -14;                           // inf/NaN inputs: outputs are non-finite anyway
+    if (!(bound > 1e-30f)) return static_cast<int>(kPScaleLog2Max);  // all-zero dO: any factor works
+    return min(static_cast<int>(kPScaleLog2Max), max(-14, ilogbf(32768.f / bound)));
+}
+
 // kSavedP: the variant that loads the probability tiles a forward pass saved (lt_attn_save_p's store)
 // instead of recomputing them.  It issues no S product; the producer asks for each P^T tile to be
 // brought into L2 one iteration ahead and every softmax thread reads its own 128 bytes of the tile
@@ -436,7 +494,6 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         mbar_init(&sm.bar_dkv_full, 1);
         mbar_init(&sm.bar_acc_free, kNumReduceWarps);
         for (int r = 0; r < kItemRing; ++r) mbar_init(&sm.bar_item[r], 1);
-        mbar_init(&sm.bar_scale_ready, 1);
         for (int s = 0; s < kQStages; ++s) {
             mbar_init(&sm.bar_q_full[s], 1);
             mbar_init(&sm.bar_q_empty[s], 1);
@@ -485,194 +542,204 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     // Every role walks the same list of work items and keeps its own running iteration count
     // `it` (over all items): each per-iteration barrier completes once per iteration, so its
     // phase parity is a function of `it`; the per-item barriers use the item count `ic`.
-    if (warp == 0) {
-        // ================================================================= TMA producer
-        if (lane == 0 && smem_ok) {
-            LT_TRACE_BEGIN();
-            bool ok = true;
-            int it = 0, ic = 0;
-            int last_q = -1, last_do = -1, kv_loads = 0;  // for the cleanup after an abandoned wait
-            // claim the next unclaimed item (heavy ones have the low numbers) and publish it to the
-            // other roles; -1 tells everybody that the list is exhausted
-            auto claim = [&](int slot_ic) -> int {
-                const unsigned int v = atomicAdd(p.status + kStatusWordItemCounter, 1u);
-                const int item = v < static_cast<unsigned int>(n_items) ? static_cast<int>(v) : -1;
-                sm.item_ring[slot_ic % kItemRing] = item;
-                mbar_arrive(&sm.bar_item[slot_ic % kItemRing]);
-                return item;
-            };
-            int item = claim(0);
-            while (item >= 0 && ok) {
-                const BwdItem w = bwd_item<kSplit>(p, item);
-                int next_item = -1;
-                for (int n = 0; n < w.n_iter && ok; ++n, ++it) {
-                    const int s = it & 1, k = it >> 1;
-                    const BwdQTile qt = bwd_q_tile(p, w, n);
-                    if (k >= 1 && !(ok = LT_WAIT(&sm.bar_q_empty[s], (k - 1) & 1, kWaitStageEmpty))) break;
-                    mbar_arrive_expect_tx(&sm.bar_q_full[s], kSavedP ? kTileBytes : kTileBytes + kExtBytes);
-#pragma unroll
-                    for (int x = 0; x < kBoxes; ++x)
-                        tma_load_4d(sm.q[s] + x * kBoxBytesBwd, &map_q, &sm.bar_q_full[s], x * 64, qt.s0, qt.h, qt.b);
-                    if constexpr (kSavedP)
-                        bulk_prefetch_l2(saved_p_tile(p, w, qt), kTileRows * kTileRows * 2);
-                    else
-                        bulk_load_1d(sm.ext_q[s], p.lse_ext + qt.padded_row0, kExtBytes, &sm.bar_q_full[s]);
-                    last_q = it;
-                    if (it >= 1 && !(ok = LT_WAIT(&sm.bar_do_empty, (it - 1) & 1, kWaitDoEmpty))) break;
-                    mbar_arrive_expect_tx(&sm.bar_do_full, kTileBytes + kExtBytes);
-#pragma unroll
-                    for (int x = 0; x < kBoxes; ++x)
-                        tma_load_4d(sm.d_o + x * kBoxBytesBwd, &map_do, &sm.bar_do_full, x * 64, qt.s0, qt.h, qt.b);
-                    bulk_load_1d(sm.ext_do, p.delta_ext + qt.padded_row0, kExtBytes, &sm.bar_do_full);
-                    last_do = it;
-                    if (n == 0) {
-                        // K_j and V_j follow the first query tile: they may only be overwritten once every
-                        // product of the previous item has completed
-                        if (ic >= 1 && !(ok = LT_WAIT(&sm.bar_dkv_full, (ic - 1) & 1, kWaitDkvFull))) break;
-                        mbar_arrive_expect_tx(&sm.bar_kv, 2 * kTileBytes);
-#pragma unroll
-                        for (int x = 0; x < kBoxes; ++x) {
-                            tma_load_4d(sm.k + x * kBoxBytesBwd, &map_k, &sm.bar_kv, x * 64, w.j * kTileRows, w.g, w.b);
-                            tma_load_4d(sm.v + x * kBoxBytesBwd, &map_v, &sm.bar_kv, x * 64, w.j * kTileRows, w.g, w.b);
-                        }
-                        ++kv_loads;
-                    }
-                    if (n == w.n_iter - 1) {
-                        // with the last query tile of this item on its way, claim the next item and ask for
-                        // its K/V tiles to be brought into L2 while this item finishes
-                        next_item = claim(ic + 1);
-                        if (next_item >= 0) {
-                            const BwdItem wn = bwd_item<kSplit>(p, next_item);
-#pragma unroll
+    if (warp < kComputeWarp0) {
+        // ================================================================= control group
+        warpgroup_regs_release<kRegsControl>();
+        if (warp == 0) {
+            // ================================================================= TMA producer
+            if (lane == 0 && smem_ok) {
+                LT_TRACE_BEGIN();
+                bool ok = true;
+                int it = 0, ic = 0;
+                int last_q = -1, last_do = -1, kv_loads = 0;  // for the cleanup after an abandoned wait
+                // claim the next unclaimed item (heavy ones have the low numbers) and publish it to the
+                // other roles; -1 tells everybody that the list is exhausted
+                auto claim = [&](int slot_ic) -> int {
+                    const unsigned int v = atomicAdd(p.status + kStatusWordItemCounter, 1u);
+                    const int item = v < static_cast<unsigned int>(n_items) ? static_cast<int>(v) : -1;
+                    sm.item_ring[slot_ic % kItemRing] = item;
+                    mbar_arrive(&sm.bar_item[slot_ic % kItemRing]);
+                    return item;
+                };
+                int item = claim(0);
+                while (item >= 0 && ok) {
+                    const BwdItem w = bwd_item<kSplit>(p, item);
+                    int next_item = -1;
+                    for (int n = 0; n < w.n_iter && ok; ++n, ++it) {
+                        const int s = it & 1, k = it >> 1;
+                        const BwdQTile qt = bwd_q_tile(p, w, n);
+                        if (k >= 1 && !(ok = LT_WAIT(&sm.bar_q_empty[s], (k - 1) & 1, kWaitStageEmpty))) break;
+                        mbar_arrive_expect_tx(&sm.bar_q_full[s], kSavedP ? kTileBytes : kTileBytes + kExtBytes);
+    #pragma unroll
+                        for (int x = 0; x < kBoxes; ++x)
+                            tma_load_4d(sm.q[s] + x * kBoxBytesBwd, &map_q, &sm.bar_q_full[s], x * 64, qt.s0, qt.h, qt.b);
+                        if constexpr (kSavedP)
+                            bulk_prefetch_l2(saved_p_tile(p, w, qt), kTileRows * kTileRows * 2);
+                        else
+                            bulk_load_1d(sm.ext_q[s], p.lse_ext + qt.padded_row0, kExtBytes, &sm.bar_q_full[s]);
+                        last_q = it;
+                        if (it >= 1 && !(ok = LT_WAIT(&sm.bar_do_empty, (it - 1) & 1, kWaitDoEmpty))) break;
+                        mbar_arrive_expect_tx(&sm.bar_do_full, kTileBytes + kExtBytes);
+    #pragma unroll
+                        for (int x = 0; x < kBoxes; ++x)
+                            tma_load_4d(sm.d_o + x * kBoxBytesBwd, &map_do, &sm.bar_do_full, x * 64, qt.s0, qt.h, qt.b);
+                        bulk_load_1d(sm.ext_do, p.delta_ext + qt.padded_row0, kExtBytes, &sm.bar_do_full);
+                        last_do = it;
+                        if (n == 0) {
+                            // K_j and V_j follow the first query tile: they may only be overwritten once every
+                            // product of the previous item has completed
+                            if (ic >= 1 && !(ok = LT_WAIT(&sm.bar_dkv_full, (ic - 1) & 1, kWaitDkvFull))) break;
+                            mbar_arrive_expect_tx(&sm.bar_kv, 2 * kTileBytes);
+    #pragma unroll
                             for (int x = 0; x < kBoxes; ++x) {
-                                tma_prefetch_l2_4d(&map_k, x * 64, wn.j * kTileRows, wn.g, wn.b);
-                                tma_prefetch_l2_4d(&map_v, x * 64, wn.j * kTileRows, wn.g, wn.b);
+                                tma_load_4d(sm.k + x * kBoxBytesBwd, &map_k, &sm.bar_kv, x * 64, w.j * kTileRows, w.g, w.b);
+                                tma_load_4d(sm.v + x * kBoxBytesBwd, &map_v, &sm.bar_kv, x * 64, w.j * kTileRows, w.g, w.b);
+                            }
+                            ++kv_loads;
+                        }
+                        if (n == w.n_iter - 1) {
+                            // with the last query tile of this item on its way, claim the next item and ask for
+                            // its K/V tiles to be brought into L2 while this item finishes
+                            next_item = claim(ic + 1);
+                            if (next_item >= 0) {
+                                const BwdItem wn = bwd_item<kSplit>(p, next_item);
+    #pragma unroll
+                                for (int x = 0; x < kBoxes; ++x) {
+                                    tma_prefetch_l2_4d(&map_k, x * 64, wn.j * kTileRows, wn.g, wn.b);
+                                    tma_prefetch_l2_4d(&map_v, x * 64, wn.j * kTileRows, wn.g, wn.b);
+                                }
                             }
                         }
                     }
+                    item = next_item;
+                    ++ic;
                 }
-                item = next_item;
-                ++ic;
+                LT_TRACE_END(kRoleProducer);
+                if (*abort_flag) {
+                    // abandoned: give this CTA's own copies a bounded time to land before shared memory is released
+                    if (kv_loads > 0)
+                        for (int t = 0; t < (1 << 16) && !mbar_try_wait(&sm.bar_kv, (kv_loads - 1) & 1); ++t) {}
+                    for (int n = max(0, last_q - 1); n <= last_q; ++n)
+                        for (int t = 0; t < (1 << 16) && !mbar_try_wait(&sm.bar_q_full[n & 1], (n >> 1) & 1); ++t) {}
+                    if (last_do >= 0)
+                        for (int t = 0; t < (1 << 16) && !mbar_try_wait(&sm.bar_do_full, last_do & 1); ++t) {}
+                }
             }
-            LT_TRACE_END(kRoleProducer);
-            if (*abort_flag) {
-                // abandoned: give this CTA's own copies a bounded time to land before shared memory is released
-                if (kv_loads > 0)
-                    for (int t = 0; t < (1 << 16) && !mbar_try_wait(&sm.bar_kv, (kv_loads - 1) & 1); ++t) {}
-                for (int n = max(0, last_q - 1); n <= last_q; ++n)
-                    for (int t = 0; t < (1 << 16) && !mbar_try_wait(&sm.bar_q_full[n & 1], (n >> 1) & 1); ++t) {}
-                if (last_do >= 0)
-                    for (int t = 0; t < (1 << 16) && !mbar_try_wait(&sm.bar_do_full, last_do & 1); ++t) {}
-            }
-        }
-        __syncwarp();
-    } else if (warp == 1) {
-        // ================================================================= tensor-core issuer
-        if (lane == 0 && smem_ok) {
-            LT_TRACE_BEGIN();
-            // Every operand descriptor is a base computed once plus a compile-time constant in its
-            // address field (bits 0-13, units of 16 bytes; shared memory stays below 256 KB, so the
-            // sum never carries out of the field): the issuing thread then spends two integer adds
-            // per product and the tensor pipe, not this thread, sets the pace.
-            const uint32_t s_zero = smem_u32(sm.ext_zero);
-            const uint64_t dK_k = desc_kmajor(smem_u32(sm.k)), dV_k = desc_kmajor(smem_u32(sm.v));
-            const uint64_t dK_mn = desc_mnmajor(smem_u32(sm.k), kBoxBytesBwd);
-            const uint64_t ddS_mn = desc_mnmajor(smem_u32(sm.ds), kBoxBytesBwd);
-            const uint64_t ddO_k = desc_kmajor(smem_u32(sm.d_o)), ddO_mn = desc_mnmajor(smem_u32(sm.d_o), kBoxBytesBwd);
-            const uint64_t dQ_k0 = desc_kmajor(smem_u32(sm.q[0])), dQ_mn0 = desc_mnmajor(smem_u32(sm.q[0]), kBoxBytesBwd);
-            constexpr uint64_t kQStageStep = static_cast<uint64_t>(Smem::kTile) >> 4;  // next Q stage
-            const uint64_t desc_ones = desc_kmajor_noswz(smem_u32(sm.ext_ones), s_zero - smem_u32(sm.ext_ones), 128);
-            const uint64_t desc_ext_do = desc_kmajor_noswz(smem_u32(sm.ext_do), s_zero - smem_u32(sm.ext_do), 128);
-            const uint64_t desc_ext_q0 = desc_kmajor_noswz(smem_u32(sm.ext_q[0]), s_zero - smem_u32(sm.ext_q[0]), 128);
-            const uint64_t desc_ext_q1 = desc_kmajor_noswz(smem_u32(sm.ext_q[1]), s_zero - smem_u32(sm.ext_q[1]), 128);
-            // address-field increments of contraction step kk: within a contraction-contiguous tile
-            // (32 bytes per step, next 64-column tile after four steps) and within a row-contracted
-            // tile (16 rows of 128 bytes per step)
-            auto koff = [](int kk) -> uint64_t { return static_cast<uint64_t>((kk >> 2) * (kBoxBytesBwd >> 4) + (kk & 3) * 2); };
-            auto roff = [](int kk) -> uint64_t { return static_cast<uint64_t>(kk * (2048 >> 4)); };
-            constexpr uint32_t idesc_s = make_idesc(128, 128, false, false, kBf16);
-            constexpr uint32_t idesc_dv = make_idesc(128, D, false, true, kBf16);
-            constexpr uint32_t idesc_dq = make_idesc(128, D == 128 ? 128 : D, true, true, kBf16);
-            auto issue_s = [&](int t) {  // S^T = K_j Q_i^T - LSE_i / scale, for running iteration t
-                const uint64_t dQ_k = dQ_k0 + (t & 1) * kQStageStep;
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk)
-                    umma_ss(tmem + kColS, dK_k + koff(kk), dQ_k + koff(kk), idesc_s, kk > 0);
-                umma_ss(tmem + kColS, desc_ones, (t & 1) ? desc_ext_q1 : desc_ext_q0, idesc_s, 1);
-                umma_commit(&sm.bar_s_full);
-            };
-            bool ok = true;
-            int it = 0, ic = 0;
-            for (;; ++ic) {
-                if (!(ok = LT_WAIT(&sm.bar_item[ic % kItemRing], (ic / kItemRing) & 1, kWaitItem))) break;
-                const int item = sm.item_ring[ic % kItemRing];
-                if (item < 0) break;
-                const BwdItem w = bwd_item<kSplit>(p, item);
-                ok = LT_WAIT(&sm.bar_kv, ic & 1, kWaitKV) &&
-                     LT_WAIT(&sm.bar_q_full[it & 1], (it >> 1) & 1, kWaitStageFull);
-                if (!ok) break;
-                tc_fence_after_sync();
-                if constexpr (!kSavedP) issue_s(it);
-                for (int n = 0; n < w.n_iter && ok; ++n, ++it) {
-                    const int s = it & 1;
-                    const uint64_t dQ_mn = dQ_mn0 + s * kQStageStep;
-                    // dP^T = V_j dO_i^T - delta_i   (its columns held the previous dQ partial until the
-                    //                                reduce warps drained it)
-                    if (!(ok = LT_WAIT(&sm.bar_do_full, it & 1, kWaitDoFull))) break;
-                    if (it > 0 && !(ok = LT_WAIT(&sm.bar_dq_empty, (it - 1) & 1, kWaitDqEmpty))) break;
-                    tc_fence_after_sync();
-#pragma unroll
+            __syncwarp();
+        } else if (warp == 1) {
+            // ================================================================= tensor-core issuer
+            if (lane == 0 && smem_ok) {
+                LT_TRACE_BEGIN();
+                // Every operand descriptor is a base computed once plus a compile-time constant in its
+                // address field (bits 0-13, units of 16 bytes; shared memory stays below 256 KB, so the
+                // sum never carries out of the field): the issuing thread then spends two integer adds
+                // per product and the tensor pipe, not this thread, sets the pace.
+                const uint32_t s_zero = smem_u32(sm.ext_zero);
+                const uint64_t dK_k = desc_kmajor(smem_u32(sm.k)), dV_k = desc_kmajor(smem_u32(sm.v));
+                const uint64_t dK_mn = desc_mnmajor(smem_u32(sm.k), kBoxBytesBwd);
+                const uint64_t ddS_mn = desc_mnmajor(smem_u32(sm.ds), kBoxBytesBwd);
+                const uint64_t ddO_k = desc_kmajor(smem_u32(sm.d_o)), ddO_mn = desc_mnmajor(smem_u32(sm.d_o), kBoxBytesBwd);
+                const uint64_t dQ_k0 = desc_kmajor(smem_u32(sm.q[0])), dQ_mn0 = desc_mnmajor(smem_u32(sm.q[0]), kBoxBytesBwd);
+                constexpr uint64_t kQStageStep = static_cast<uint64_t>(Smem::kTile) >> 4;  // next Q stage
+                const uint64_t desc_ones = desc_kmajor_noswz(smem_u32(sm.ext_ones), s_zero - smem_u32(sm.ext_ones), 128);
+                const uint64_t desc_ext_do = desc_kmajor_noswz(smem_u32(sm.ext_do), s_zero - smem_u32(sm.ext_do), 128);
+                const uint64_t desc_ext_q0 = desc_kmajor_noswz(smem_u32(sm.ext_q[0]), s_zero - smem_u32(sm.ext_q[0]), 128);
+                const uint64_t desc_ext_q1 = desc_kmajor_noswz(smem_u32(sm.ext_q[1]), s_zero - smem_u32(sm.ext_q[1]), 128);
+                // address-field increments of contraction step kk: within a contraction-contiguous tile
+                // (32 bytes per step, next 64-column tile after four steps) and within a row-contracted
+                // tile (16 rows of 128 bytes per step)
+                auto koff = [](int kk) -> uint64_t { return static_cast<uint64_t>((kk >> 2) * (kBoxBytesBwd >> 4) + (kk & 3) * 2); };
+                auto roff = [](int kk) -> uint64_t { return static_cast<uint64_t>(kk * (2048 >> 4)); };
+                constexpr uint32_t idesc_s = make_idesc(128, 128, false, false, kBf16);
+                constexpr uint32_t idesc_dv = make_idesc(128, D, false, true, kBf16);
+                constexpr uint32_t idesc_dq = make_idesc(128, D == 128 ? 128 : D, true, true, kBf16);
+                auto issue_s = [&](int t) {  // S^T = K_j Q_i^T - LSE_i / scale, for running iteration t
+                    const uint64_t dQ_k = dQ_k0 + (t & 1) * kQStageStep;
+    #pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk)
-                        umma_ss(tmem + kColdP, dV_k + koff(kk), ddO_k + koff(kk), idesc_s, kk > 0);
-                    umma_ss(tmem + kColdP, desc_ones, desc_ext_do, idesc_s, 1);
-                    umma_commit(&sm.bar_dp_full);
-                    // dV_j += P'^T dO_i   (A = P'^T from tensor memory; query columns 0-63 sit at columns
-                    //                      0-31, query columns 64-127 at columns 64-95 of the S region)
-                    if (!(ok = LT_WAIT(&sm.bar_p_ready, it & 1, kWaitPReady))) break;
-                    // the first product of an item overwrites accumulators the previous item's epilogue reads
-                    if (n == 0 && ic > 0 && !(ok = LT_WAIT(&sm.bar_acc_free, (ic - 1) & 1, kWaitAccFree))) break;
+                        umma_ss(tmem + kColS, dK_k + koff(kk), dQ_k + koff(kk), idesc_s, kk > 0);
+                    umma_ss(tmem + kColS, desc_ones, (t & 1) ? desc_ext_q1 : desc_ext_q0, idesc_s, 1);
+                    umma_commit(&sm.bar_s_full);
+                };
+                bool ok = true;
+                int it = 0, ic = 0;
+                for (;; ++ic) {
+                    if (!(ok = LT_WAIT(&sm.bar_item[ic % kItemRing], (ic / kItemRing) & 1, kWaitItem))) break;
+                    const int item = sm.item_ring[ic % kItemRing];
+                    if (item < 0) break;
+                    const BwdItem w = bwd_item<kSplit>(p, item);
+                    ok = LT_WAIT(&sm.bar_kv, ic & 1, kWaitKV) &&
+                         LT_WAIT(&sm.bar_q_full[it & 1], (it >> 1) & 1, kWaitStageFull);
+                    if (!ok) break;
                     tc_fence_after_sync();
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)
-                        umma_ts(tmem + kColdV, tmem + kColS + (kk >> 2) * 64 + (kk & 3) * 8, ddO_mn + roff(kk), idesc_dv,
-                                (n > 0) | (kk > 0));
-                    umma_commit(&sm.bar_do_empty);
-                    // the next S^T overwrites P'^T; the tensor pipe executes in issue order
-                    if (n + 1 < w.n_iter) {
-                        if (!(ok = LT_WAIT(&sm.bar_q_full[(it + 1) & 1], ((it + 1) >> 1) & 1, kWaitStageFull))) break;
-                        if constexpr (!kSavedP) issue_s(it + 1);
+                    if constexpr (!kSavedP) issue_s(it);
+                    for (int n = 0; n < w.n_iter && ok; ++n, ++it) {
+                        const int s = it & 1;
+                        const uint64_t dQ_mn = dQ_mn0 + s * kQStageStep;
+                        // dP^T = V_j dO_i^T - delta_i   (its columns held the previous dQ partial until the
+                        //                                reduce warps drained it)
+                        if (!(ok = LT_WAIT(&sm.bar_do_full, it & 1, kWaitDoFull))) break;
+                        if (it > 0 && !(ok = LT_WAIT(&sm.bar_dq_empty, (it - 1) & 1, kWaitDqEmpty))) break;
+                        tc_fence_after_sync();
+    #pragma unroll
+                        for (int kk = 0; kk < D / 16; ++kk)
+                            umma_ss(tmem + kColdP, dV_k + koff(kk), ddO_k + koff(kk), idesc_s, kk > 0);
+                        umma_ss(tmem + kColdP, desc_ones, desc_ext_do, idesc_s, 1);
+#ifdef LT_BWD_GIVEUP_TEST
+                        // test build only: the hand-off of running iteration LT_BWD_GIVEUP_TEST is dropped, so
+                        // the waits downstream of it run out and the kernel has to leave through its give-up path
+                        if (it != LT_BWD_GIVEUP_TEST)
+#endif
+                        umma_commit(&sm.bar_dp_full);
+                        // dV_j += P'^T dO_i   (A = P'^T from tensor memory; query columns 0-63 sit at columns
+                        //                      0-31, query columns 64-127 at columns 64-95 of the S region)
+                        if (!(ok = LT_WAIT(&sm.bar_p_ready, it & 1, kWaitPReady))) break;
+                        // the first product of an item overwrites accumulators the previous item's epilogue reads
+                        if (n == 0 && ic > 0 && !(ok = LT_WAIT(&sm.bar_acc_free, (ic - 1) & 1, kWaitAccFree))) break;
+                        tc_fence_after_sync();
+    #pragma unroll
+                        for (int kk = 0; kk < 8; ++kk)
+                            umma_ts(tmem + kColdV, tmem + kColS + (kk >> 2) * 64 + (kk & 3) * 8, ddO_mn + roff(kk), idesc_dv,
+                                    (n > 0) | (kk > 0));
+                        umma_commit(&sm.bar_do_empty);
+                        // the next S^T overwrites P'^T; the tensor pipe executes in issue order
+                        if (n + 1 < w.n_iter) {
+                            if (!(ok = LT_WAIT(&sm.bar_q_full[(it + 1) & 1], ((it + 1) >> 1) & 1, kWaitStageFull))) break;
+                            if constexpr (!kSavedP) issue_s(it + 1);
+                        }
+                        if (!(ok = LT_WAIT(&sm.bar_ds_ready, it & 1, kWaitDsReady))) break;
+                        tc_fence_after_sync();
+                        // dK_j += dS'^T Q_i   (A = dS'^T from tensor memory, stored like P'^T: query columns
+                        //                       0-63 at columns 0-31 and 64-127 at columns 64-95 of the dP region)
+    #pragma unroll
+                        for (int kk = 0; kk < 8; ++kk)
+                            umma_ts(tmem + kColdK, tmem + kColdP + (kk >> 2) * 64 + (kk & 3) * 8, dQ_mn + roff(kk), idesc_dv,
+                                    (n > 0) | (kk > 0));
+                        umma_commit(&sm.bar_q_empty[s]);
+                        // dQ_i partial (contraction over key rows); it overwrites the dP columns, which is safe
+                        // after dK because the tensor pipe executes in issue order.  For D = 128 it is
+                        // produced transposed, dQ^T = K_j^T dS^T (lanes = head dim, columns = query rows), so
+                        // that the reduction moves whole accumulator rows; for D = 64 as dQ = dS K_j.
+    #pragma unroll
+                        for (int kk = 0; kk < 8; ++kk) {
+                            if constexpr (D == 128)
+                                umma_ss(tmem + kColdP, dK_mn + roff(kk), ddS_mn + roff(kk), idesc_dq, kk > 0);
+                            else
+                                umma_ss(tmem + kColdP, ddS_mn + roff(kk), dK_mn + roff(kk), idesc_dq, kk > 0);
+                        }
+                        umma_commit(&sm.bar_dq_full);
+                        umma_commit(&sm.bar_ds_free);
                     }
-                    if (!(ok = LT_WAIT(&sm.bar_ds_ready, it & 1, kWaitDsReady))) break;
-                    tc_fence_after_sync();
-                    // dK_j += dS'^T Q_i   (A = dS'^T from tensor memory, stored like P'^T: query columns
-                    //                       0-63 at columns 0-31 and 64-127 at columns 64-95 of the dP region)
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)
-                        umma_ts(tmem + kColdK, tmem + kColdP + (kk >> 2) * 64 + (kk & 3) * 8, dQ_mn + roff(kk), idesc_dv,
-                                (n > 0) | (kk > 0));
-                    umma_commit(&sm.bar_q_empty[s]);
-                    // dQ_i partial (contraction over key rows); it overwrites the dP columns, which is safe
-                    // after dK because the tensor pipe executes in issue order.  For D = 128 it is
-                    // produced transposed, dQ^T = K_j^T dS^T (lanes = head dim, columns = query rows), so
-                    // that the reduction moves whole accumulator rows; for D = 64 as dQ = dS K_j.
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {
-                        if constexpr (D == 128)
-                            umma_ss(tmem + kColdP, dK_mn + roff(kk), ddS_mn + roff(kk), idesc_dq, kk > 0);
-                        else
-                            umma_ss(tmem + kColdP, ddS_mn + roff(kk), dK_mn + roff(kk), idesc_dq, kk > 0);
-                    }
-                    umma_commit(&sm.bar_dq_full);
-                    umma_commit(&sm.bar_ds_free);
+                    if (!ok) break;
+                    umma_commit(&sm.bar_dkv_full);
                 }
-                if (!ok) break;
-                umma_commit(&sm.bar_dkv_full);
+                LT_TRACE_END(kRoleMma);
             }
-            LT_TRACE_END(kRoleMma);
+            __syncwarp();
         }
-        __syncwarp();
     } else if (warp < kReduceWarp0) {
         // ================================================================= softmax / dS warps
+        warpgroup_regs_take<kRegsCompute>();
         const int quad = warp & 3;                           // tensor-memory lane quadrant
         const int half_sel = (warp - kComputeWarp0) >> 2;    // 0: query columns 0-63, 1: 64-127
         const int row = quad * 32 + lane;                    // key row inside the tile
@@ -681,7 +748,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const float scale_log2 = p.scale * kLog2e;
         uint8_t *ds_tile = sm.ds + half_sel * kBoxBytesBwd;
         uint32_t pv[64];  // bits of this thread's 64 fp32 values of P' = P * 2^c for the current tile pair
-        float p_scale_log2 = 0.f;
+        const float p_scale_log2 = static_cast<float>(bwd_p_scale_log2(p.status));
         bool ok = smem_ok;
         int it = 0, ic = 0;
         LT_TRACE_BEGIN();
@@ -762,63 +829,10 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         };
 
         for (;; ++ic) {
-            // (after an abandoned wait the loop still comes here, so that the vote below is never short of a warp)
-            ok = ok && LT_WAIT(&sm.bar_item[ic % kItemRing], (ic / kItemRing) & 1, kWaitItem);
-            const int item = ok ? sm.item_ring[ic % kItemRing] : -1;
-            const BwdItem w = bwd_item<kSplit>(p, item < 0 ? 0 : item);
-            // ---- per item: a power-of-two factor 2^c carried by dS before it is rounded to fp16, chosen
-            // from a bound on |dS| <= |dP| + |delta| <= max||dO_row|| * max||V_row|| + max|delta| so that
-            // the scaled values use fp16's normal range without overflow.  The factor rides on P
-            // (P' = P * 2^c, c <= 14); dV and dQ/dK undo it exactly in their epilogues.
-            ok = ok && (item < 0 || LT_WAIT(&sm.bar_kv, ic & 1, kWaitKV));
-            if (ok && item >= 0 && half_sel == 0) {
-                // squared row norm of V: only a bound is needed (it picks a power of two, with a factor of two
-                // to spare), so the squares are summed in the operands' own packed precision, four
-                // independent sums.  fp16 values are scaled by 2^-4 first, so that elements up to 4080 square
-                // without overflow (beyond that the sum is inf and the most cautious factor is taken).
-                constexpr uint32_t kPre = 0x2C002C00u;   // (2^-4, 2^-4) as fp16
-                uint32_t acc2[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-                for (int x = 0; x < kBoxes; ++x) {
-                    const uint4 *src = reinterpret_cast<const uint4 *>(sm.v + x * kBoxBytesBwd + row * 128);
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        const uint4 u = src[(c + row) & 7];  // rotated start: conflict-free across the warp
-                        acc2[0] = sq_acc2<kBf16>(kBf16 ? u.x : hmul2_bits(u.x, kPre), acc2[0]);
-                        acc2[1] = sq_acc2<kBf16>(kBf16 ? u.y : hmul2_bits(u.y, kPre), acc2[1]);
-                        acc2[2] = sq_acc2<kBf16>(kBf16 ? u.z : hmul2_bits(u.z, kPre), acc2[2]);
-                        acc2[3] = sq_acc2<kBf16>(kBf16 ? u.w : hmul2_bits(u.w, kPre), acc2[3]);
-                    }
-                }
-                float n2 = 0.f;
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const float2 f = unpack2<kBf16>(acc2[e]);
-                    n2 += f.x + f.y;
-                }
-                n2 *= (kBf16 ? 1.0625f : 256.f * 1.0625f);  // undo the pre-scaling; head room for the packed sums' rounding
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) n2 = fmaxf(n2, __shfl_xor_sync(0xffffffffu, n2, off));
-                if (lane == 0) sm.red[ic & 1][quad] = n2;
-            }
-            // all eight warps vote here, also when leaving after an abandoned wait, so nobody is left behind
-            ok = named_barrier_and(kBarComputeWarps, kNumComputeWarps * 32, ok);
-            if (!ok || item < 0) break;  // every warp sees the same item, so they leave together
-            {
-                const float *rd = sm.red[ic & 1];
-                const float vmax2 = fmaxf(fmaxf(rd[0], rd[1]), fmaxf(rd[2], rd[3]));
-                const float do2 = __uint_as_float(p.status[kStatusWordMaxDoNorm2]);
-                const float dmax = __uint_as_float(p.status[kStatusWordMaxAbsDelta]);
-                const float bound = sqrtf(do2) * sqrtf(vmax2) + dmax;
-                int e = static_cast<int>(kPScaleLog2Max);    // all-zero dO: any factor works
-                if (!(bound < 3.0e38f)) e = -14;             // inf/NaN inputs: outputs are non-finite anyway
-                else if (bound > 1e-30f) e = min(static_cast<int>(kPScaleLog2Max), max(-14, ilogbf(32768.f / bound)));
-                p_scale_log2 = static_cast<float>(e);
-                if (warp == kComputeWarp0 && lane == 0) {
-                    sm.p_scale[ic & 1] = p_scale_log2;
-                    mbar_arrive(&sm.bar_scale_ready);  // the reduction warps read it
-                }
-            }
+            if (!ok || !LT_WAIT(&sm.bar_item[ic % kItemRing], (ic / kItemRing) & 1, kWaitItem)) break;
+            const int item = sm.item_ring[ic % kItemRing];
+            if (item < 0) break;
+            const BwdItem w = bwd_item<kSplit>(p, item);
             if constexpr (kSavedP) load_saved_p(w, 0, ph);
             ok = compute_p(w, 0, it);
             for (int n = 0; n < w.n_iter && ok; ++n, ++it) {
@@ -876,7 +890,11 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         LT_TRACE_END(kRoleCompute);
     } else {
         // ================================================================= dQ reduction warps
+        warpgroup_regs_take<kRegsReduce>();
         const int quad = warp & 3;
+        // P carried the factor 2^c through dS into the accumulators; the epilogues take it out again (exact)
+        const float inv_p_scale = exp2f(-static_cast<float>(bwd_p_scale_log2(p.status)));
+        const float dq_mult = p.scale * inv_p_scale;
         bool ok = smem_ok;
         int it = 0, ic = 0;
         LT_TRACE_BEGIN();
@@ -889,14 +907,8 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             const int item = sm.item_ring[ic % kItemRing];
             if (item < 0) break;
             const BwdItem w = bwd_item<kSplit>(p, item);
-            float dq_mult = 0.f, inv_p_scale = 0.f;
             for (int n = 0; n < w.n_iter; ++n, ++it) {
                 ok = LT_WAIT(&sm.bar_dq_full, it & 1, kWaitDqFull);
-                if (ok && n == 0) {
-                    ok = LT_WAIT(&sm.bar_scale_ready, ic & 1, kWaitScale);
-                    inv_p_scale = exp2f(-sm.p_scale[ic & 1]);  // 2^-c, exact
-                    dq_mult = p.scale * inv_p_scale;
-                }
                 // the four reduction warps share named barriers below, so they leave the loop together;
                 // the vote also tells them that the staging buffers of the previous tile are free
                 if constexpr (D == 128) ok = named_barrier_and(kBarReduceWarps, kNumReduceWarps * 32, ok);
@@ -1091,16 +1103,26 @@ extern "C" int lt_dbg_bwd_trace(unsigned long long *out, int reset) {
 // group (dK_j, dV_j of all its heads accumulate in one CTA's tensor memory).  Shapes that would give
 // the 148 SMs only a few, heavy items get the group split over several items instead; their shares of
 // dK_j, dV_j are then summed in fp32 in the workspace and rounded by a small extra kernel.
-constexpr int kSplitBelowItems = 148 + 148 / 2;  // split when there are fewer than 1.5 whole-group items per SM
-constexpr int kSplitTargetItems = 2 * 148;       // and then aim at two items per SM (every item pays a pipeline fill)
-constexpr long long kSplitMinIterations = 20 * 148;  // problems below this are launch-bound anyway
+// Multiprocessors of the current device (148 on a B200; that figure is also the answer when the query fails,
+// so that the sizes derived from it never depend on an error path).
+static int sm_count() {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        return 148;
+    return sms;
+}
 static int heads_per_item(int B, int Hq, int Hkv, int S, int causal) {
+    const int sms = sm_count();
+    const long long split_below_items = sms + sms / 2;  // split when there are fewer than 1.5 whole-group items per SM
+    const long long split_target_items = 2 * sms;       // and then aim at two items per SM (every item pays a pipeline fill)
+    const long long split_min_iterations = 20 * sms;    // problems below this are launch-bound anyway
     const int G = Hq / Hkv;
     const long long n_tiles = padded_rows(S) / kTileRows;
     const long long n_base = static_cast<long long>(B) * Hkv * n_tiles;
     const long long iters = static_cast<long long>(B) * Hq * (causal ? n_tiles * (n_tiles + 1) / 2 : n_tiles * n_tiles);
-    if (G == 1 || n_base >= kSplitBelowItems || iters < kSplitMinIterations) return G;
-    const long long split = (kSplitTargetItems + n_base - 1) / n_base;
+    if (G == 1 || n_base >= split_below_items || iters < split_min_iterations) return G;
+    const long long split = (split_target_items + n_base - 1) / n_base;
     const int hs = static_cast<int>(split < G ? split : G);
     return (G + hs - 1) / hs;
 }
@@ -1145,12 +1167,7 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
     cudaError_t e = cudaMemsetAsync(status, 0, kStatusBytes, stream);
     if (e != cudaSuccess) return record_cuda_error("cudaMemsetAsync(status)", e);
 
-    int sms = 148;
-    {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    }
+    const int sms = sm_count();
     constexpr int kRowsPerBlock = 8 * (32 / (D / 8)) * kPreUnroll;
     const long long want = (n_rows + kRowsPerBlock - 1) / kRowsPerBlock;
     const int pre_blocks = static_cast<int>(want < static_cast<long long>(sms) * 16 ? want : sms * 16);
@@ -1158,7 +1175,10 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
                                                              reinterpret_cast<const __half *>(O), LSE, delta_ext,
                                                              lse_ext, dq_acc, n_rows, S, S_pad, Hq, lay.d_o, lay.o, plain_pre,
                                                              1.f / scale, status, reinterpret_cast<float4 *>(dk_acc),
-                                                             parts > 1 ? static_cast<long long>(kv_floats / 2) : 0LL);
+                                                             parts > 1 ? static_cast<long long>(kv_floats / 2) : 0LL,
+                                                             reinterpret_cast<const __half *>(V),
+                                                             static_cast<long long>(B) * Hkv * S, Hkv, lay.v,
+                                                             is_contig(lay.v, Hkv) ? 1 : 0);
     e = cudaGetLastError();
     if (e != cudaSuccess) return record_cuda_error("bwd_preprocess_kernel launch", e);
 
@@ -1265,7 +1285,11 @@ size_t lt_attn_bwd_workspace_bytes(int B, int Hq, int Hkv, int S, int D) {
     return bytes;
 }
 
-int lt_attn_bwd_num_launches(void) { return 3; }
+int lt_attn_bwd_num_launches(int B, int Hq, int Hkv, int S, int D, int causal) {
+    if (lt::check_shape(B, Hq, Hkv, S, D, 1.0f) != LT_OK) return 0;
+    // preprocess, main, dQ conversion; plus the dK/dV conversion when groups are split over work items
+    return lt::heads_per_item(B, Hq, Hkv, S, causal) < Hq / Hkv ? 4 : 3;
+}
 
 static int bwd_entry(const lt_half *Q, const lt_half *K, const lt_half *V, const lt_half *O, const lt_half *dO,
                      const float *LSE, lt_half *dQ, lt_half *dK, lt_half *dV, const lt_attn_layout *layout, int B,
@@ -1407,6 +1431,20 @@ int lt_attn_bwd_noalloc(const lt_half *Q, const lt_half *K, const lt_half *V, co
     // every call, so nothing left in the scratch by an earlier call is read
     return lt_attn_bwd(Q, K, V, O, dO, LSE, dQ, dK, dV, B, Hq, Hkv, S, D, causal, scale, scratch,
                        kNoAllocScratchBytes, stream);
+}
+
+int lt_attn_bwd_noalloc_check_status(lt_stream_t stream) {
+    using namespace lt;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return record_cuda_error("cudaGetDevice", e);
+    void *scratch = nullptr;
+    if (dev >= 0 && dev < kNoAllocMaxDevices) {
+        std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+        scratch = g_noalloc_scratch_addr[dev];
+    }
+    if (!scratch) return LT_OK;  // no lt_attn_bwd_noalloc call on this device yet: nothing to report
+    return lt_attn_check_status(scratch, stream);
 }
 
 }  // extern "C"

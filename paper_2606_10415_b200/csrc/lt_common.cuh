@@ -13,15 +13,21 @@ namespace lt {
 
 // ----------------------------------------------------------------------------- status block
 // First 256 bytes of every workspace.  Word 0: 0 = ok, otherwise the code of the wait
-// that gave up.  Word 1: max |delta| bits, word 2: max ||dO_row||^2 bits (backward).
+// that gave up.  Word 1: max |delta| bits, word 2: max ||dO_row||^2 bits, word 4: max ||V_row||^2
+// bits (backward).
 constexpr int kStatusBytes = 256;
 constexpr int kStatusWordTimeout = 0;
 constexpr int kStatusWordMaxAbsDelta = 1;
 constexpr int kStatusWordMaxDoNorm2 = 2;
 constexpr int kStatusWordItemCounter = 3;  // next unclaimed work item of the backward main kernel
+constexpr int kStatusWordMaxVNorm2 = 4;
 
-// A wait gives up after this many clock cycles (about one second) ...
-constexpr long long kWaitLimitCycles = 2000000000LL;
+// A wait gives up after this many clock cycles (about one second; the build of the give-up test
+// shortens it).
+#ifndef LT_WAIT_LIMIT_CYCLES
+#define LT_WAIT_LIMIT_CYCLES 2000000000LL
+#endif
+constexpr long long kWaitLimitCycles = LT_WAIT_LIMIT_CYCLES;
 
 // ----------------------------------------------------------------------------- small helpers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
@@ -97,6 +103,20 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
 // CTA of that kernel has executed it or exited).  Without the launch attribute both are no-ops.
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// ----------------------------------------------------------------------------- register budget
+// The registers of a CTA are split evenly between its warps at launch.  A warpgroup (four
+// consecutive warps, the first a multiple of four) can hand registers back or take more; every
+// warp of the group must execute the same instruction, and an increase waits until other groups
+// have released enough.  N: registers per thread afterwards, a multiple of 8 in [24, 256].
+template <int N>
+__device__ __forceinline__ void warpgroup_regs_release() {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N>
+__device__ __forceinline__ void warpgroup_regs_take() {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
 
 // ----------------------------------------------------------------------------- fences
 __device__ __forceinline__ void fence_proxy_async_smem() {

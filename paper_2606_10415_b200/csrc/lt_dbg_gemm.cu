@@ -1,7 +1,8 @@
 // Bring-up check of one 128x128x128 tensor-core tile product in each operand
-// arrangement the attention kernels use (see lt_dbg_tile_gemm in lt_attn.h).
+// arrangement the attention kernels use (see lt_dbg_tile_gemm in lt_attn_debug.h).
 #include "lt_common.cuh"
 #include "lt_host.h"
+#include "../../include/lt_attn_debug.h"
 
 namespace lt {
 

@@ -1,0 +1,89 @@
+"""Error measures and gates shared by the GPU parity tests.
+
+Every gradient tensor has to pass four gates against the fp64 oracle:
+
+  rel_fro   ||g - ref||_F / ||ref||_F <= 5e-3           (the stated target tolerance)
+  max_abs   max |g - ref| <= 2e-2                        (the stated target tolerance)
+  elem      max |g - ref| <= elem * max |ref|            (scale-normalised element bound)
+  row       for every row (the D elements of one sequence position of one head):
+            ||g_row - ref_row|| <= row * max(||ref_row||, 0.25 * rms row norm of ref)
+
+The last two exist because the benchmark inputs (dO with standard deviation 1e-2) give gradients
+of 1e-4 ... 1e-2, where max_abs <= 2e-2 cannot fail: `elem` catches a wrong element or 16-byte chunk,
+`row` a wrong row among thousands of right ones (which moves the Frobenius norm of a 4096-row head by
+only 1.6e-2 / sqrt(tiles)).  Rows whose exact norm is far below the typical one (the first rows under a
+causal mask see a handful of keys) are measured against a quarter of the root-mean-square row norm.
+
+The numbers are about three times the largest values measured over the whole suite with the fp16
+and bf16 kernels (fp16: elem 1.5e-3, row 1.2e-2; bf16: elem 4.6e-3, row 3.3e-2); bf16 keeps 8
+significant bits where fp16 keeps 11, which is the factor between the two sets.  A wrong value of
+typical size misses them by a factor of ten or more: a typical element is about a quarter of the
+largest one, and one such element is 1/sqrt(D) ~ 0.09 of its row's norm.
+"""
+import json
+import os
+
+import numpy as np
+
+REL_FRO_TOL = 5e-3
+MAX_ABS_TOL = 2e-2
+ELEM_TOL = {"fp16": 4e-3, "bf16": 1.6e-2}
+ROW_TOL = {"fp16": 3e-2, "bf16": 1e-1}
+ROW_FLOOR = 0.25
+# an exactly zero gradient (a single visible key) comes out as rounding residue of the -delta split
+ZERO_REF_ABS_TOL = 1e-6
+
+
+def rel_fro(a, ref):
+    a = np.asarray(a, dtype=np.float64)
+    return float(np.linalg.norm(a - ref) / max(np.linalg.norm(ref), 1e-300))
+
+
+def max_abs(a, ref):
+    return float(np.abs(np.asarray(a, dtype=np.float64) - ref).max())
+
+
+def error_measures(g, ref):
+    """rel_fro, max_abs, elem (max error over max |ref|) and row (worst floored relative row error)."""
+    g = np.asarray(g, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    err = g - ref
+    D = ref.shape[-1]
+    row_err = np.linalg.norm(err.reshape(-1, D), axis=1)
+    row_ref = np.linalg.norm(ref.reshape(-1, D), axis=1)
+    rms = float(np.sqrt(np.mean(row_ref ** 2)))
+    max_ref = float(np.abs(ref).max())
+    return {
+        "rel_fro": float(np.linalg.norm(err) / max(np.linalg.norm(ref), 1e-300)),
+        "max_abs": float(np.abs(err).max()),
+        "elem": float(np.abs(err).max() / max_ref) if max_ref > 0 else float(np.abs(err).max() > 0),
+        "row": float((row_err / np.maximum(row_ref, max(ROW_FLOOR * rms, 1e-300))).max()),
+        "max_ref": max_ref,
+    }
+
+
+def check_tensor(name, g, ref, what, dtype="fp16", rel_fro_tol=REL_FRO_TOL, absolute=True):
+    """absolute=False leaves the max_abs gate out (inputs scaled far away from the usual magnitudes)."""
+    g = np.asarray(g, dtype=np.float64)
+    assert np.all(np.isfinite(g)), f"{what} {name}: non-finite output"
+    m = error_measures(g, ref)
+    if os.environ.get("LT_PARITY_REPORT"):  # development aid: every measured value, one JSON line each
+        with open(os.environ["LT_PARITY_REPORT"], "a") as f:
+            f.write(json.dumps({"what": str(what), "tensor": name, "dtype": dtype, **m}) + "\n")
+    if m["max_ref"] == 0.0:
+        assert np.abs(g).max() <= ZERO_REF_ABS_TOL, f"{what} {name}: exact gradient is zero, got {np.abs(g).max():.3e}"
+        return m
+    assert m["rel_fro"] <= rel_fro_tol, f"{what} {name}: rel Frobenius {m['rel_fro']:.3e}"
+    assert not absolute or m["max_abs"] <= MAX_ABS_TOL, f"{what} {name}: max abs {m['max_abs']:.3e}"
+    assert m["elem"] <= ELEM_TOL[dtype], f"{what} {name}: max error / max |ref| {m['elem']:.3e}"
+    assert m["row"] <= ROW_TOL[dtype], f"{what} {name}: worst relative row error {m['row']:.3e}"
+    return m
+
+
+def check_grads(got, ref, what, dtype="fp16", **kw):
+    """got: (dQ, dK, dV) torch tensors (any device) or arrays; ref: the oracle's fp64 arrays."""
+    out = {}
+    for name, g, r in zip(("dQ", "dK", "dV"), got, ref):
+        g = g.detach().cpu().double().numpy() if hasattr(g, "detach") else g
+        out[name] = check_tensor(name, g, r, what, dtype, **kw)
+    return out

@@ -17,8 +17,8 @@ def binding():
     return b
 
 
-def declared_functions():
-    text = (ROOT / "include" / "lt_attn.h").read_text()
+def declared_functions(header="lt_attn.h"):
+    text = (ROOT / "include" / header).read_text()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     return sorted(set(re.findall(r"\b(lt_[a-z0-9_]+)\s*\(", text)))
 
@@ -32,9 +32,12 @@ def test_header_declares_the_documented_entry_points():
 
 def test_library_exports_every_declared_symbol(binding):
     lib = ctypes.CDLL(str(binding.LIB_PATH))
-    for name in declared_functions():
+    for name in declared_functions() + declared_functions("lt_attn_debug.h"):
         assert hasattr(lib, name), name
     assert set(declared_functions()) == set(binding.EXPORTS)
+    # the test-support entry points live in a header of their own, outside the product interface
+    assert set(declared_functions("lt_attn_debug.h")) == set(binding.DEBUG_EXPORTS)
+    assert not any(n.startswith("lt_dbg") for n in declared_functions())
 
 
 def test_workspace_sizes(binding):
@@ -50,6 +53,15 @@ def test_workspace_sizes(binding):
     assert binding.lt_attn_bwd_workspace_bytes(1, 2, 2, 128, 96) == 0
     assert binding.lt_attn_bwd_workspace_bytes(1, 3, 2, 128, 64) == 0
     assert binding.lt_attn_host_arena_bytes(1, 2, 2, 128, 64) > binding.lt_attn_bwd_workspace_bytes(1, 2, 2, 128, 64)
+
+
+def test_launch_counts(binding):
+    # three kernels per backward call; four on grouped-query shapes with few, heavy work items
+    assert binding.lt_attn_bwd_num_launches(1, 32, 32, 4096, 128, True) == 3
+    assert binding.lt_attn_bwd_num_launches(1, 40, 8, 4096, 128, True) == 3
+    assert binding.lt_attn_bwd_num_launches(1, 40, 8, 2048, 128, True) == 4
+    assert binding.lt_attn_bwd_num_launches(1, 2, 2, 128, 96, True) == 0
+    assert binding.lt_attn_fwd_num_launches() == 1
 
 
 def test_status_strings(binding):

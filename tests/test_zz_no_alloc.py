@@ -1,4 +1,4 @@
-"""The allocation-free backward entry point against the ordinary one.
+"""The allocation-free backward entry point against the ordinary one and against the CPU oracle.
 
 Some users of the library cannot allocate device memory where they call the backward (a
 fixed memory pool, a plugin without an allocator, an allocation-free steady state), so
@@ -11,6 +11,7 @@ import pytest
 import torch
 
 from paper_2606_10415_b200 import workloads
+from parity_checks import check_grads
 
 pytestmark = pytest.mark.gpu
 
@@ -36,7 +37,7 @@ def _inputs(lt, cfg):
     return Q, K, V, O, dO, LSE
 
 
-def test_noalloc_matches_workspace_entry_point_twice_in_a_row(lt):
+def test_noalloc_matches_workspace_entry_point_twice_in_a_row(lt, oracle):
     # two different shapes back to back: the second call finds the first call's leftovers in the scratch
     for cfg in (workloads.custom(1, 4, 2, 512, 128, True, seed=21), workloads.custom(2, 2, 2, 256, 64, True, seed=22)):
         Q, K, V, O, dO, LSE = _inputs(lt, cfg)
@@ -47,12 +48,16 @@ def test_noalloc_matches_workspace_entry_point_twice_in_a_row(lt):
         for _ in range(2):
             got = [torch.full_like(t, float("nan")) for t in ref]
             lt.lt_attn_bwd_noalloc(Q, K, V, O, dO, LSE, *got, cfg.causal, cfg.scale)
-            torch.cuda.synchronize()
+            # the status word of the built-in scratch: no wait gave up (this call synchronises the stream)
+            assert lt.lt_attn_bwd_noalloc_check_status() == lt.LT_OK, lt.last_cuda_error()
             # dK and dV have a fixed summation order; dQ is reduced with atomics
             assert torch.equal(got[1].cpu(), ref[1].cpu())
             assert torch.equal(got[2].cpu(), ref[2].cpu())
             assert torch.isfinite(got[0].float()).all()
             assert _rel_fro(got[0].cpu(), ref[0].cpu()) < 1e-3
+        # and the entry point's own output against the fp64 oracle, to the gates of the parity tests
+        exact = oracle.attn_bwd(*(t.cpu().double().numpy() for t in (Q, K, V, dO)), cfg.causal, cfg.scale)
+        check_grads(got, exact, f"noalloc {cfg}")
 
 
 def test_noalloc_rejects_shapes_beyond_its_scratch(lt):
