@@ -100,12 +100,14 @@ def time_oracle(cfg, n_heads, steps, warmup):
     import oracle
     sub, arrs = oracle_sample(cfg, n_heads)
     times = []
+    result = None
     for it in range(warmup + steps):
         t0 = time.perf_counter()
-        oracle.attn_bwd(*arrs, sub.causal, sub.scale)
+        result = oracle.attn_bwd(*arrs, sub.causal, sub.scale)
         dt = time.perf_counter() - t0
         if it >= warmup:
             times.append(dt)
+    time_oracle.last_result = result  # (dQ, dK, dV) of the sample, fp64
     return sub, times, oracle.num_threads()
 
 
@@ -166,7 +168,7 @@ class ClockSampler:
             self.proc = None
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "power_w": None}
         if self.proc is None:
             return out
         self.proc.terminate()
@@ -174,7 +176,7 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        clocks, maxes, reasons = [], [], set()
+        clocks, maxes, power, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for ln in Path(self.path).read_text().splitlines():
             parts = [x.strip() for x in ln.split(",")]
@@ -185,13 +187,17 @@ class ClockSampler:
                 maxes.append(float(parts[1]))
             except ValueError:
                 continue
+            try:
+                power.append(float(parts[2]))
+            except ValueError:
+                pass
             for name, val in zip(names, parts[3:7]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
         os.unlink(self.path)
         if clocks:
             out.update(sm_mhz=statistics.median(clocks), sm_max_mhz=max(maxes), reasons=sorted(reasons),
-                       samples=len(clocks))
+                       samples=len(clocks), power_w=statistics.median(power) if power else None)
         return out
 
 
@@ -327,11 +333,11 @@ def run_ours(args, cfg):
     if lt.lt_attn_check_status(ws) != lt.LT_OK:
         raise SystemExit("backward kernel reported: " + lt.last_cuda_error())
 
-    kernel_events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-                     for _ in range(args.steps)]
-    for a, b in kernel_events:  # materialise the event handles
-        a.record()
-        b.record()
+    # per step: call begin, main kernel begin, main kernel end, call end
+    kernel_events = [tuple(torch.cuda.Event(enable_timing=True) for _ in range(4)) for _ in range(args.steps)]
+    for evs in kernel_events:  # materialise the event handles
+        for e in evs:
+            e.record()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(torch.cuda.current_device()).uuid))
     barrier()
@@ -352,8 +358,10 @@ def run_ours(args, cfg):
     t1.record()
     # ... and the same number of steps again, now with an event on either side of the main kernel, give
     # its average duration under the same sustained load
-    for a, b in kernel_events:
+    for c0, a, b, c1 in kernel_events:
+        c0.record()
         step(a, b)
+        c1.record()
     barrier()
     total_ms = t0.elapsed_time(t1)
     busy_until = time.perf_counter() + args.clock_sample_ms * 0.5e-3
@@ -363,7 +371,11 @@ def run_ours(args, cfg):
     clocks = sampler.stop() if rank == 0 else None
     if lt.lt_attn_check_status(ws) != lt.LT_OK:
         raise SystemExit("backward kernel reported: " + lt.last_cuda_error())
-    main_ms = [a.elapsed_time(b) for a, b in kernel_events]
+    main_ms = [a.elapsed_time(b) for _, a, b, _ in kernel_events]
+    # what runs before the main kernel (status clear + preprocess kernel) and after it (dQ conversion, and the
+    # dK/dV conversion on split-group shapes), from the same profiled calls
+    pre_ms = [c0.elapsed_time(a) for c0, a, _, _ in kernel_events]
+    post_ms = [b.elapsed_time(c1) for _, _, b, c1 in kernel_events]
 
     # the main kernel timed alone: single launches with the GPU idle in between (the way the burst
     # GEMM peak was taken: best of 10)
@@ -480,6 +492,13 @@ def run_ours(args, cfg):
                          "algorithmic_hbm_bytes": _step_bytes(cfg) - 4.0 * cfg.B * cfg.Hq * cfg.S * cfg.D,
                          "peak_source": sustained_kind + " bf16 sustained (kernel timed inside the step loop)",
                          "avg_launch_ms": main_avg_ms, "median_launch_ms": statistics.median(main_ms),
+                         "other_kernels": {"preprocess_ms": sum(pre_ms) / len(pre_ms),
+                                           "finalize_ms": sum(post_ms) / len(post_ms),
+                                           "how": "CUDA events around the profiled calls: call begin to main "
+                                                  "kernel begin (status clear + preprocess kernel), main kernel "
+                                                  "end to call end (conversion kernels); with the events in "
+                                                  "place the kernels do not overlap, so the three add up to a "
+                                                  "little more than ms_per_step"},
                          "best_launch_ms": min(main_ms),
                          "burst_peak": peak, "frac_of_burst_peak": achieved / peak,
                          "timed_alone": {"best_launch_ms": iso_best_ms, "achieved": iso_achieved, "peak": peak,

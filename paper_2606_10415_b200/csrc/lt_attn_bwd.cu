@@ -36,6 +36,7 @@
 // variant that loads the probability tiles a forward pass saved (Section 4.1's own forward state,
 // written by lt_attn_save_p) instead of recomputing them.
 #include <mutex>
+#include <stddef.h>
 #include <stdio.h>
 
 #include "lt_common.cuh"
@@ -62,7 +63,7 @@ enum {
 constexpr int kPreUnroll = 4;
 
 template <int D, bool kBf16>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 3)  // three blocks per multiprocessor keep enough loads in flight
 bwd_preprocess_kernel(const __half *__restrict__ dO, const __half *__restrict__ O, const float *__restrict__ lse,
                       uint4 *__restrict__ delta_ext, uint4 *__restrict__ lse_ext, float *__restrict__ dq_acc,
                       long long n_rows, int S, int S_pad, int Hq, lt_tensor_strides do_st, lt_tensor_strides o_st,
@@ -319,7 +320,8 @@ constexpr int kBwdThreads = 512;  // 16 warps; 128 registers per thread at launc
 constexpr int kComputeWarp0 = 4, kNumComputeWarps = 8;
 constexpr int kReduceWarp0 = 12, kNumReduceWarps = 4;
 // registers per thread once the warpgroups have resized their shares (the SM has 64 K)
-constexpr int kRegsControl = 96, kRegsCompute = 144, kRegsReduce = 128;
+constexpr int kRegsAtLaunch = 65536 / kBwdThreads;
+constexpr int kRegsControl = 56, kRegsCompute = 168, kRegsReduce = 120;
 static_assert(128 * kRegsControl + kNumComputeWarps * 32 * kRegsCompute + kNumReduceWarps * 32 * kRegsReduce <= 65536,
               "register shares exceed the register file");
 constexpr int kDqStageBufs = 3, kDqStageRows = 16;
@@ -544,7 +546,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     // phase parity is a function of `it`; the per-item barriers use the item count `ic`.
     if (warp < kComputeWarp0) {
         // ================================================================= control group
-        warpgroup_regs_release<kRegsControl>();
+        warpgroup_regs_set<kRegsControl, kRegsAtLaunch>();
         if (warp == 0) {
             // ================================================================= TMA producer
             if (lane == 0 && smem_ok) {
@@ -570,7 +572,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         const BwdQTile qt = bwd_q_tile(p, w, n);
                         if (k >= 1 && !(ok = LT_WAIT(&sm.bar_q_empty[s], (k - 1) & 1, kWaitStageEmpty))) break;
                         mbar_arrive_expect_tx(&sm.bar_q_full[s], kSavedP ? kTileBytes : kTileBytes + kExtBytes);
-    #pragma unroll
+#pragma unroll
                         for (int x = 0; x < kBoxes; ++x)
                             tma_load_4d(sm.q[s] + x * kBoxBytesBwd, &map_q, &sm.bar_q_full[s], x * 64, qt.s0, qt.h, qt.b);
                         if constexpr (kSavedP)
@@ -580,7 +582,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         last_q = it;
                         if (it >= 1 && !(ok = LT_WAIT(&sm.bar_do_empty, (it - 1) & 1, kWaitDoEmpty))) break;
                         mbar_arrive_expect_tx(&sm.bar_do_full, kTileBytes + kExtBytes);
-    #pragma unroll
+#pragma unroll
                         for (int x = 0; x < kBoxes; ++x)
                             tma_load_4d(sm.d_o + x * kBoxBytesBwd, &map_do, &sm.bar_do_full, x * 64, qt.s0, qt.h, qt.b);
                         bulk_load_1d(sm.ext_do, p.delta_ext + qt.padded_row0, kExtBytes, &sm.bar_do_full);
@@ -590,7 +592,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                             // product of the previous item has completed
                             if (ic >= 1 && !(ok = LT_WAIT(&sm.bar_dkv_full, (ic - 1) & 1, kWaitDkvFull))) break;
                             mbar_arrive_expect_tx(&sm.bar_kv, 2 * kTileBytes);
-    #pragma unroll
+#pragma unroll
                             for (int x = 0; x < kBoxes; ++x) {
                                 tma_load_4d(sm.k + x * kBoxBytesBwd, &map_k, &sm.bar_kv, x * 64, w.j * kTileRows, w.g, w.b);
                                 tma_load_4d(sm.v + x * kBoxBytesBwd, &map_v, &sm.bar_kv, x * 64, w.j * kTileRows, w.g, w.b);
@@ -603,7 +605,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                             next_item = claim(ic + 1);
                             if (next_item >= 0) {
                                 const BwdItem wn = bwd_item<kSplit>(p, next_item);
-    #pragma unroll
+#pragma unroll
                                 for (int x = 0; x < kBoxes; ++x) {
                                     tma_prefetch_l2_4d(&map_k, x * 64, wn.j * kTileRows, wn.g, wn.b);
                                     tma_prefetch_l2_4d(&map_v, x * 64, wn.j * kTileRows, wn.g, wn.b);
@@ -630,35 +632,47 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             // ================================================================= tensor-core issuer
             if (lane == 0 && smem_ok) {
                 LT_TRACE_BEGIN();
-                // Every operand descriptor is a base computed once plus a compile-time constant in its
-                // address field (bits 0-13, units of 16 bytes; shared memory stays below 256 KB, so the
-                // sum never carries out of the field): the issuing thread then spends two integer adds
-                // per product and the tensor pipe, not this thread, sets the pace.
-                const uint32_t s_zero = smem_u32(sm.ext_zero);
-                const uint64_t dK_k = desc_kmajor(smem_u32(sm.k)), dV_k = desc_kmajor(smem_u32(sm.v));
-                const uint64_t dK_mn = desc_mnmajor(smem_u32(sm.k), kBoxBytesBwd);
-                const uint64_t ddS_mn = desc_mnmajor(smem_u32(sm.ds), kBoxBytesBwd);
-                const uint64_t ddO_k = desc_kmajor(smem_u32(sm.d_o)), ddO_mn = desc_mnmajor(smem_u32(sm.d_o), kBoxBytesBwd);
-                const uint64_t dQ_k0 = desc_kmajor(smem_u32(sm.q[0])), dQ_mn0 = desc_mnmajor(smem_u32(sm.q[0]), kBoxBytesBwd);
+                // Every operand descriptor is a compile-time constant (built from the operand's offset inside
+                // the shared window) plus the window's base in the address field (bits 0-13, units of 16
+                // bytes; shared memory stays below 256 KB, so the sum never carries out of the field).  The
+                // issuing thread spends one 64-bit add per descriptor, so the tensor pipe, not this thread,
+                // sets the pace.  The base is re-read through window_base() once per tile pair: otherwise the
+                // compiler keeps all ~80 sums of an iteration in registers across the loop, and the control
+                // group could not hand most of its registers to the other warpgroups.
+                const uint32_t base16 = smem_u32(smem_raw) >> 4;
+                auto window_base = [&]() -> uint64_t {
+                    uint32_t v;
+                    asm volatile("mov.u32 %0, %1;" : "=r"(v) : "r"(base16));
+                    return static_cast<uint64_t>(v);
+                };
+                constexpr uint32_t oK = offsetof(Smem, k), oV = offsetof(Smem, v), oQ = offsetof(Smem, q);
+                constexpr uint32_t oDo = offsetof(Smem, d_o), oDs = offsetof(Smem, ds), oZero = offsetof(Smem, ext_zero);
+                constexpr uint32_t oOnes = offsetof(Smem, ext_ones), oExtQ = offsetof(Smem, ext_q), oExtDo = offsetof(Smem, ext_do);
+                constexpr uint64_t dK_k = desc_kmajor(oK), dV_k = desc_kmajor(oV);
+                constexpr uint64_t dK_mn = desc_mnmajor(oK, kBoxBytesBwd);
+                constexpr uint64_t ddS_mn = desc_mnmajor(oDs, kBoxBytesBwd);
+                constexpr uint64_t ddO_k = desc_kmajor(oDo), ddO_mn = desc_mnmajor(oDo, kBoxBytesBwd);
+                constexpr uint64_t dQ_k0 = desc_kmajor(oQ), dQ_mn0 = desc_mnmajor(oQ, kBoxBytesBwd);
                 constexpr uint64_t kQStageStep = static_cast<uint64_t>(Smem::kTile) >> 4;  // next Q stage
-                const uint64_t desc_ones = desc_kmajor_noswz(smem_u32(sm.ext_ones), s_zero - smem_u32(sm.ext_ones), 128);
-                const uint64_t desc_ext_do = desc_kmajor_noswz(smem_u32(sm.ext_do), s_zero - smem_u32(sm.ext_do), 128);
-                const uint64_t desc_ext_q0 = desc_kmajor_noswz(smem_u32(sm.ext_q[0]), s_zero - smem_u32(sm.ext_q[0]), 128);
-                const uint64_t desc_ext_q1 = desc_kmajor_noswz(smem_u32(sm.ext_q[1]), s_zero - smem_u32(sm.ext_q[1]), 128);
+                constexpr uint64_t desc_ones = desc_kmajor_noswz(oOnes, oZero - oOnes, 128);
+                constexpr uint64_t desc_ext_do = desc_kmajor_noswz(oExtDo, oZero - oExtDo, 128);
+                constexpr uint64_t desc_ext_q0 = desc_kmajor_noswz(oExtQ, oZero - oExtQ, 128);
+                constexpr uint64_t desc_ext_q1 = desc_kmajor_noswz(oExtQ + kExtBytes, oZero - oExtQ - kExtBytes, 128);
                 // address-field increments of contraction step kk: within a contraction-contiguous tile
                 // (32 bytes per step, next 64-column tile after four steps) and within a row-contracted
                 // tile (16 rows of 128 bytes per step)
-                auto koff = [](int kk) -> uint64_t { return static_cast<uint64_t>((kk >> 2) * (kBoxBytesBwd >> 4) + (kk & 3) * 2); };
-                auto roff = [](int kk) -> uint64_t { return static_cast<uint64_t>(kk * (2048 >> 4)); };
+                constexpr auto koff = [](int kk) -> uint64_t { return static_cast<uint64_t>((kk >> 2) * (kBoxBytesBwd >> 4) + (kk & 3) * 2); };
+                constexpr auto roff = [](int kk) -> uint64_t { return static_cast<uint64_t>(kk * (2048 >> 4)); };
                 constexpr uint32_t idesc_s = make_idesc(128, 128, false, false, kBf16);
                 constexpr uint32_t idesc_dv = make_idesc(128, D, false, true, kBf16);
                 constexpr uint32_t idesc_dq = make_idesc(128, D == 128 ? 128 : D, true, true, kBf16);
                 auto issue_s = [&](int t) {  // S^T = K_j Q_i^T - LSE_i / scale, for running iteration t
-                    const uint64_t dQ_k = dQ_k0 + (t & 1) * kQStageStep;
-    #pragma unroll
+                    const uint64_t wb = window_base();
+                    const uint64_t dQ_k = wb + (t & 1) * kQStageStep;
+#pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk)
-                        umma_ss(tmem + kColS, dK_k + koff(kk), dQ_k + koff(kk), idesc_s, kk > 0);
-                    umma_ss(tmem + kColS, desc_ones, (t & 1) ? desc_ext_q1 : desc_ext_q0, idesc_s, 1);
+                        umma_ss(tmem + kColS, wb + (dK_k + koff(kk)), dQ_k + (dQ_k0 + koff(kk)), idesc_s, kk > 0);
+                    umma_ss(tmem + kColS, wb + desc_ones, wb + ((t & 1) ? desc_ext_q1 : desc_ext_q0), idesc_s, 1);
                     umma_commit(&sm.bar_s_full);
                 };
                 bool ok = true;
@@ -675,32 +689,40 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     if constexpr (!kSavedP) issue_s(it);
                     for (int n = 0; n < w.n_iter && ok; ++n, ++it) {
                         const int s = it & 1;
-                        const uint64_t dQ_mn = dQ_mn0 + s * kQStageStep;
+                        const uint64_t wb = window_base();
+                        const uint64_t dQ_mn = wb + s * kQStageStep;
+                        // dO_i and the -delta rows have landed: both dP and dV read them
+                        if (!(ok = LT_WAIT(&sm.bar_do_full, it & 1, kWaitDoFull))) break;
                         // dP^T = V_j dO_i^T - delta_i   (its columns held the previous dQ partial until the
                         //                                reduce warps drained it)
-                        if (!(ok = LT_WAIT(&sm.bar_do_full, it & 1, kWaitDoFull))) break;
-                        if (it > 0 && !(ok = LT_WAIT(&sm.bar_dq_empty, (it - 1) & 1, kWaitDqEmpty))) break;
-                        tc_fence_after_sync();
-    #pragma unroll
-                        for (int kk = 0; kk < D / 16; ++kk)
-                            umma_ss(tmem + kColdP, dV_k + koff(kk), ddO_k + koff(kk), idesc_s, kk > 0);
-                        umma_ss(tmem + kColdP, desc_ones, desc_ext_do, idesc_s, 1);
+                        auto issue_dp = [&]() {
+#pragma unroll
+                            for (int kk = 0; kk < D / 16; ++kk)
+                                umma_ss(tmem + kColdP, wb + (dV_k + koff(kk)), wb + (ddO_k + koff(kk)), idesc_s, kk > 0);
+                            umma_ss(tmem + kColdP, wb + desc_ones, wb + desc_ext_do, idesc_s, 1);
 #ifdef LT_BWD_GIVEUP_TEST
-                        // test build only: the hand-off of running iteration LT_BWD_GIVEUP_TEST is dropped, so
-                        // the waits downstream of it run out and the kernel has to leave through its give-up path
-                        if (it != LT_BWD_GIVEUP_TEST)
+                            // test build only: the hand-off of running iteration LT_BWD_GIVEUP_TEST is dropped, so
+                            // the waits downstream of it run out and the kernel has to leave through its give-up path
+                            if (it != LT_BWD_GIVEUP_TEST)
 #endif
-                        umma_commit(&sm.bar_dp_full);
+                            umma_commit(&sm.bar_dp_full);
+                        };
                         // dV_j += P'^T dO_i   (A = P'^T from tensor memory; query columns 0-63 sit at columns
                         //                      0-31, query columns 64-127 at columns 64-95 of the S region)
+                        auto issue_dv = [&]() {
+#pragma unroll
+                            for (int kk = 0; kk < 8; ++kk)
+                                umma_ts(tmem + kColdV, tmem + kColS + (kk >> 2) * 64 + (kk & 3) * 8, wb + (ddO_mn + roff(kk)),
+                                        idesc_dv, (n > 0) | (kk > 0));
+                        };
+                        if (it > 0 && !(ok = LT_WAIT(&sm.bar_dq_empty, (it - 1) & 1, kWaitDqEmpty))) break;
+                        tc_fence_after_sync();
+                        issue_dp();
                         if (!(ok = LT_WAIT(&sm.bar_p_ready, it & 1, kWaitPReady))) break;
                         // the first product of an item overwrites accumulators the previous item's epilogue reads
                         if (n == 0 && ic > 0 && !(ok = LT_WAIT(&sm.bar_acc_free, (ic - 1) & 1, kWaitAccFree))) break;
                         tc_fence_after_sync();
-    #pragma unroll
-                        for (int kk = 0; kk < 8; ++kk)
-                            umma_ts(tmem + kColdV, tmem + kColS + (kk >> 2) * 64 + (kk & 3) * 8, ddO_mn + roff(kk), idesc_dv,
-                                    (n > 0) | (kk > 0));
+                        issue_dv();
                         umma_commit(&sm.bar_do_empty);
                         // the next S^T overwrites P'^T; the tensor pipe executes in issue order
                         if (n + 1 < w.n_iter) {
@@ -711,21 +733,21 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         tc_fence_after_sync();
                         // dK_j += dS'^T Q_i   (A = dS'^T from tensor memory, stored like P'^T: query columns
                         //                       0-63 at columns 0-31 and 64-127 at columns 64-95 of the dP region)
-    #pragma unroll
+#pragma unroll
                         for (int kk = 0; kk < 8; ++kk)
-                            umma_ts(tmem + kColdK, tmem + kColdP + (kk >> 2) * 64 + (kk & 3) * 8, dQ_mn + roff(kk), idesc_dv,
+                            umma_ts(tmem + kColdK, tmem + kColdP + (kk >> 2) * 64 + (kk & 3) * 8, dQ_mn + (dQ_mn0 + roff(kk)), idesc_dv,
                                     (n > 0) | (kk > 0));
                         umma_commit(&sm.bar_q_empty[s]);
                         // dQ_i partial (contraction over key rows); it overwrites the dP columns, which is safe
                         // after dK because the tensor pipe executes in issue order.  For D = 128 it is
                         // produced transposed, dQ^T = K_j^T dS^T (lanes = head dim, columns = query rows), so
                         // that the reduction moves whole accumulator rows; for D = 64 as dQ = dS K_j.
-    #pragma unroll
+#pragma unroll
                         for (int kk = 0; kk < 8; ++kk) {
                             if constexpr (D == 128)
-                                umma_ss(tmem + kColdP, dK_mn + roff(kk), ddS_mn + roff(kk), idesc_dq, kk > 0);
+                                umma_ss(tmem + kColdP, wb + (dK_mn + roff(kk)), wb + (ddS_mn + roff(kk)), idesc_dq, kk > 0);
                             else
-                                umma_ss(tmem + kColdP, ddS_mn + roff(kk), dK_mn + roff(kk), idesc_dq, kk > 0);
+                                umma_ss(tmem + kColdP, wb + (ddS_mn + roff(kk)), wb + (dK_mn + roff(kk)), idesc_dq, kk > 0);
                         }
                         umma_commit(&sm.bar_dq_full);
                         umma_commit(&sm.bar_ds_free);
@@ -739,7 +761,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
     } else if (warp < kReduceWarp0) {
         // ================================================================= softmax / dS warps
-        warpgroup_regs_take<kRegsCompute>();
+        warpgroup_regs_set<kRegsCompute, kRegsAtLaunch>();
         const int quad = warp & 3;                           // tensor-memory lane quadrant
         const int half_sel = (warp - kComputeWarp0) >> 2;    // 0: query columns 0-63, 1: 64-127
         const int row = quad * 32 + lane;                    // key row inside the tile
@@ -792,6 +814,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             const bool diag = p.causal && (w.i_first + (n - hh * w.tiles_per_head) == w.j);
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
+                // (one load at a time: asking for both halves before the first is used measured 2 % slower)
                 uint32_t sv[32];
                 tmem_ld32(tmem + lane_base + kColS + cbase + c * 32, sv);
                 tmem_wait_ld();
@@ -890,7 +913,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         LT_TRACE_END(kRoleCompute);
     } else {
         // ================================================================= dQ reduction warps
-        warpgroup_regs_take<kRegsReduce>();
+        warpgroup_regs_set<kRegsReduce, kRegsAtLaunch>();
         const int quad = warp & 3;
         // P carried the factor 2^c through dS into the accumulators; the epilogues take it out again (exact)
         const float inv_p_scale = exp2f(-static_cast<float>(bwd_p_scale_log2(p.status)));

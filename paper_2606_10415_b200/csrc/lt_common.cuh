@@ -109,13 +109,13 @@ __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddep
 // consecutive warps, the first a multiple of four) can hand registers back or take more; every
 // warp of the group must execute the same instruction, and an increase waits until other groups
 // have released enough.  N: registers per thread afterwards, a multiple of 8 in [24, 256].
-template <int N>
-__device__ __forceinline__ void warpgroup_regs_release() {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
-}
-template <int N>
-__device__ __forceinline__ void warpgroup_regs_take() {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+// kFrom is the count the group holds before the call: handing registers back and taking more are two
+// different instructions, and asking for "more" with a smaller count (or the reverse) is undefined.
+template <int N, int kFrom>
+__device__ __forceinline__ void warpgroup_regs_set() {
+    static_assert(N % 8 == 0 && N >= 24 && N <= 256, "register count must be a multiple of 8 in [24, 256]");
+    if constexpr (N < kFrom) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+    else if constexpr (N > kFrom) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
 }
 
 // ----------------------------------------------------------------------------- fences
@@ -299,13 +299,16 @@ __device__ __forceinline__ void umma_commit_pair(uint64_t *bar, uint16_t cta_mas
 //   row-index-contracted ("MN-major") operand   : rows are the contraction index; the 64
 //       M/N elements of a row are contiguous; the next 64 M/N elements live in the next
 //       tile (`mn_atom_stride` bytes away, leading field); 8-row groups are 1024 bytes apart.
+// The address field (bits 0-13, units of 16 bytes) is linear in the address: a descriptor built for an
+// offset inside the shared window plus (window base >> 4) is the descriptor of base + offset, as long as
+// the window ends below 256 KB (the sum then never carries out of the field).
 constexpr uint64_t kDescFixed = (1ull << 46) /* descriptor version for sm_100 */ | (2ull << 61) /* 128B swizzle */;
 
-__device__ __forceinline__ uint64_t desc_kmajor(uint32_t smem_addr) {
+__host__ __device__ constexpr uint64_t desc_kmajor(uint32_t smem_addr) {
     return kDescFixed | (static_cast<uint64_t>(1) << 16) | (static_cast<uint64_t>(1024 >> 4) << 32) |
            static_cast<uint64_t>((smem_addr & 0x3FFFF) >> 4);
 }
-__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t smem_addr, uint32_t mn_atom_stride) {
+__host__ __device__ constexpr uint64_t desc_mnmajor(uint32_t smem_addr, uint32_t mn_atom_stride) {
     return kDescFixed | (static_cast<uint64_t>((mn_atom_stride >> 4) & 0x3FFF) << 16) |
            (static_cast<uint64_t>(1024 >> 4) << 32) | static_cast<uint64_t>((smem_addr & 0x3FFFF) >> 4);
 }
@@ -313,7 +316,7 @@ __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t smem_addr, uint32_t mn
 // Unswizzled contraction-contiguous operand for one 16-element contraction step: rows of
 // 16 bytes (8 fp16) grouped in blocks of 8 rows (128 contiguous bytes); `sbo` bytes between
 // 8-row blocks, `lbo` bytes from the block holding elements 0-7 to the one holding 8-15.
-__device__ __forceinline__ uint64_t desc_kmajor_noswz(uint32_t smem_addr, uint32_t lbo, uint32_t sbo) {
+__host__ __device__ constexpr uint64_t desc_kmajor_noswz(uint32_t smem_addr, uint32_t lbo, uint32_t sbo) {
     return (1ull << 46) | (static_cast<uint64_t>((lbo >> 4) & 0x3FFF) << 16) |
            (static_cast<uint64_t>((sbo >> 4) & 0x3FFF) << 32) | static_cast<uint64_t>((smem_addr & 0x3FFFF) >> 4);
 }

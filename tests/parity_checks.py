@@ -14,11 +14,12 @@ of 1e-4 ... 1e-2, where max_abs <= 2e-2 cannot fail: `elem` catches a wrong elem
 only 1.6e-2 / sqrt(tiles)).  Rows whose exact norm is far below the typical one (the first rows under a
 causal mask see a handful of keys) are measured against a quarter of the root-mean-square row norm.
 
-The numbers are about three times the largest values measured over the whole suite with the fp16
-and bf16 kernels (fp16: elem 1.5e-3, row 1.2e-2; bf16: elem 4.6e-3, row 3.3e-2); bf16 keeps 8
-significant bits where fp16 keeps 11, which is the factor between the two sets.  A wrong value of
-typical size misses them by a factor of ten or more: a typical element is about a quarter of the
-largest one, and one such element is 1/sqrt(D) ~ 0.09 of its row's norm.
+The numbers are two to three times the largest values measured over the whole suite with the fp16
+and bf16 kernels (fp16: elem 1.5e-3, row 2.3e-2, the latter on an early, short row of the largest
+configuration; bf16: elem 4.8e-3, row 3.3e-2); bf16 keeps 8 significant bits where fp16 keeps 11,
+which is the factor between the two element bounds.  A wrong value of typical size misses them by a
+wide margin: a typical element is about a quarter of the largest one (60 times the fp16 bound), and
+one such element is 1/sqrt(D) ~ 0.09 of its row's norm, a wrong 16-byte chunk 0.25, a wrong row 1.
 """
 import json
 import os
@@ -28,7 +29,7 @@ import numpy as np
 REL_FRO_TOL = 5e-3
 MAX_ABS_TOL = 2e-2
 ELEM_TOL = {"fp16": 4e-3, "bf16": 1.6e-2}
-ROW_TOL = {"fp16": 3e-2, "bf16": 1e-1}
+ROW_TOL = {"fp16": 5e-2, "bf16": 1e-1}
 ROW_FLOOR = 0.25
 # an exactly zero gradient (a single visible key) comes out as rounding residue of the -delta split
 ZERO_REF_ABS_TOL = 1e-6
