@@ -131,6 +131,10 @@ def test_delta_preprocess_matches_oracle(lt, oracle):
     assert np.all(rows[:, 2:] == 0)
     delta = -(256.0 * rows[:, 0] + rows[:, 1]).reshape(cfg.B, cfg.Hq, cfg.S)
     ref = oracle.delta(dO.double().numpy(), O16.double().numpy())
+    # The stored row is a two-term fp16 split (256*hi + lo): hi carries 11 bits of delta/256 and lo 11 bits of
+    # the remainder, so a value keeps about 22 bits relative to its own size, but lo goes subnormal (absolute
+    # step 2^-24) for deltas far below the largest one: hence an absolute term of 2e-6 of the largest |delta|
+    # beside the relative one.
     np.testing.assert_allclose(delta, ref, rtol=1e-5, atol=2e-6 * np.abs(ref).max())
 
 
@@ -245,7 +249,7 @@ def test_sharp_softmax_and_large_scores(lt, oracle):
     Qn, Kn, Vn, dOn = (t.double().numpy() for t in (Q, K, V, dO))
     O_ref, LSE_ref = oracle.attn_fwd(Qn, Kn, Vn, True, cfg.scale)
     assert rel_fro(O.cpu().double().numpy(), O_ref) <= FWD_O_REL_FRO_TOL
-    assert max_abs(LSE.cpu().double().numpy(), LSE_ref) <= 4 * FWD_LSE_ABS_TOL  # |LSE| itself is ~50 here
+    assert max_abs(LSE.cpu().double().numpy(), LSE_ref) <= FWD_LSE_ABS_TOL
     got = run_bwd(lt, Q, K, V, O.cpu(), dO, LSE.cpu(), cfg)
     ref = oracle.attn_bwd(Qn, Kn, Vn, dOn, True, cfg.scale)
     check_grads(got, ref, "sharp softmax")

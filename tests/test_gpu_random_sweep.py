@@ -7,6 +7,7 @@ import pytest
 import torch
 
 from paper_2606_10415_b200 import workloads
+from parity_checks import check_tensor
 
 pytestmark = pytest.mark.gpu
 
@@ -79,11 +80,8 @@ def test_random_sweep(lt, oracle, seed):
         O_ref, LSE_ref = oracle.attn_fwd(*n[:3], cfg.causal, scale)
         ref = oracle.attn_bwd(*n, cfg.causal, scale)
         assert rel(O.cpu().double().numpy(), O_ref) <= (4e-3 if bf16 else 2e-3), what
-        assert np.abs(LSE.cpu().double().numpy() - LSE_ref).max() <= 2e-3 * max(1.0, np.abs(LSE_ref).max() / 10), what
+        assert np.abs(LSE.cpu().double().numpy() - LSE_ref).max() <= 1e-3, what
         for name, g, r in zip(("dQ", "dK", "dV"), (dQ, dK, dV), ref):
-            g = g.cpu().double().numpy()
-            assert np.all(np.isfinite(g)), f"{what} {name}"
-            if np.linalg.norm(r) > 1e-12:  # (a single visible key makes dQ and dK exactly zero)
-                assert rel(g, r) <= (6e-3 if bf16 else 5e-3), f"{what} {name}: {rel(g, r):.3e}"
-            else:
-                assert np.abs(g).max() <= 1e-6, f"{what} {name}"
+            # (a single visible key makes dQ and dK exactly zero: check_tensor then bounds the residue)
+            check_tensor(name, g.cpu().double().numpy(), r, what, dtype="bf16" if bf16 else "fp16",
+                         absolute=False)  # magnitudes vary over the sweep: the scale-free gates decide

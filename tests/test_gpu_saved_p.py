@@ -12,22 +12,12 @@ import pytest
 import torch
 
 from paper_2606_10415_b200 import workloads
+from parity_checks import check_grads
 
 pytestmark = pytest.mark.gpu
 
 P_ABS_TOL = 1e-3
-REL_FRO_TOL = 5e-3
-MAX_ABS_TOL = 2e-2
 
-
-def check_grads(got, ref, what):
-    for name, g, r in zip(("dQ", "dK", "dV"), got, ref):
-        g = g.double().numpy()
-        assert np.all(np.isfinite(g)), f"{what} {name}: non-finite output"
-        rf = float(np.linalg.norm(g - r) / max(np.linalg.norm(r), 1e-300))
-        ma = float(np.abs(g - r).max())
-        assert rf <= REL_FRO_TOL, f"{what} {name}: rel Frobenius {rf:.3e}"
-        assert ma <= MAX_ABS_TOL, f"{what} {name}: max abs {ma:.3e}"
 
 SHAPES = [
     # B, Hq, Hkv, S, D, causal
