@@ -22,8 +22,14 @@ constexpr int kFwdTileRows = 128;
 constexpr int kFwdBoxBytes = 128 * 128;
 constexpr float kFwdLog2e = 1.4426950408889634f;
 constexpr float kFwdLn2 = 0.6931471805599453f;
-constexpr int kFwdThreads = 320;              // producer warp, issuer warp, 2 x 4 softmax warps
-constexpr int kFwdSoftmaxWarp0 = 2;
+// three warpgroups: control (producer warp, issuer warp, two warps that only fill up the group) and 2 x 4
+// softmax warps; the control group hands most of its registers to the softmax warps, each of whose threads
+// keeps the 128 scores of a query row in registers
+constexpr int kFwdThreads = 384;
+constexpr int kFwdSoftmaxWarp0 = 4;
+constexpr int kFwdRegsAtLaunch = 168, kFwdRegsControl = 80, kFwdRegsSoftmax = 208;
+static_assert(kFwdRegsAtLaunch * kFwdThreads <= 65536 && 128 * kFwdRegsControl + 256 * kFwdRegsSoftmax <= 65536,
+              "register shares exceed the register file");
 constexpr float kFwdRescaleLog2 = 8.f;        // P <= 2^8 stays far inside fp16 range
 
 enum {
@@ -133,133 +139,137 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
     volatile int *abort_flag = &sm.abort_flag;
 
 
-    if (warp == 0) {
-        // ------------------------------------------------------------------ producer
-        if (lane == 0) {
-            for (int t = 0; t < (has_b ? 2 : 1); ++t) {
-                mbar_arrive_expect_tx(&sm.bar_q[t], kTileBytes);
+    if (warp < kFwdSoftmaxWarp0) {
+        warpgroup_regs_set<kFwdRegsControl, kFwdRegsAtLaunch>();
+        if (warp == 0) {
+            // ------------------------------------------------------------------ producer
+            if (lane == 0) {
+                for (int t = 0; t < (has_b ? 2 : 1); ++t) {
+                    mbar_arrive_expect_tx(&sm.bar_q[t], kTileBytes);
 #pragma unroll
-                for (int x = 0; x < kBoxes; ++x)
-                    tma_load_4d(sm.q[t] + x * kFwdBoxBytes, &map_q, &sm.bar_q[t], x * 64, (i0 + t) * kFwdTileRows, h, b);
-            }
-            bool ok = true;
-            int armed = 0;  // key/value tiles whose loads were started
-            for (int j = 0; j <= j_end; ++j) {
-                const int s = j & 1;
-                const uint32_t ph = (j >> 1) & 1;
-                const int kv_row0 = j * kFwdTileRows;  // inside the head; rows past S arrive as zeros
-                if (j >= 2 && !(ok = mbar_wait(&sm.bar_k_empty[s], ph ^ 1, abort_flag, p.status, kWaitFwdKEmpty))) break;
-                mbar_arrive_expect_tx(&sm.bar_k_full[s], kTileBytes);
-#pragma unroll
-                for (int x = 0; x < kBoxes; ++x)
-                    tma_load_4d(sm.k[s] + x * kFwdBoxBytes, &map_k, &sm.bar_k_full[s], x * 64, kv_row0, g, b);
-                if (j >= 2 && !(ok = mbar_wait(&sm.bar_v_empty[s], ph ^ 1, abort_flag, p.status, kWaitFwdVEmpty))) {
-                    // the key tile just started still has to land before shared memory is given up
-                    for (int w = 0; w < (1 << 16) && !mbar_try_wait(&sm.bar_k_full[s], ph); ++w) {}
-                    break;
+                    for (int x = 0; x < kBoxes; ++x)
+                        tma_load_4d(sm.q[t] + x * kFwdBoxBytes, &map_q, &sm.bar_q[t], x * 64, (i0 + t) * kFwdTileRows, h, b);
                 }
-                mbar_arrive_expect_tx(&sm.bar_v_full[s], kTileBytes);
+                bool ok = true;
+                int armed = 0;  // key/value tiles whose loads were started
+                for (int j = 0; j <= j_end; ++j) {
+                    const int s = j & 1;
+                    const uint32_t ph = (j >> 1) & 1;
+                    const int kv_row0 = j * kFwdTileRows;  // inside the head; rows past S arrive as zeros
+                    if (j >= 2 && !(ok = mbar_wait(&sm.bar_k_empty[s], ph ^ 1, abort_flag, p.status, kWaitFwdKEmpty))) break;
+                    mbar_arrive_expect_tx(&sm.bar_k_full[s], kTileBytes);
 #pragma unroll
-                for (int x = 0; x < kBoxes; ++x)
-                    tma_load_4d(sm.v[s] + x * kFwdBoxBytes, &map_v, &sm.bar_v_full[s], x * 64, kv_row0, g, b);
-                armed = j + 1;
-            }
-            if (!ok || *abort_flag) {
-                // somebody gave up: wait (bounded) for the copies in flight before the CTA exits
-                for (int t = 0; t < (has_b ? 2 : 1); ++t)
-                    for (int w = 0; w < (1 << 16) && !mbar_try_wait(&sm.bar_q[t], 0); ++w) {}
-                for (int j = armed > 2 ? armed - 2 : 0; j < armed; ++j) {
-                    for (int w = 0; w < (1 << 16) && !mbar_try_wait(&sm.bar_k_full[j & 1], (j >> 1) & 1); ++w) {}
-                    for (int w = 0; w < (1 << 16) && !mbar_try_wait(&sm.bar_v_full[j & 1], (j >> 1) & 1); ++w) {}
+                    for (int x = 0; x < kBoxes; ++x)
+                        tma_load_4d(sm.k[s] + x * kFwdBoxBytes, &map_k, &sm.bar_k_full[s], x * 64, kv_row0, g, b);
+                    if (j >= 2 && !(ok = mbar_wait(&sm.bar_v_empty[s], ph ^ 1, abort_flag, p.status, kWaitFwdVEmpty))) {
+                        // the key tile just started still has to land before shared memory is given up
+                        for (int w = 0; w < (1 << 16) && !mbar_try_wait(&sm.bar_k_full[s], ph); ++w) {}
+                        break;
+                    }
+                    mbar_arrive_expect_tx(&sm.bar_v_full[s], kTileBytes);
+#pragma unroll
+                    for (int x = 0; x < kBoxes; ++x)
+                        tma_load_4d(sm.v[s] + x * kFwdBoxBytes, &map_v, &sm.bar_v_full[s], x * 64, kv_row0, g, b);
+                    armed = j + 1;
                 }
-            }
-        }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            // descriptors of slot 0; slot 1 of each ring follows one tile later
-            const uint64_t dQ0 = desc_kmajor(smem_u32(sm.q[0])), dK0 = desc_kmajor(smem_u32(sm.k[0]));
-            const uint64_t dV0 = desc_mnmajor(smem_u32(sm.v[0]), kFwdBoxBytes);
-            constexpr uint64_t kSlotStep = static_cast<uint64_t>(kTileBytes) >> 4;
-            auto koff = [](int kk) -> uint64_t { return static_cast<uint64_t>((kk >> 2) * (kFwdBoxBytes >> 4) + (kk & 3) * 2); };
-            auto roff = [](int kk) -> uint64_t { return static_cast<uint64_t>(kk * (2048 >> 4)); };
-            constexpr uint32_t idesc_s = make_idesc(128, 128, false, false, kBf16);
-            constexpr uint32_t idesc_o = make_idesc(128, D, false, true, kBf16);
-            auto issue_s = [&](int t, int s) {  // S_t = Q_t K^T with the key tile in ring slot s
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk)
-                    umma_ss(tmem + kColS + t * 128, dQ0 + t * kSlotStep + koff(kk), dK0 + s * kSlotStep + koff(kk), idesc_s, kk > 0);
-                umma_commit(&sm.bar_s_full[t]);
-            };
-            // O_t (+)= P_t V, P_t read from tensor memory; the keys of a tile in two halves of 64, so that the
-            // first half's products run while the softmax warps exponentiate the second half (quarters were
-            // measured too and lost to the extra hand-offs)
-            auto issue_pv_half = [&](int t, int s, bool acc, int half) {
-#pragma unroll
-                for (int kk = 4 * half; kk < 4 * half + 4; ++kk)
-                    umma_ts(tmem + kColO + t * D, tmem + kColS + t * 128 + kk * 8, dV0 + s * kSlotStep + roff(kk), idesc_o,
-                            acc | (kk > 0));
-                if (half == 1) umma_commit(&sm.bar_o_done[t]);
-            };
-            bool ok = mbar_wait(&sm.bar_q[0], 0, abort_flag, p.status, kWaitFwdQ) &&
-                      (!has_b || mbar_wait(&sm.bar_q[1], 0, abort_flag, p.status, kWaitFwdQ)) &&
-                      mbar_wait(&sm.bar_k_full[0], 0, abort_flag, p.status, kWaitFwdK);
-            if (ok) {
-                tc_fence_after_sync();
-                issue_s(0, 0);
-                if (has_b) issue_s(1, 0);
-                umma_commit(&sm.bar_k_empty[0]);
-            }
-            LT_FT_DECL;
-            for (int j = 0; j <= j_end && ok; ++j) {
-                const int s = j & 1, sn = s ^ 1;
-                LT_FT(0);
-                if (!(ok = mbar_wait(&sm.bar_v_full[s], (j >> 1) & 1, abort_flag, p.status, kWaitFwdV))) break;
-                LT_FT(1);
-                bool k_next_ready = false;
-#pragma unroll
-                for (int t = 0; t < 2; ++t) {
-                    const int j_last_t = t == 0 ? j_last0 : j_last1;
-                    if (j > j_last_t) continue;
-                    LT_FT(0);
-                    if (!(ok = mbar_wait(&sm.bar_p_half[t], j & 1, abort_flag, p.status, kWaitFwdP))) break;
-                    tc_fence_after_sync();
-                    issue_pv_half(t, s, j > 0, 0);
-                    if (!(ok = mbar_wait(&sm.bar_p_ready[t], j & 1, abort_flag, p.status, kWaitFwdP))) break;
-                    LT_FT(2 + t);
-                    tc_fence_after_sync();
-                    LT_FT(0);
-                    issue_pv_half(t, s, j > 0, 1);
-                    LT_FT(5);
-                    // the second tile of the pair, when it uses this key tile, uses it last
-                    const int last_user = (j <= j_last1) ? 1 : 0;
-                    if (t == last_user) umma_commit(&sm.bar_v_empty[s]);
-                    if (j + 1 <= j_last_t) {
-                        if (!k_next_ready) {
-                            LT_FT(0);
-                            if (!(ok = mbar_wait(&sm.bar_k_full[sn], ((j + 1) >> 1) & 1, abort_flag, p.status, kWaitFwdK))) break;
-                            LT_FT(4);
-                            tc_fence_after_sync();
-                            k_next_ready = true;
-                        }
-                        LT_FT(0);
-                        issue_s(t, sn);
-                        LT_FT(6);
-                        const int last_user_next = (j + 1 <= j_last1) ? 1 : 0;
-                        if (t == last_user_next) umma_commit(&sm.bar_k_empty[sn]);
+                if (!ok || *abort_flag) {
+                    // somebody gave up: wait (bounded) for the copies in flight before the CTA exits
+                    for (int t = 0; t < (has_b ? 2 : 1); ++t)
+                        for (int w = 0; w < (1 << 16) && !mbar_try_wait(&sm.bar_q[t], 0); ++w) {}
+                    for (int j = armed > 2 ? armed - 2 : 0; j < armed; ++j) {
+                        for (int w = 0; w < (1 << 16) && !mbar_try_wait(&sm.bar_k_full[j & 1], (j >> 1) & 1); ++w) {}
+                        for (int w = 0; w < (1 << 16) && !mbar_try_wait(&sm.bar_v_full[j & 1], (j >> 1) & 1); ++w) {}
                     }
                 }
             }
-            LT_FT(0);
-            LT_FT_FLUSH(0);
-            LT_FT_COUNT(17, j_end + 1);
-            // every product issued above has finished before tensor memory is released
-            umma_commit(&sm.bar_done);
-            if (!mbar_wait(&sm.bar_done, 0, abort_flag, p.status, kWaitFwdDone))
-                for (int w = 0; w < (1 << 16) && !mbar_try_wait(&sm.bar_done, 0); ++w) {}
+        } else if (warp == 1) {
+            // ------------------------------------------------------------------ MMA issuer
+            if (lane == 0) {
+                // descriptors of slot 0; slot 1 of each ring follows one tile later
+                const uint64_t dQ0 = desc_kmajor(smem_u32(sm.q[0])), dK0 = desc_kmajor(smem_u32(sm.k[0]));
+                const uint64_t dV0 = desc_mnmajor(smem_u32(sm.v[0]), kFwdBoxBytes);
+                constexpr uint64_t kSlotStep = static_cast<uint64_t>(kTileBytes) >> 4;
+                auto koff = [](int kk) -> uint64_t { return static_cast<uint64_t>((kk >> 2) * (kFwdBoxBytes >> 4) + (kk & 3) * 2); };
+                auto roff = [](int kk) -> uint64_t { return static_cast<uint64_t>(kk * (2048 >> 4)); };
+                constexpr uint32_t idesc_s = make_idesc(128, 128, false, false, kBf16);
+                constexpr uint32_t idesc_o = make_idesc(128, D, false, true, kBf16);
+                auto issue_s = [&](int t, int s) {  // S_t = Q_t K^T with the key tile in ring slot s
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk)
+                        umma_ss(tmem + kColS + t * 128, dQ0 + t * kSlotStep + koff(kk), dK0 + s * kSlotStep + koff(kk), idesc_s, kk > 0);
+                    umma_commit(&sm.bar_s_full[t]);
+                };
+                // O_t (+)= P_t V, P_t read from tensor memory; the keys of a tile in two halves of 64, so that the
+                // first half's products run while the softmax warps exponentiate the second half (quarters were
+                // measured too and lost to the extra hand-offs)
+                auto issue_pv_half = [&](int t, int s, bool acc, int half) {
+#pragma unroll
+                    for (int kk = 4 * half; kk < 4 * half + 4; ++kk)
+                        umma_ts(tmem + kColO + t * D, tmem + kColS + t * 128 + kk * 8, dV0 + s * kSlotStep + roff(kk), idesc_o,
+                                acc | (kk > 0));
+                    if (half == 1) umma_commit(&sm.bar_o_done[t]);
+                };
+                bool ok = mbar_wait(&sm.bar_q[0], 0, abort_flag, p.status, kWaitFwdQ) &&
+                          (!has_b || mbar_wait(&sm.bar_q[1], 0, abort_flag, p.status, kWaitFwdQ)) &&
+                          mbar_wait(&sm.bar_k_full[0], 0, abort_flag, p.status, kWaitFwdK);
+                if (ok) {
+                    tc_fence_after_sync();
+                    issue_s(0, 0);
+                    if (has_b) issue_s(1, 0);
+                    umma_commit(&sm.bar_k_empty[0]);
+                }
+                LT_FT_DECL;
+                for (int j = 0; j <= j_end && ok; ++j) {
+                    const int s = j & 1, sn = s ^ 1;
+                    LT_FT(0);
+                    if (!(ok = mbar_wait(&sm.bar_v_full[s], (j >> 1) & 1, abort_flag, p.status, kWaitFwdV))) break;
+                    LT_FT(1);
+                    bool k_next_ready = false;
+#pragma unroll
+                    for (int t = 0; t < 2; ++t) {
+                        const int j_last_t = t == 0 ? j_last0 : j_last1;
+                        if (j > j_last_t) continue;
+                        LT_FT(0);
+                        if (!(ok = mbar_wait(&sm.bar_p_half[t], j & 1, abort_flag, p.status, kWaitFwdP))) break;
+                        tc_fence_after_sync();
+                        issue_pv_half(t, s, j > 0, 0);
+                        if (!(ok = mbar_wait(&sm.bar_p_ready[t], j & 1, abort_flag, p.status, kWaitFwdP))) break;
+                        LT_FT(2 + t);
+                        tc_fence_after_sync();
+                        LT_FT(0);
+                        issue_pv_half(t, s, j > 0, 1);
+                        LT_FT(5);
+                        // the second tile of the pair, when it uses this key tile, uses it last
+                        const int last_user = (j <= j_last1) ? 1 : 0;
+                        if (t == last_user) umma_commit(&sm.bar_v_empty[s]);
+                        if (j + 1 <= j_last_t) {
+                            if (!k_next_ready) {
+                                LT_FT(0);
+                                if (!(ok = mbar_wait(&sm.bar_k_full[sn], ((j + 1) >> 1) & 1, abort_flag, p.status, kWaitFwdK))) break;
+                                LT_FT(4);
+                                tc_fence_after_sync();
+                                k_next_ready = true;
+                            }
+                            LT_FT(0);
+                            issue_s(t, sn);
+                            LT_FT(6);
+                            const int last_user_next = (j + 1 <= j_last1) ? 1 : 0;
+                            if (t == last_user_next) umma_commit(&sm.bar_k_empty[sn]);
+                        }
+                    }
+                }
+                LT_FT(0);
+                LT_FT_FLUSH(0);
+                LT_FT_COUNT(17, j_end + 1);
+                // every product issued above has finished before tensor memory is released
+                umma_commit(&sm.bar_done);
+                if (!mbar_wait(&sm.bar_done, 0, abort_flag, p.status, kWaitFwdDone))
+                    for (int w = 0; w < (1 << 16) && !mbar_try_wait(&sm.bar_done, 0); ++w) {}
+            }
         }
     } else {
         // ------------------------------------------------------------------ softmax warps
+        warpgroup_regs_set<kFwdRegsSoftmax, kFwdRegsAtLaunch>();
         const int t = (warp - kFwdSoftmaxWarp0) >> 2;   // which query tile of the pair
         const int quad = warp & 3;                      // tensor-memory lane quadrant of this warp
         const int row = quad * 32 + lane;               // query row inside the tile
