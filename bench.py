@@ -522,6 +522,20 @@ def run_ours(args, cfg):
                 "value": sub.flops / times[0] / 1e12, "unit": UNIT, "cores": threads, "kind": "oracle",
                 "sample": f"{sub.Hq} query heads ({sub.Hkv} kv groups) of batch 0, full S={cfg.S}, one pass",
                 "seconds": times[0]}
+            # the same oracle pass checks the gradients the timed calls left on the device (the parity tests
+            # compare every unit; this is the benchmark's own record on its sample)
+            import numpy as np
+            errs = {}
+            for name, got, ref in zip(("dQ", "dK", "dV"), (dQ[:1, :sub.Hq], dK[:1, :sub.Hkv], dV[:1, :sub.Hkv]),
+                                      time_oracle.last_result):
+                g = got.cpu().double().numpy()
+                errs[name] = {"rel_fro": float(np.linalg.norm(g - ref) / max(np.linalg.norm(ref), 1e-300)),
+                              "max_abs": float(np.abs(g - ref).max()),
+                              "max_err_over_max_ref": float(np.abs(g - ref).max() / max(np.abs(ref).max(), 1e-300))}
+            line["parity"] = {"against": "fp64 oracle, forward state from lt_attn_fwd", "sample": line["cpu_baseline"]["sample"],
+                              "errors": errs,
+                              "ok": all(e["rel_fro"] <= 5e-3 and e["max_abs"] <= 2e-2 and e["max_err_over_max_ref"] <= 4e-3
+                                        for e in errs.values())}
         print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
