@@ -16,7 +16,9 @@ causal mask see a handful of keys) are measured against a quarter of the root-me
 
 The numbers are two to three times the largest values measured over the whole suite with the fp16
 and bf16 kernels (fp16: elem 1.5e-3, row 2.3e-2, the latter on an early, short row of the largest
-configuration; bf16: elem 4.8e-3, row 3.3e-2); bf16 keeps 8 significant bits where fp16 keeps 11,
+configuration; bf16: elem 4.8e-3, row 3.3e-2 on the fixed cases and 1.2e-1 on one case of the random
+sweep, a softmax flattened by a scale of 0.3/sqrt(D), where a dQ row is the small difference of large
+terms whose bf16 rounding does not shrink with it); bf16 keeps 8 significant bits where fp16 keeps 11,
 which is the factor between the two element bounds.  A wrong value of typical size misses them by a
 wide margin: a typical element is about a quarter of the largest one (60 times the fp16 bound), and
 one such element is 1/sqrt(D) ~ 0.09 of its row's norm, a wrong 16-byte chunk 0.25, a wrong row 1.
@@ -29,7 +31,7 @@ import numpy as np
 REL_FRO_TOL = 5e-3
 MAX_ABS_TOL = 2e-2
 ELEM_TOL = {"fp16": 4e-3, "bf16": 1.6e-2}
-ROW_TOL = {"fp16": 5e-2, "bf16": 1e-1}
+ROW_TOL = {"fp16": 5e-2, "bf16": 2e-1}
 ROW_FLOOR = 0.25
 # an exactly zero gradient (a single visible key) comes out as rounding residue of the -delta split
 ZERO_REF_ABS_TOL = 1e-6
