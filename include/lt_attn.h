@@ -194,7 +194,9 @@ int lt_attn_bwd_bf16(const lt_bf16 *Q, const lt_bf16 *K, const lt_bf16 *V,
  * (B*Hq*nT*nT*32768; 0 for an unsupported shape) and is 256-byte aligned.  Entries hidden by the
  * causal mask or past the end of the sequence are zero; with causal != 0, tiles with i < j are not
  * written and never read.  Q, K, LSE as for lt_attn_bwd (contiguous [B,H,S,D], fp16); `workspace` needs
- * only the 256-byte status block.  One kernel launch.
+ * only the 256-byte status block.  One kernel launch.  lt_attn_save_p stands in for a forward pass that would
+ * write P as it goes (it recomputes the scores from Q, K and LSE); it is there to produce the paper's forward
+ * state for lt_attn_bwd_saved_p, not tuned, and runs at about a third of the HBM write rate of its output.
  *
  * lt_attn_bwd_saved_p computes dQ, dK, dV as lt_attn_bwd does, with `P` (the store above, same shape
  * arguments and mask) in place of LSE: the main kernel issues no S = Q K^T product and no exponentials;
