@@ -23,7 +23,8 @@
 //   warps 4-11   softmax / dS warps: warps 4-7 take query columns 0-63 of a tile pair,
 //                warps 8-11 columns 64-127; each thread owns one key row
 //   warps 12-15  dQ reduction (tensor memory -> shared memory -> bulk add.f32 into the fp32
-//                accumulator) and the per-item dK/dV epilogue
+//                accumulator: linear 8 KB pieces at D = 128, swizzled boxes through a tensor map at
+//                D = 64) and the per-item dK/dV epilogue
 // Transposed scores are used (S^T = K Q^T, dP^T = V dO^T) so that P^T, written back to
 // tensor memory as fp16, is directly the A operand of dV += P^T dO; dS^T is written both to
 // tensor memory (A operand of dK += dS^T Q) and to shared memory (operand of the dQ product).
@@ -347,7 +348,8 @@ struct BwdSmem {
     uint8_t ext_zero[kExtBytes];       // contraction elements 8-15 of all of the above
     // staging of the dQ partial for bulk reduction into global memory (D = 128 only):
     // each buffer holds 16 accumulator rows (16 query rows x 128 floats)
-    float dq_stage[D == 128 ? kDqStageBufs : 1][D == 128 ? kDqStageRows * 128 : 4];
+    // (D = 64: two buffers of a whole partial, 128 query rows x 64 floats, each as two swizzled boxes of 32 columns)
+    float dq_stage[D == 128 ? kDqStageBufs : 2][D == 128 ? kDqStageRows * 128 : kTileRows * 64];
     // per work item: K/V landed; dK/dV accumulators complete; accumulators read out
     uint64_t bar_kv, bar_dkv_full, bar_acc_free;
     // work items are claimed from a global counter by the producer and published to the other roles
@@ -470,7 +472,8 @@ template <int D, bool kBf16, bool kSplit, bool kSavedP = false>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
-                const BwdParams p) {
+                const BwdParams p, const __grid_constant__ CUtensorMap map_dq) {
+    // map_dq (D = 64 only): the fp32 dQ accumulator as rows of 64 floats, boxes of 128 rows x 32 columns
     using Smem = BwdSmem<D>;
     constexpr int kBoxes = D / 64;
     constexpr uint32_t kTileBytes = kBoxes * kBoxBytesBwd;
@@ -925,7 +928,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             // the four reduction warps share named barriers (D = 128), so after every wait they vote
             // and leave together
             ok = ok && LT_WAIT(&sm.bar_item[ic % kItemRing], (ic / kItemRing) & 1, kWaitItem);
-            if constexpr (D == 128) ok = named_barrier_and(kBarReduceWarps, kNumReduceWarps * 32, ok);
+            ok = named_barrier_and(kBarReduceWarps, kNumReduceWarps * 32, ok);
             if (!ok) break;
             const int item = sm.item_ring[ic % kItemRing];
             if (item < 0) break;
@@ -934,7 +937,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 ok = LT_WAIT(&sm.bar_dq_full, it & 1, kWaitDqFull);
                 // the four reduction warps share named barriers below, so they leave the loop together;
                 // the vote also tells them that the staging buffers of the previous tile are free
-                if constexpr (D == 128) ok = named_barrier_and(kBarReduceWarps, kNumReduceWarps * 32, ok);
+                ok = named_barrier_and(kBarReduceWarps, kNumReduceWarps * 32, ok);
                 if (!ok) break;
                 tc_fence_after_sync();
                 LT_TRACE_MARK(tr0);
@@ -997,35 +1000,40 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     stage_rows(7, r0 + 16);
                     if (elected) bulk_wait_group_read<0>();
                 } else {
-                    // D = 64: dQ partial with lanes = query rows; four neighbouring threads add 32
-                    // contiguous bytes of one query row
+                    // D = 64: dQ partial with lanes = query rows.  A thread holds the 64 floats of one query row.
+                    // The partial is scaled and staged in shared memory as two boxes of 128 rows x 32 floats with
+                    // the 128-byte swizzle (rows 128 bytes apart: the swizzle spreads a warp's 16-byte stores over
+                    // all banks), and two tiled reductions add the boxes to the accumulator; two staging buffers.
+                    const int q_row = quad * 32 + lane;
+                    const uint32_t taddr = tmem + (static_cast<uint32_t>(quad * 32) << 16) + kColdP;
+                    const bool elected = (warp == kReduceWarp0) && (lane == 0);
+                    uint32_t r[2][32];
+                    tmem_ld32(taddr, r[0]);
+                    tmem_ld32(taddr + 32, r[1]);
+                    tmem_wait_ld();
+                    // the whole partial is in registers: the dP columns may be overwritten
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm.bar_dq_empty);
+                    LT_TRACE_SINCE(12, tr0);
+                    // the buffer of this tile was last read by the reductions issued two tiles ago
+                    if (elected) bulk_wait_group_read<1>();
+                    named_barrier_sync(kBarReduceWarps, kNumReduceWarps * 32);
+                    uint8_t *buf = reinterpret_cast<uint8_t *>(sm.dq_stage[it & 1]);
 #pragma unroll
-                    for (int ch = 0; ch < D / 64; ++ch) {
-                        uint32_t r[2][32];
+                    for (int bx = 0; bx < 2; ++bx)
 #pragma unroll
-                        for (int lh = 0; lh < 2; ++lh)
-                            tmem_ld_16x256b_x8(tmem + (static_cast<uint32_t>(quad * 32 + lh * 16) << 16) + kColdP + ch * 64,
-                                               r[lh]);
-                        tmem_wait_ld();
-                        if (ch == D / 64 - 1) {
-                            // the whole partial is in registers: the dP columns may be overwritten
-                            tc_fence_before_sync();
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(&sm.bar_dq_empty);
-                            LT_TRACE_SINCE(12, tr0);
-                        }
-#pragma unroll
-                        for (int lh = 0; lh < 2; ++lh) {
-                            float *base = dq_tile + static_cast<long long>(quad * 32 + lh * 16 + (lane >> 2)) * D +
-                                          ch * 64 + 2 * (lane & 3);
-#pragma unroll
-                            for (int k = 0; k < 8; ++k) {
-                                red_add_v2(base + 8 * k, __uint_as_float(r[lh][4 * k]) * dq_mult,
-                                           __uint_as_float(r[lh][4 * k + 1]) * dq_mult);
-                                red_add_v2(base + 8 * D + 8 * k, __uint_as_float(r[lh][4 * k + 2]) * dq_mult,
-                                           __uint_as_float(r[lh][4 * k + 3]) * dq_mult);
-                            }
-                        }
+                        for (int c = 0; c < 8; ++c)
+                            *reinterpret_cast<float4 *>(buf + bx * (kTileRows * 128) + q_row * 128 + ((c ^ (q_row & 7)) << 4)) =
+                                make_float4(__uint_as_float(r[bx][4 * c]) * dq_mult, __uint_as_float(r[bx][4 * c + 1]) * dq_mult,
+                                            __uint_as_float(r[bx][4 * c + 2]) * dq_mult, __uint_as_float(r[bx][4 * c + 3]) * dq_mult);
+                    fence_proxy_async_smem();
+                    named_barrier_sync(kBarReduceWarps, kNumReduceWarps * 32);
+                    if (elected) {
+                        const int y = static_cast<int>(bwd_q_tile(p, w, n).padded_row0);
+                        tma_reduce_add_2d(&map_dq, buf, 0, y);
+                        tma_reduce_add_2d(&map_dq, buf + kTileRows * 128, 32, y);
+                        bulk_commit_group();
                     }
                 }
                 LT_TRACE_SINCE(13, tr0);
@@ -1034,7 +1042,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             // item epilogue (these warps are idle while the pipeline of the next item fills):
             // dK_j and dV_j leave tensor memory as fp16; thread = key row
             ok = LT_WAIT(&sm.bar_dkv_full, ic & 1, kWaitDkvFull);
-            if constexpr (D == 128) ok = named_barrier_and(kBarReduceWarps, kNumReduceWarps * 32, ok);
+            ok = named_barrier_and(kBarReduceWarps, kNumReduceWarps * 32, ok);
             if (!ok) break;
             tc_fence_after_sync();
             {
@@ -1086,7 +1094,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             }
         }
         // shared memory must stay valid until the bulk reductions have read it
-        if constexpr (D == 128) bulk_wait_group_all();
+        bulk_wait_group_all();
         LT_TRACE_END(kRoleReduce);
 #ifdef LT_BWD_TRACE
         trace_iters = it;
@@ -1259,7 +1267,10 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
     cfg_main.stream = stream;
     cfg_main.attrs = &pdl;
     cfg_main.numAttrs = 1;
-    e = cudaLaunchKernelEx(&cfg_main, main_kernel, mq, mk, mv, mdo, prm);
+    CUtensorMap mdq = mq;  // (D = 128 never touches it)
+    if constexpr (D == 64)
+        if ((rc = make_f32_tile_map(&mdq, dq_acc, static_cast<uint64_t>(n_rows), 64, 128)) != LT_OK) return rc;
+    e = cudaLaunchKernelEx(&cfg_main, main_kernel, mq, mk, mv, mdo, prm, mdq);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return record_cuda_error("bwd_main_kernel launch", e);
     if (ev_main_end && (e = cudaEventRecord(ev_main_end, stream)) != cudaSuccess)

@@ -187,6 +187,15 @@ __device__ __forceinline__ void bulk_reduce_add_f32(float *dst_gmem, const void 
                  "r"(smem_u32(src_smem)), "r"(bytes)
                  : "memory");
 }
+// 2-D tiled reduction shared -> global through a tensor map: adds the box at (x, y) (x = innermost element
+// coordinate, x * element size a multiple of 16 bytes; both coordinates non-negative) of fp32 values from shared
+// memory, laid out with the map's swizzle, into global memory.  Completion is tracked in bulk groups like above.
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap *map, const void *src_smem, int x, int y) {
+    asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];" ::"l"(
+                     reinterpret_cast<uint64_t>(map)),
+                 "r"(smem_u32(src_smem)), "r"(x), "r"(y)
+                 : "memory");
+}
 __device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void bulk_wait_group_read() {

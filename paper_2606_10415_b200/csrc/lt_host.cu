@@ -103,6 +103,25 @@ int make_bhsd_map(CUtensorMap *map, const void *base, uint64_t B, uint64_t H, ui
     return LT_OK;
 }
 
+int make_f32_tile_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    EncodeTiledFn enc = get_encoder();
+    if (!enc) return LT_ERR_CUDA;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * sizeof(float)};
+    cuuint32_t box[2] = {32u, box_rows};
+    cuuint32_t estr[2] = {1u, 1u};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void *>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        char buf[64];
+        snprintf(buf, sizeof(buf), "CUresult %d", static_cast<int>(r));
+        set_last_error("cuTensorMapEncodeTiled(f32)", buf);
+        return LT_ERR_CUDA;
+    }
+    return LT_OK;
+}
+
 lt_attn_layout contiguous_layout(int Hq, int Hkv, int S, int D) {
     lt_attn_layout lay;
     lay.q = lay.o = lay.d_o = lay.dq = contiguous_strides(Hq, S, D);

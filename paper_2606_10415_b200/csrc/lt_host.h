@@ -33,6 +33,9 @@ int make_tile_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t co
 // 64 elements x box_rows rows of one head, 128-byte swizzle, zero fill past the last row).
 int make_bhsd_map(CUtensorMap *map, const void *base, uint64_t B, uint64_t H, uint64_t S, uint64_t D,
                   const lt_tensor_strides &st, uint32_t box_rows, bool bf16 = false);
+// fp32 matrix [rows, cols] row-major (cols a multiple of 32) viewed as a 2-D tensor; tiles of box_rows x 32
+// columns (128 bytes per row) with the 128-byte swizzle, for tiled reductions from shared memory.
+int make_f32_tile_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows);
 // strides of a contiguous [B,H,S,D] tensor
 inline lt_tensor_strides contiguous_strides(int H, int S, int D) {
     lt_tensor_strides st;
