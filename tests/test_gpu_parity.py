@@ -517,6 +517,33 @@ def test_other_sequence_lengths_and_unmasked(lt, oracle, name):
     _full_size_check(lt, oracle, name)
 
 
+# ------------------------------------------------------------------ head dimension 64 at length
+
+@pytest.mark.parametrize("B,Hq,Hkv,S,causal,bf16", [
+    (1, 8, 8, 2048, True, False),    # 16 key tiles per head: long dQ accumulation chains through the tiled reductions
+    (2, 8, 2, 1900, True, True),     # grouped heads, ragged last tile, bf16
+    (1, 4, 4, 1536, False, False),   # no mask
+])
+def test_head_dim_64_matches_oracle(lt, oracle, B, Hq, Hkv, S, causal, bf16):
+    """D = 64 takes its own dQ path (swizzled staging, tiled reductions through a tensor map over the
+    accumulator); every unit is compared."""
+    cfg = workloads.custom(B, Hq, Hkv, S, 64, causal, seed=91 + S)
+    dt = torch.bfloat16 if bf16 else torch.float16
+    Q, K, V, dO = (t.float().to(dt) for t in workloads.make_inputs(cfg))
+    Qn, Kn, Vn, dOn = (t.double().numpy() for t in (Q, K, V, dO))
+    O_ref, LSE_ref = oracle.attn_fwd(Qn, Kn, Vn, causal, cfg.scale)
+    ref = oracle.attn_bwd(Qn, Kn, Vn, dOn, causal, cfg.scale)
+    Qd, Kd, Vd, dOd = (t.cuda() for t in (Q, K, V, dO))
+    Od = torch.from_numpy(O_ref).to(dt).cuda()
+    dQ, dK, dV = (torch.full_like(t, float("nan")) for t in (Qd, Kd, Vd))
+    ws = lt.alloc_workspace(lt.lt_attn_bwd_workspace_bytes(B, Hq, Hkv, S, 64))
+    ws.fill_(0xFF)
+    bwd = lt.lt_attn_bwd_bf16 if bf16 else lt.lt_attn_bwd
+    bwd(Qd, Kd, Vd, Od, dOd, torch.from_numpy(LSE_ref).float().cuda(), dQ, dK, dV, causal, cfg.scale, ws)
+    assert lt.lt_attn_check_status(ws) == lt.LT_OK, lt.last_cuda_error()
+    check_grads((dQ, dK, dV), ref, f"D=64 {cfg} bf16={bf16}", dtype="bf16" if bf16 else "fp16")
+
+
 # ------------------------------------------------------------------ split-group variant
 
 # Shapes with few, heavy work items: a group's query heads are spread over several items per key tile
