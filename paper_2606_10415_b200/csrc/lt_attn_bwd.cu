@@ -314,6 +314,8 @@ __device__ __forceinline__ bool traced_wait(Trace &tr, uint64_t *bar, uint32_t p
 #define LT_TRACE_END(role)
 #define LT_WAIT(bar, parity, code) mbar_wait(bar, parity, abort_flag, p.status, code)
 #endif
+// the same wait by every lane of a warp, with the outcome voted (warp-uniform)
+#define LT_WAIT_ALL(bar, parity, code) __all_sync(0xffffffffu, LT_WAIT(bar, parity, code))
 
 // ----------------------------------------------------------------------------- main kernel
 constexpr int kQStages = 2;   // Q_i ring; dO_i is single-buffered (it is dead once dV has been issued)
@@ -633,7 +635,10 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             __syncwarp();
         } else if (warp == 1) {
             // ================================================================= tensor-core issuer
-            if (lane == 0 && smem_ok) {
+            // The whole warp walks the loop, so that loop counters, wait results (voted) and descriptor arithmetic are
+            // warp-uniform; one elected lane issues the products and commits.
+            if (smem_ok) {
+                const bool leader = elect_one();
                 LT_TRACE_BEGIN();
                 // Every operand descriptor is a compile-time constant (built from the operand's offset inside
                 // the shared window) plus the window's base in the address field (bits 0-13, units of 16
@@ -670,6 +675,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 constexpr uint32_t idesc_dv = make_idesc(128, D, false, true, kBf16);
                 constexpr uint32_t idesc_dq = make_idesc(128, D == 128 ? 128 : D, true, true, kBf16);
                 auto issue_s = [&](int t) {  // S^T = K_j Q_i^T - LSE_i / scale, for running iteration t
+                    if (!leader) return;
                     const uint64_t wb = window_base();
                     const uint64_t dQ_k = wb + (t & 1) * kQStageStep;
 #pragma unroll
@@ -681,12 +687,12 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 bool ok = true;
                 int it = 0, ic = 0;
                 for (;; ++ic) {
-                    if (!(ok = LT_WAIT(&sm.bar_item[ic % kItemRing], (ic / kItemRing) & 1, kWaitItem))) break;
+                    if (!(ok = LT_WAIT_ALL(&sm.bar_item[ic % kItemRing], (ic / kItemRing) & 1, kWaitItem))) break;
                     const int item = sm.item_ring[ic % kItemRing];
                     if (item < 0) break;
                     const BwdItem w = bwd_item<kSplit>(p, item);
-                    ok = LT_WAIT(&sm.bar_kv, ic & 1, kWaitKV) &&
-                         LT_WAIT(&sm.bar_q_full[it & 1], (it >> 1) & 1, kWaitStageFull);
+                    ok = LT_WAIT_ALL(&sm.bar_kv, ic & 1, kWaitKV) &&
+                         LT_WAIT_ALL(&sm.bar_q_full[it & 1], (it >> 1) & 1, kWaitStageFull);
                     if (!ok) break;
                     tc_fence_after_sync();
                     if constexpr (!kSavedP) issue_s(it);
@@ -695,10 +701,11 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         const uint64_t wb = window_base();
                         const uint64_t dQ_mn = wb + s * kQStageStep;
                         // dO_i and the -delta rows have landed: both dP and dV read them
-                        if (!(ok = LT_WAIT(&sm.bar_do_full, it & 1, kWaitDoFull))) break;
+                        if (!(ok = LT_WAIT_ALL(&sm.bar_do_full, it & 1, kWaitDoFull))) break;
                         // dP^T = V_j dO_i^T - delta_i   (its columns held the previous dQ partial until the
                         //                                reduce warps drained it)
                         auto issue_dp = [&]() {
+                            if (!leader) return;
 #pragma unroll
                             for (int kk = 0; kk < D / 16; ++kk)
                                 umma_ss(tmem + kColdP, wb + (dV_k + koff(kk)), wb + (ddO_k + koff(kk)), idesc_s, kk > 0);
@@ -713,50 +720,55 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         // dV_j += P'^T dO_i   (A = P'^T from tensor memory; query columns 0-63 sit at columns
                         //                      0-31, query columns 64-127 at columns 64-95 of the S region)
                         auto issue_dv = [&]() {
+                            if (!leader) return;
 #pragma unroll
                             for (int kk = 0; kk < 8; ++kk)
                                 umma_ts(tmem + kColdV, tmem + kColS + (kk >> 2) * 64 + (kk & 3) * 8, wb + (ddO_mn + roff(kk)),
                                         idesc_dv, (n > 0) | (kk > 0));
                         };
-                        if (it > 0 && !(ok = LT_WAIT(&sm.bar_dq_empty, (it - 1) & 1, kWaitDqEmpty))) break;
+                        if (it > 0 && !(ok = LT_WAIT_ALL(&sm.bar_dq_empty, (it - 1) & 1, kWaitDqEmpty))) break;
                         tc_fence_after_sync();
                         issue_dp();
-                        if (!(ok = LT_WAIT(&sm.bar_p_ready, it & 1, kWaitPReady))) break;
+                        if (!(ok = LT_WAIT_ALL(&sm.bar_p_ready, it & 1, kWaitPReady))) break;
                         // the first product of an item overwrites accumulators the previous item's epilogue reads
-                        if (n == 0 && ic > 0 && !(ok = LT_WAIT(&sm.bar_acc_free, (ic - 1) & 1, kWaitAccFree))) break;
+                        if (n == 0 && ic > 0 && !(ok = LT_WAIT_ALL(&sm.bar_acc_free, (ic - 1) & 1, kWaitAccFree))) break;
                         tc_fence_after_sync();
                         issue_dv();
-                        umma_commit(&sm.bar_do_empty);
+                        if (leader) umma_commit(&sm.bar_do_empty);
                         // the next S^T overwrites P'^T; the tensor pipe executes in issue order
                         if (n + 1 < w.n_iter) {
-                            if (!(ok = LT_WAIT(&sm.bar_q_full[(it + 1) & 1], ((it + 1) >> 1) & 1, kWaitStageFull))) break;
+                            if (!(ok = LT_WAIT_ALL(&sm.bar_q_full[(it + 1) & 1], ((it + 1) >> 1) & 1, kWaitStageFull))) break;
                             if constexpr (!kSavedP) issue_s(it + 1);
                         }
-                        if (!(ok = LT_WAIT(&sm.bar_ds_ready, it & 1, kWaitDsReady))) break;
+                        if (!(ok = LT_WAIT_ALL(&sm.bar_ds_ready, it & 1, kWaitDsReady))) break;
                         tc_fence_after_sync();
                         // dK_j += dS'^T Q_i   (A = dS'^T from tensor memory, stored like P'^T: query columns
                         //                       0-63 at columns 0-31 and 64-127 at columns 64-95 of the dP region)
+                        if (leader) {
 #pragma unroll
-                        for (int kk = 0; kk < 8; ++kk)
-                            umma_ts(tmem + kColdK, tmem + kColdP + (kk >> 2) * 64 + (kk & 3) * 8, dQ_mn + (dQ_mn0 + roff(kk)), idesc_dv,
-                                    (n > 0) | (kk > 0));
-                        umma_commit(&sm.bar_q_empty[s]);
+                            for (int kk = 0; kk < 8; ++kk)
+                                umma_ts(tmem + kColdK, tmem + kColdP + (kk >> 2) * 64 + (kk & 3) * 8, dQ_mn + (dQ_mn0 + roff(kk)), idesc_dv,
+                                        (n > 0) | (kk > 0));
+                            umma_commit(&sm.bar_q_empty[s]);
+                        }
                         // dQ_i partial (contraction over key rows); it overwrites the dP columns, which is safe
                         // after dK because the tensor pipe executes in issue order.  For D = 128 it is
                         // produced transposed, dQ^T = K_j^T dS^T (lanes = head dim, columns = query rows), so
                         // that the reduction moves whole accumulator rows; for D = 64 as dQ = dS K_j.
+                        if (leader) {
 #pragma unroll
-                        for (int kk = 0; kk < 8; ++kk) {
-                            if constexpr (D == 128)
-                                umma_ss(tmem + kColdP, wb + (dK_mn + roff(kk)), wb + (ddS_mn + roff(kk)), idesc_dq, kk > 0);
-                            else
-                                umma_ss(tmem + kColdP, wb + (ddS_mn + roff(kk)), wb + (dK_mn + roff(kk)), idesc_dq, kk > 0);
+                            for (int kk = 0; kk < 8; ++kk) {
+                                if constexpr (D == 128)
+                                    umma_ss(tmem + kColdP, wb + (dK_mn + roff(kk)), wb + (ddS_mn + roff(kk)), idesc_dq, kk > 0);
+                                else
+                                    umma_ss(tmem + kColdP, wb + (ddS_mn + roff(kk)), wb + (dK_mn + roff(kk)), idesc_dq, kk > 0);
+                            }
+                            umma_commit(&sm.bar_dq_full);
+                            umma_commit(&sm.bar_ds_free);
                         }
-                        umma_commit(&sm.bar_dq_full);
-                        umma_commit(&sm.bar_ds_free);
                     }
                     if (!ok) break;
-                    umma_commit(&sm.bar_dkv_full);
+                    if (leader) umma_commit(&sm.bar_dkv_full);
                 }
                 LT_TRACE_END(kRoleMma);
             }
