@@ -184,7 +184,13 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
             }
         } else if (warp == 1) {
             // ------------------------------------------------------------------ MMA issuer
-            if (lane == 0) {
+            // The whole warp walks the loop, so that counters, wait results (voted) and descriptor arithmetic are
+            // warp-uniform; one elected lane issues the products and commits.
+            {
+                const bool leader = elect_one();
+                auto wait_all = [&](uint64_t *bar, uint32_t parity, int code) {
+                    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, p.status, code));
+                };
                 // descriptors of slot 0; slot 1 of each ring follows one tile later
                 const uint64_t dQ0 = desc_kmajor(smem_u32(sm.q[0])), dK0 = desc_kmajor(smem_u32(sm.k[0]));
                 const uint64_t dV0 = desc_mnmajor(smem_u32(sm.v[0]), kFwdBoxBytes);
@@ -194,6 +200,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
                 constexpr uint32_t idesc_s = make_idesc(128, 128, false, false, kBf16);
                 constexpr uint32_t idesc_o = make_idesc(128, D, false, true, kBf16);
                 auto issue_s = [&](int t, int s) {  // S_t = Q_t K^T with the key tile in ring slot s
+                    if (!leader) return;
 #pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk)
                         umma_ss(tmem + kColS + t * 128, dQ0 + t * kSlotStep + koff(kk), dK0 + s * kSlotStep + koff(kk), idesc_s, kk > 0);
@@ -203,26 +210,27 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
                 // first half's products run while the softmax warps exponentiate the second half (quarters were
                 // measured too and lost to the extra hand-offs)
                 auto issue_pv_half = [&](int t, int s, bool acc, int half) {
+                    if (!leader) return;
 #pragma unroll
                     for (int kk = 4 * half; kk < 4 * half + 4; ++kk)
                         umma_ts(tmem + kColO + t * D, tmem + kColS + t * 128 + kk * 8, dV0 + s * kSlotStep + roff(kk), idesc_o,
                                 acc | (kk > 0));
                     if (half == 1) umma_commit(&sm.bar_o_done[t]);
                 };
-                bool ok = mbar_wait(&sm.bar_q[0], 0, abort_flag, p.status, kWaitFwdQ) &&
-                          (!has_b || mbar_wait(&sm.bar_q[1], 0, abort_flag, p.status, kWaitFwdQ)) &&
-                          mbar_wait(&sm.bar_k_full[0], 0, abort_flag, p.status, kWaitFwdK);
+                bool ok = wait_all(&sm.bar_q[0], 0, kWaitFwdQ) &&
+                          (!has_b || wait_all(&sm.bar_q[1], 0, kWaitFwdQ)) &&
+                          wait_all(&sm.bar_k_full[0], 0, kWaitFwdK);
                 if (ok) {
                     tc_fence_after_sync();
                     issue_s(0, 0);
                     if (has_b) issue_s(1, 0);
-                    umma_commit(&sm.bar_k_empty[0]);
+                    if (leader) umma_commit(&sm.bar_k_empty[0]);
                 }
                 LT_FT_DECL;
                 for (int j = 0; j <= j_end && ok; ++j) {
                     const int s = j & 1, sn = s ^ 1;
                     LT_FT(0);
-                    if (!(ok = mbar_wait(&sm.bar_v_full[s], (j >> 1) & 1, abort_flag, p.status, kWaitFwdV))) break;
+                    if (!(ok = wait_all(&sm.bar_v_full[s], (j >> 1) & 1, kWaitFwdV))) break;
                     LT_FT(1);
                     bool k_next_ready = false;
 #pragma unroll
@@ -230,10 +238,10 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
                         const int j_last_t = t == 0 ? j_last0 : j_last1;
                         if (j > j_last_t) continue;
                         LT_FT(0);
-                        if (!(ok = mbar_wait(&sm.bar_p_half[t], j & 1, abort_flag, p.status, kWaitFwdP))) break;
+                        if (!(ok = wait_all(&sm.bar_p_half[t], j & 1, kWaitFwdP))) break;
                         tc_fence_after_sync();
                         issue_pv_half(t, s, j > 0, 0);
-                        if (!(ok = mbar_wait(&sm.bar_p_ready[t], j & 1, abort_flag, p.status, kWaitFwdP))) break;
+                        if (!(ok = wait_all(&sm.bar_p_ready[t], j & 1, kWaitFwdP))) break;
                         LT_FT(2 + t);
                         tc_fence_after_sync();
                         LT_FT(0);
@@ -241,11 +249,11 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
                         LT_FT(5);
                         // the second tile of the pair, when it uses this key tile, uses it last
                         const int last_user = (j <= j_last1) ? 1 : 0;
-                        if (t == last_user) umma_commit(&sm.bar_v_empty[s]);
+                        if (t == last_user && leader) umma_commit(&sm.bar_v_empty[s]);
                         if (j + 1 <= j_last_t) {
                             if (!k_next_ready) {
                                 LT_FT(0);
-                                if (!(ok = mbar_wait(&sm.bar_k_full[sn], ((j + 1) >> 1) & 1, abort_flag, p.status, kWaitFwdK))) break;
+                                if (!(ok = wait_all(&sm.bar_k_full[sn], ((j + 1) >> 1) & 1, kWaitFwdK))) break;
                                 LT_FT(4);
                                 tc_fence_after_sync();
                                 k_next_ready = true;
@@ -254,7 +262,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
                             issue_s(t, sn);
                             LT_FT(6);
                             const int last_user_next = (j + 1 <= j_last1) ? 1 : 0;
-                            if (t == last_user_next) umma_commit(&sm.bar_k_empty[sn]);
+                            if (t == last_user_next && leader) umma_commit(&sm.bar_k_empty[sn]);
                         }
                     }
                 }
@@ -262,8 +270,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CU
                 LT_FT_FLUSH(0);
                 LT_FT_COUNT(17, j_end + 1);
                 // every product issued above has finished before tensor memory is released
-                umma_commit(&sm.bar_done);
-                if (!mbar_wait(&sm.bar_done, 0, abort_flag, p.status, kWaitFwdDone))
+                if (leader) umma_commit(&sm.bar_done);
+                if (!wait_all(&sm.bar_done, 0, kWaitFwdDone))
                     for (int w = 0; w < (1 << 16) && !mbar_try_wait(&sm.bar_done, 0); ++w) {}
             }
         }
