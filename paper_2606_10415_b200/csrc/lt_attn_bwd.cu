@@ -317,6 +317,17 @@ __device__ __forceinline__ bool traced_wait(Trace &tr, uint64_t *bar, uint32_t p
 // the same wait by every lane of a warp, with the outcome voted (warp-uniform)
 #define LT_WAIT_ALL(bar, parity, code) __all_sync(0xffffffffu, LT_WAIT(bar, parity, code))
 
+// Built only with -DLT_BWD_TIMELINE=<cta> (development aid): clock stamps of that CTA's first 256 iterations.
+#ifdef LT_BWD_TIMELINE
+__device__ long long g_bwd_timeline[16 * 256];
+#define LT_TL(cond, ev, iter)                                                                        \
+    do {                                                                                             \
+        if ((cond) && blockIdx.x == LT_BWD_TIMELINE && (iter) < 256) g_bwd_timeline[(ev) * 256 + (iter)] = clock64(); \
+    } while (0)
+#else
+#define LT_TL(cond, ev, iter) do {} while (0)
+#endif
+
 // ----------------------------------------------------------------------------- main kernel
 constexpr int kQStages = 2;   // Q_i ring; dO_i is single-buffered (it is dead once dV has been issued)
 constexpr int kBwdThreads = 512;  // 16 warps; 128 registers per thread at launch
@@ -324,7 +335,7 @@ constexpr int kComputeWarp0 = 4, kNumComputeWarps = 8;
 constexpr int kReduceWarp0 = 12, kNumReduceWarps = 4;
 // registers per thread once the warpgroups have resized their shares (the SM has 64 K)
 constexpr int kRegsAtLaunch = 65536 / kBwdThreads;
-constexpr int kRegsControl = 56, kRegsCompute = 168, kRegsReduce = 120;
+constexpr int kRegsControl = 56, kRegsCompute = 160, kRegsReduce = 136;
 static_assert(128 * kRegsControl + kNumComputeWarps * 32 * kRegsCompute + kNumReduceWarps * 32 * kRegsReduce <= 65536,
               "register shares exceed the register file");
 constexpr int kDqStageBufs = 3, kDqStageRows = 16;
@@ -726,10 +737,14 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                                 umma_ts(tmem + kColdV, tmem + kColS + (kk >> 2) * 64 + (kk & 3) * 8, wb + (ddO_mn + roff(kk)),
                                         idesc_dv, (n > 0) | (kk > 0));
                         };
+                        LT_TL(leader, 0, it);
                         if (it > 0 && !(ok = LT_WAIT_ALL(&sm.bar_dq_empty, (it - 1) & 1, kWaitDqEmpty))) break;
                         tc_fence_after_sync();
+                        LT_TL(leader, 1, it);
                         issue_dp();
+                        LT_TL(leader, 2, it);
                         if (!(ok = LT_WAIT_ALL(&sm.bar_p_ready, it & 1, kWaitPReady))) break;
+                        LT_TL(leader, 3, it);
                         // the first product of an item overwrites accumulators the previous item's epilogue reads
                         if (n == 0 && ic > 0 && !(ok = LT_WAIT_ALL(&sm.bar_acc_free, (ic - 1) & 1, kWaitAccFree))) break;
                         tc_fence_after_sync();
@@ -740,8 +755,10 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                             if (!(ok = LT_WAIT_ALL(&sm.bar_q_full[(it + 1) & 1], ((it + 1) >> 1) & 1, kWaitStageFull))) break;
                             if constexpr (!kSavedP) issue_s(it + 1);
                         }
+                        LT_TL(leader, 4, it);
                         if (!(ok = LT_WAIT_ALL(&sm.bar_ds_ready, it & 1, kWaitDsReady))) break;
                         tc_fence_after_sync();
+                        LT_TL(leader, 5, it);
                         // dK_j += dS'^T Q_i   (A = dS'^T from tensor memory, stored like P'^T: query columns
                         //                       0-63 at columns 0-31 and 64-127 at columns 64-95 of the dP region)
                         if (leader) {
@@ -766,6 +783,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                             umma_commit(&sm.bar_dq_full);
                             umma_commit(&sm.bar_ds_free);
                         }
+                        LT_TL(leader, 6, it);
                     }
                     if (!ok) break;
                     if (leader) umma_commit(&sm.bar_dkv_full);
@@ -824,6 +842,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             }
             if (!LT_WAIT(&sm.bar_s_full, t & 1, kWaitSFull)) return false;
             tc_fence_after_sync();
+            LT_TL(tid == kComputeWarp0 * 32, 7, t);
             LT_TRACE_MARK(tp0);
             const int hh = n / w.tiles_per_head;
             const bool diag = p.causal && (w.i_first + (n - hh * w.tiles_per_head) == w.j);
@@ -862,6 +881,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.bar_p_ready);
+            LT_TL(tid == kComputeWarp0 * 32, 8, t);
             LT_TRACE_SINCE(12, tp0);
             return true;
         };
@@ -878,6 +898,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     if (n + 1 < w.n_iter) load_saved_p(w, n + 1, pn);
                 if (!(ok = LT_WAIT(&sm.bar_dp_full, it & 1, kWaitDpFull))) break;
                 tc_fence_after_sync();
+                LT_TL(tid == kComputeWarp0 * 32, 9, it);
                 // the previous dS^T tile must have been consumed by the dQ product before it is overwritten
                 if (it > 0 && !(ok = LT_WAIT(&sm.bar_ds_free, (it - 1) & 1, kWaitDsFree))) break;
                 LT_TRACE_MARK(td0);
@@ -916,6 +937,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sm.bar_ds_ready);
+                LT_TL(tid == kComputeWarp0 * 32, 10, it);
                 LT_TRACE_SINCE(14, td0);
                 if constexpr (kSavedP) {
 #pragma unroll
@@ -935,6 +957,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const float dq_mult = p.scale * inv_p_scale;
         bool ok = smem_ok;
         int it = 0, ic = 0;
+        uint32_t gq = 0;  // running number of the sixteen-row groups staged so far (D = 128)
         LT_TRACE_BEGIN();
         for (;; ++ic) {
             // the four reduction warps share named barriers (D = 128), so after every wait they vote
@@ -947,11 +970,16 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             const BwdItem w = bwd_item<kSplit>(p, item);
             for (int n = 0; n < w.n_iter; ++n, ++it) {
                 ok = LT_WAIT(&sm.bar_dq_full, it & 1, kWaitDqFull);
-                // the four reduction warps share named barriers below, so they leave the loop together;
-                // the vote also tells them that the staging buffers of the previous tile are free
+                // The four reduction warps share named barriers below, so they leave the loop together.  The
+                // staging buffers form a ring that runs on across tile pairs (running group number gq): at
+                // most the last two reductions of the previous pair are still reading their buffers here,
+                // the buffer the first group of this pair goes to is free.
+                if constexpr (D == 128)
+                    if (warp == kReduceWarp0 && lane == 0) bulk_wait_group_read<2>();
                 ok = named_barrier_and(kBarReduceWarps, kNumReduceWarps * 32, ok);
                 if (!ok) break;
                 tc_fence_after_sync();
+                LT_TL(tid == kReduceWarp0 * 32, 11, it);
                 LT_TRACE_MARK(tr0);
                 float *dq_tile = p.dq_acc + bwd_q_tile(p, w, n).padded_row0 * D;
                 if constexpr (D == 128) {
@@ -963,39 +991,39 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     const uint32_t taddr = tmem + (static_cast<uint32_t>(quad * 32) << 16) + kColdP;
                     const bool elected = (warp == kReduceWarp0) && (lane == 0);
                     auto store_rows = [&](int k, const uint32_t *r) {  // r: 16 values, query rows 16k .. 16k+15
-                        float *buf = sm.dq_stage[k % kDqStageBufs];
+                        float *buf = sm.dq_stage[(gq + k) % kDqStageBufs];
 #pragma unroll
                         for (int e = 0; e < kDqStageRows; ++e) buf[e * 128 + d_idx] = __uint_as_float(r[e]) * dq_mult;
                     };
                     auto add_rows = [&](int k) {
-                        bulk_reduce_add_f32(dq_tile + k * kDqStageRows * 128, sm.dq_stage[k % kDqStageBufs],
+                        bulk_reduce_add_f32(dq_tile + k * kDqStageRows * 128, sm.dq_stage[(gq + k) % kDqStageBufs],
                                             kDqStageRows * 128 * sizeof(float));
                         bulk_commit_group();
                     };
-                    // All staging buffers are free here (the elected thread waited for its bulk reductions
-                    // before the vote above).  Three quarters of the partial are read, two groups of rows
-                    // are parked in shared memory to make room for the last quarter, and the dP columns
-                    // are released before any reduction is issued.
-                    uint32_t r0[32], r1[32], r2[32];
-                    tmem_ld32(taddr, r0);
+                    // Seven eighths of the partial are read, one group of rows is parked in shared memory to make
+                    // room for the last eighth, and the dP columns are released before any reduction of this
+                    // pair is issued.
+                    uint32_t r0a[16], r0b[16], r1[32], r2[32], r3[16];
+                    tmem_ld16(taddr, r0a);
+                    tmem_ld16(taddr + 16, r0b);
                     tmem_ld32(taddr + 32, r1);
                     tmem_ld32(taddr + 64, r2);
+                    tmem_ld16(taddr + 96, r3);
                     tmem_wait_ld();
-                    store_rows(0, r0);
-                    store_rows(1, r0 + 16);
-                    tmem_ld32(taddr + 96, r0);
+                    store_rows(0, r0a);
+                    tmem_ld16(taddr + 112, r0a);
                     tmem_wait_ld();
                     tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&sm.bar_dq_empty);
+                    LT_TL(tid == kReduceWarp0 * 32, 12, it);
                     LT_TRACE_SINCE(12, tr0);
                     fence_proxy_async_smem();
+                    // the buffer where group 1 goes was read by the last reduction but one of the previous pair
+                    if (elected) bulk_wait_group_read<1>();
                     named_barrier_sync(kBarReduceWarps, kNumReduceWarps * 32);
-                    if (elected) {
-                        add_rows(0);
-                        add_rows(1);
-                    }
-                    // groups 2..7 rotate through the three buffers: before group k is issued, the bulk
+                    if (elected) add_rows(0);
+                    // groups 1..7 rotate through the three buffers: before group k is issued, the bulk
                     // reduction of group k-2 has finished reading, which frees the buffer of group k+1
                     auto stage_rows = [&](int k, const uint32_t *r) {
                         store_rows(k, r);
@@ -1004,13 +1032,14 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         named_barrier_sync(kBarReduceWarps, kNumReduceWarps * 32);
                         if (elected) add_rows(k);
                     };
+                    stage_rows(1, r0b);
                     stage_rows(2, r1);
                     stage_rows(3, r1 + 16);
                     stage_rows(4, r2);
                     stage_rows(5, r2 + 16);
-                    stage_rows(6, r0);
-                    stage_rows(7, r0 + 16);
-                    if (elected) bulk_wait_group_read<0>();
+                    stage_rows(6, r3);
+                    stage_rows(7, r0a);
+                    gq += 8;
                 } else {
                     // D = 64: dQ partial with lanes = query rows.  A thread holds the 64 floats of one query row.
                     // The partial is scaled and staged in shared memory as two boxes of 128 rows x 32 floats with
@@ -1048,6 +1077,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         bulk_commit_group();
                     }
                 }
+                LT_TL(tid == kReduceWarp0 * 32, 13, it);
                 LT_TRACE_SINCE(13, tr0);
             }
             if (!ok) break;
@@ -1131,6 +1161,11 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #endif
 }
 
+#ifdef LT_BWD_TIMELINE
+extern "C" int lt_dbg_bwd_timeline(long long *out) {
+    return cudaMemcpyFromSymbol(out, lt::g_bwd_timeline, sizeof(lt::g_bwd_timeline)) == cudaSuccess ? LT_OK : LT_ERR_CUDA;
+}
+#endif
 #ifdef LT_BWD_TRACE
 extern "C" int lt_dbg_bwd_trace(unsigned long long *out, int reset) {
     if (out && cudaMemcpyFromSymbol(out, g_bwd_trace, sizeof(g_bwd_trace)) != cudaSuccess) return LT_ERR_CUDA;
