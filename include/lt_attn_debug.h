@@ -44,6 +44,13 @@ int lt_dbg_tile_gemm(const lt_half *A, const lt_half *B, float *C, int mode,
  * every wait inside the attention kernels takes. */
 int lt_dbg_wait_timeout(void *workspace, size_t workspace_bytes, lt_stream_t stream);
 
+/* Development builds only (not exported by the product library, hence described, not declared):
+ *   -DLT_BWD_TIMELINE=<cta>: `int lt_dbg_bwd_timeline(long long *out)` copies 20 x 256 clock stamps to the
+ *     host buffer `out` ([event][tile pair] of that CTA's first 256 tile pairs in the last backward call;
+ *     paper_2606_10415_b200/timeline.py names the events and prints them); out == NULL clears the stamps.
+ *   -DLT_BWD_TRACE: `int lt_dbg_bwd_trace(unsigned long long *out, int reset)` copies 80 per-role cycle
+ *     totals (slot = 16 * role + wait code - 200; 64.. = per-CTA totals) summed over all CTAs. */
+
 #ifdef __cplusplus
 }
 #endif

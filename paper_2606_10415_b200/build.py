@@ -68,40 +68,71 @@ def build(force: bool = False, verbose: bool = False) -> Path:
     return LIB
 
 
-# Test build of the backward alone in which the tensor-core issuer drops one hand-off and every device-side
-# wait gives up after about 10 ms instead of a second: the main kernel then has to leave through its give-up
-# path (abort flag, every role out of its loops, tensor memory released), which tests/test_gpu_giveup.py checks.
+# Variant builds of the backward alone (libraries of their own that the binding never loads; whoever needs one loads
+# it by path).
+#  - give-up: the tensor-core issuer drops one hand-off and every device-side wait gives up after about 10 ms instead
+#    of a second: the main kernel then has to leave through its give-up path (abort flag, every role out of its
+#    loops, tensor memory released), which tests/test_gpu_giveup.py checks.
+#  - timeline: CTA 0 stamps clock64 at every hand-off of its first 256 tile pairs; paper_2606_10415_b200/timeline.py
+#    prints the table (a development aid behind the bottleneck analysis of the main kernel).
 GIVEUP_LIB = PKG / "liblt_attn_giveup.so"
 GIVEUP_FLAGS = ["-DLT_BWD_GIVEUP_TEST=1", "-DLT_WAIT_LIMIT_CYCLES=20000000LL"]
-GIVEUP_SOURCES = ["lt_attn_bwd.cu", "lt_host.cu"]
+TIMELINE_LIB = PKG / "liblt_attn_timeline.so"
+TIMELINE_FLAGS = ["-DLT_BWD_TIMELINE=0"]
+VARIANT_SOURCES = ["lt_attn_bwd.cu", "lt_host.cu"]
+MICROBENCH = OBJ / "sm_limits"
 
 
-def build_giveup_variant(force: bool = False) -> Path:
-    """Builds ``liblt_attn_giveup.so`` (never loaded by the binding; the give-up test loads it by path)."""
-    obj_dir = PKG / "build_giveup"
+def _build_variant(lib: Path, flags: list[str], tag: str, force: bool) -> Path:
+    obj_dir = PKG / f"build_{tag}"
     obj_dir.mkdir(exist_ok=True)
     headers = sorted(CSRC.glob("*.cuh")) + sorted(CSRC.glob("*.h")) + sorted((PKG.parent / "include").glob("*.h"))
     newest = max(h.stat().st_mtime for h in headers)
     objs = []
-    for name in GIVEUP_SOURCES:
+    for name in VARIANT_SOURCES:
         src, obj = CSRC / name, obj_dir / (Path(name).stem + ".o")
         objs.append(obj)
         if force or not obj.exists() or obj.stat().st_mtime < max(src.stat().st_mtime, newest):
-            res = subprocess.run([_nvcc(), *NVCC_FLAGS, *GIVEUP_FLAGS, "-c", str(src), "-o", str(obj)],
+            res = subprocess.run([_nvcc(), *NVCC_FLAGS, *flags, "-c", str(src), "-o", str(obj)],
                                  capture_output=True, text=True)
             if res.returncode != 0:
-                raise RuntimeError(f"nvcc failed for {name} (give-up variant):\n{res.stdout}\n{res.stderr}")
-    if force or not GIVEUP_LIB.exists() or GIVEUP_LIB.stat().st_mtime < max(o.stat().st_mtime for o in objs):
-        tmp = GIVEUP_LIB.with_suffix(f".so.tmp{os.getpid()}")
+                raise RuntimeError(f"nvcc failed for {name} ({tag} variant):\n{res.stdout}\n{res.stderr}")
+    if force or not lib.exists() or lib.stat().st_mtime < max(o.stat().st_mtime for o in objs):
+        tmp = lib.with_suffix(f".so.tmp{os.getpid()}")
         res = subprocess.run([_nvcc(), "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", str(tmp),
                               *map(str, objs)], capture_output=True, text=True)
         if res.returncode != 0:
-            raise RuntimeError(f"link failed (give-up variant):\n{res.stdout}\n{res.stderr}")
-        os.replace(tmp, GIVEUP_LIB)
-    return GIVEUP_LIB
+            raise RuntimeError(f"link failed ({tag} variant):\n{res.stdout}\n{res.stderr}")
+        os.replace(tmp, lib)
+    return lib
+
+
+def build_giveup_variant(force: bool = False) -> Path:
+    """Builds ``liblt_attn_giveup.so`` (the give-up test loads it by path)."""
+    return _build_variant(GIVEUP_LIB, GIVEUP_FLAGS, "giveup", force)
+
+
+def build_timeline_variant(force: bool = False) -> Path:
+    """Builds ``liblt_attn_timeline.so`` (``python -m paper_2606_10415_b200.timeline`` loads it by path)."""
+    return _build_variant(TIMELINE_LIB, TIMELINE_FLAGS, "timeline", force)
+
+
+def build_microbench() -> Path:
+    """Builds the stand-alone microbenchmark ``build/sm_limits`` from ``csrc/microbench/sm_limits.cu``."""
+    OBJ.mkdir(exist_ok=True)
+    src = CSRC / "microbench" / "sm_limits.cu"
+    res = subprocess.run([_nvcc(), *[f for f in NVCC_FLAGS if f not in ("-Xptxas", "-v")], str(src), "-o", str(MICROBENCH)],
+                         capture_output=True, text=True)
+    if res.returncode != 0:
+        raise RuntimeError(f"nvcc failed for {src.name}:\n{res.stdout}\n{res.stderr}")
+    return MICROBENCH
 
 
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
     if "--giveup" in sys.argv:
         print(build_giveup_variant(force="--force" in sys.argv))
+    if "--timeline" in sys.argv:
+        print(build_timeline_variant(force="--force" in sys.argv))
+    if "--microbench" in sys.argv:
+        print(build_microbench())

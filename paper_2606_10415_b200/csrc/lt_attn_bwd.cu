@@ -319,7 +319,7 @@ __device__ __forceinline__ bool traced_wait(Trace &tr, uint64_t *bar, uint32_t p
 
 // Built only with -DLT_BWD_TIMELINE=<cta> (development aid): clock stamps of that CTA's first 256 iterations.
 #ifdef LT_BWD_TIMELINE
-__device__ long long g_bwd_timeline[16 * 256];
+__device__ long long g_bwd_timeline[20 * 256];  // [event][iteration]; events are listed in paper_2606_10415_b200/timeline.py
 #define LT_TL(cond, ev, iter)                                                                        \
     do {                                                                                             \
         if ((cond) && blockIdx.x == LT_BWD_TIMELINE && (iter) < 256) g_bwd_timeline[(ev) * 256 + (iter)] = clock64(); \
@@ -706,6 +706,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                          LT_WAIT_ALL(&sm.bar_q_full[it & 1], (it >> 1) & 1, kWaitStageFull);
                     if (!ok) break;
                     tc_fence_after_sync();
+                    LT_TL(leader, 14, it);
                     if constexpr (!kSavedP) issue_s(it);
                     for (int n = 0; n < w.n_iter && ok; ++n, ++it) {
                         const int s = it & 1;
@@ -1107,6 +1108,7 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                             tc_fence_before_sync();
                             __syncwarp();
                             if (lane == 0) mbar_arrive(&sm.bar_acc_free);
+                            LT_TL(tid == kReduceWarp0 * 32, 15, it);
                         }
                         if constexpr (kSplit) {
                             // the group's heads are spread over several items: add this item's share to
@@ -1162,7 +1164,12 @@ bwd_main_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 }
 
 #ifdef LT_BWD_TIMELINE
-extern "C" int lt_dbg_bwd_timeline(long long *out) {
+extern "C" int lt_dbg_bwd_timeline(long long *out) {  // out == NULL: clear the stamps
+    if (!out) {
+        void *sym = nullptr;
+        if (cudaGetSymbolAddress(&sym, lt::g_bwd_timeline) != cudaSuccess) return LT_ERR_CUDA;
+        return cudaMemset(sym, 0, sizeof(lt::g_bwd_timeline)) == cudaSuccess ? LT_OK : LT_ERR_CUDA;
+    }
     return cudaMemcpyFromSymbol(out, lt::g_bwd_timeline, sizeof(lt::g_bwd_timeline)) == cudaSuccess ? LT_OK : LT_ERR_CUDA;
 }
 #endif
