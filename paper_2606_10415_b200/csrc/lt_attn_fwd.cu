@@ -605,9 +605,22 @@ int lt_attn_fwd_bwd_host(const lt_half *Q, const lt_half *K, const lt_half *V, c
     const int n_units = B * Hkv;
     const long long n_tiles = padded_rows(S) / 128;
     const long long unit_iters = static_cast<long long>(G) * (causal ? n_tiles * (n_tiles + 1) / 2 : n_tiles * n_tiles);
-    long long want = unit_iters * n_units / 3000;  // a chunk should still fill the GPU
-    int n_chunks = static_cast<int>(want < 1 ? 1 : (want > kHostMaxChunks ? kHostMaxChunks : want));
-    if (n_chunks > n_units) n_chunks = n_units;
+    // Few, large chunks (a copy of a few MB carries tens of microseconds of fixed cost, and a chunk's kernels take
+    // 0.2 ms however small it is); the last chunk is the smallest, because its kernels and its copy back are what is
+    // left to do when the input copy ends.
+    int bounds[kHostMaxChunks + 1];
+    int n_chunks = 1;
+    bounds[0] = 0;
+    bounds[1] = n_units;
+    if (unit_iters * n_units >= 3000 && n_units > 1) {  // otherwise not worth the extra streams
+        const int percent[4] = {30, 60, 85, 100};  // cumulative shares of the four chunks
+        n_chunks = 0;
+        for (int c = 0; c < 4; ++c) {
+            int end = c == 3 ? n_units : (n_units * percent[c] + 50) / 100;
+            if (end <= bounds[n_chunks]) continue;  // fewer units than chunks
+            bounds[++n_chunks] = end;
+        }
+    }
 
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -639,8 +652,7 @@ int lt_attn_fwd_bwd_host(const lt_half *Q, const lt_half *K, const lt_half *V, c
         LT_CUDA(cudaStreamWaitEvent(s_out, pipe->ev_start, 0), "cudaStreamWaitEvent");
     }
     for (int c = 0; c < n_chunks; ++c) {
-        const int u0 = static_cast<int>(static_cast<long long>(n_units) * c / n_chunks);
-        const int u1 = static_cast<int>(static_cast<long long>(n_units) * (c + 1) / n_chunks);
+        const int u0 = bounds[c], u1 = bounds[c + 1];
         const int hkv = u1 - u0, hq = hkv * G;
         const size_t oq = static_cast<size_t>(u0) * G * S * D, ok_ = static_cast<size_t>(u0) * S * D;  // elements
         const size_t ol = static_cast<size_t>(u0) * G * S;
