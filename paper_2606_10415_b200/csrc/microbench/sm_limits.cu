@@ -7,6 +7,8 @@
 //   sm_limits reduce [grid]            bytes per clock and SM of fp32 add-reductions into L2 (bulk and red.v4),
 //                                      of plain stores and of bulk stores
 //   sm_limits loadlat [grid]           latency of a 32 KB bulk load behind 0-32 KB of queued bulk reductions
+//   sm_limits dsmem [grid]             bytes per clock and SM of stores into the partner CTA's shared memory
+//                                      (clusters of two), alone and beside bulk reductions into L2
 //
 // Build: python -m paper_2606_10415_b200.build --microbench   (-> paper_2606_10415_b200/build/sm_limits)
 // Every wait is bounded; operands are whatever the fill leaves in memory (timing does not depend on them).
@@ -312,6 +314,69 @@ __global__ void __launch_bounds__(128, 1) loadlat_kernel(float *g, const uint8_t
     __syncthreads();
 }
 
+// ------------------------------------------------------------------------------------------- dsmem
+// Clusters of two CTAs: warps 0-3 of each CTA store into the partner's shared memory (16 bytes per lane, 512
+// contiguous bytes per warp instruction; `with_reduce`: thread 128 issues 8 KB bulk reductions into L2 beside
+// them, two in flight).  out[2*cta] = cycles, out[2*cta+1] = reduction bytes of that CTA.
+__global__ void __launch_bounds__(160, 1) dsmem_kernel(float *g, int reps, int with_store, int with_reduce, long long *out) {
+    extern __shared__ __align__(1024) uint8_t raw[];
+    __shared__ int stop_flag;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    for (int i = tid; i < 96 * 1024 / 4; i += blockDim.x) reinterpret_cast<float *>(raw)[i] = 1.0f;
+    if (tid == 0) stop_flag = 0;
+    fence_proxy_async_smem();
+    __syncthreads();
+    cluster_sync_all();
+    volatile int *stop = &stop_flag;
+    const uint32_t partner = cluster_cta_rank() ^ 1u;
+    float *dst = g + (static_cast<size_t>(blockIdx.x) << 18);
+    const long long t0 = clock64();
+    if (warp < 4) {
+        if (with_store) {
+            // 32 KB window of the partner, walked round and round
+            const uint32_t remote = cluster_map_shared(smem_u32(raw + 32768), partner);
+            for (int r = 0; r < reps; ++r) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const uint32_t a = remote + ((r * 4 + u) % 16) * 2048 + warp * 512 + lane * 16;
+                    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(a), "f"(1.f), "f"(2.f), "f"(3.f), "f"(4.f)
+                                 : "memory");
+                }
+            }
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (tid == 0) {
+            out[2 * blockIdx.x] = clock64() - t0;
+            *stop = 1;
+        }
+    } else if (with_reduce && lane == 0) {
+        unsigned long long bytes = 0;
+        uint32_t n = 0;
+        if (!with_store) {
+            for (int r = 0; r < reps / 4; ++r) {  // fixed amount of work when nothing else sets the pace
+                bulk_reduce_add_f32(dst + static_cast<size_t>(n & 15) * 2048, raw + (n & 3) * 8192, 8192);
+                bulk_commit_group();
+                bulk_wait_group_read<1>();
+                ++n;
+                bytes += 8192;
+            }
+        } else {
+            while (!*stop) {
+                bulk_reduce_add_f32(dst + static_cast<size_t>(n & 15) * 2048, raw + (n & 3) * 8192, 8192);
+                bulk_commit_group();
+                bulk_wait_group_read<1>();
+                ++n;
+                bytes += 8192;
+            }
+        }
+        bulk_wait_group_all();
+        out[2 * blockIdx.x + 1] = static_cast<long long>(bytes);
+        if (!with_store) out[2 * blockIdx.x] = clock64() - t0;
+    }
+    __syncthreads();
+    cluster_sync_all();  // the partner may still be storing into this CTA's shared memory
+}
+
 bool check(const char *what) {
     const cudaError_t e = cudaDeviceSynchronize();
     if (e != cudaSuccess) std::printf("%s: %s\n", what, cudaGetErrorString(e));
@@ -389,8 +454,44 @@ int main(int argc, char **argv) {
                 std::printf("grid %3d, red.v4 from registers beside it      : 32 KB load latency avg %6lld, worst %6lld cycles\n", grid,
                             avg / grid, worst);
         }
+    } else if (!std::strcmp(mode, "dsmem")) {
+        const int grid = argc > 2 ? std::atoi(argv[2]) : 2, reps = 2000;
+        if (grid < 2 || grid > 148 || (grid & 1)) return 2;
+        float *g;
+        cudaMalloc(&g, static_cast<size_t>(148) << 20);
+        cudaMemset(g, 0, static_cast<size_t>(148) << 20);
+        cudaFuncSetAttribute(dsmem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(grid);
+        cfg.blockDim = dim3(160);
+        cfg.dynamicSmemBytes = 96 * 1024;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = 2;
+        attr.val.clusterDim.y = 1;
+        attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        const int modes[3][2] = {{1, 0}, {0, 1}, {1, 1}};
+        for (auto &m : modes) {
+            cudaMemset(out, 0, 148 * 2 * sizeof(long long));
+            for (int rep = 0; rep < 2; ++rep)
+                if (cudaLaunchKernelEx(&cfg, dsmem_kernel, g, reps, m[0], m[1], out) != cudaSuccess) {
+                    std::printf("cluster launch failed: %s\n", cudaGetErrorString(cudaGetLastError()));
+                    return 1;
+                }
+            if (!check("dsmem")) return 1;
+            long long h[296], worst = 0, red = 0;
+            cudaMemcpy(h, out, grid * 2 * sizeof(long long), cudaMemcpyDeviceToHost);
+            for (int i = 0; i < grid; ++i) {
+                worst = h[2 * i] > worst ? h[2 * i] : worst;
+                red += h[2 * i + 1];
+            }
+            std::printf("grid %3d (clusters of 2): remote shared-memory stores %6.2f B/clock/SM, bulk reductions into L2 %6.2f B/clock/SM\n", grid,
+                        m[0] ? 2048.0 * 4 * reps / worst : 0.0, static_cast<double>(red) / grid / worst);
+        }
     } else {
-        std::printf("usage: sm_limits products [reps] [grid] | reduce [grid] | loadlat [grid]\n");
+        std::printf("usage: sm_limits products [reps] [grid] | reduce [grid] | loadlat [grid] | dsmem [grid]\n");
         return 2;
     }
     return 0;
