@@ -212,6 +212,28 @@ def max_over_ranks(values, dist, device):
     return t.tolist()
 
 
+# fp32 add-reductions into L2 with every SM reducing: bytes per clock and SM, measured with
+# paper_2606_10415_b200/csrc/microbench/sm_limits.cu (`sm_limits reduce 148`; 25.4 for one SM alone)
+REDUCTION_BYTES_PER_CLOCK_PER_SM = 20.7
+N_SMS = 148
+
+
+def reduction_path(cfg, main_ms, clocks):
+    """Bytes of dQ partial the main kernel adds into L2 per launch against the measured rate of that path."""
+    n = -(-cfg.S // 128)
+    pairs = cfg.B * cfg.Hq * (n * (n + 1) // 2 if cfg.causal else n * n)
+    nbytes = pairs * 128 * cfg.D * 4
+    sm_hz = 1e6 * float(clocks.get("sm_mhz") or clocks.get("sm_max_mhz") or 0.0)
+    achieved = nbytes / (main_ms * 1e-3) / 1e9
+    out = {"bytes_per_launch": nbytes, "achieved": achieved, "unit": "GB/s",
+           "how": "executed tile pairs x 128 x D x 4 bytes / average main-kernel launch"}
+    if sm_hz > 0:
+        limit = REDUCTION_BYTES_PER_CLOCK_PER_SM * N_SMS * sm_hz / 1e9
+        out.update({"peak": limit, "frac": achieved / limit,
+                    "peak_source": "20.7 B/clock/SM (sm_limits microbenchmark) x 148 SMs x the median SM clock sampled under load"})
+    return out
+
+
 def job_throughput(flops_per_rank, world, seconds_per_step):
     """Whole-job metric for replicas: every rank processes its own copy of the workload."""
     return world * flops_per_rank / seconds_per_step / 1e12
@@ -500,6 +522,9 @@ def run_ours(args, cfg):
                                                   "place the kernels do not overlap, so the three add up to a "
                                                   "little more than ms_per_step"},
                          "best_launch_ms": min(main_ms),
+                         # what the kernel is closest to: the SMs' write path into L2, which carries one fp32 dQ
+                         # partial per executed (query tile, key tile) pair
+                         "l2_reduction_path": reduction_path(cfg, main_avg_ms, clocks),
                          "burst_peak": peak, "frac_of_burst_peak": achieved / peak,
                          "timed_alone": {"best_launch_ms": iso_best_ms, "achieved": iso_achieved, "peak": peak,
                                          "frac": iso_achieved / peak,

@@ -56,3 +56,20 @@ def test_reference_arm_prints_one_json_line_on_cpu():
     res = subprocess.run([sys.executable, str(ROOT / "bench.py"), "--impl", "reference", "--config", "tiny",
                           "--steps", "1", "--warmup", "0"], capture_output=True, text=True, env=env, check=True)
     assert res.stdout.strip() == ""
+
+
+def test_reduction_path_bytes_match_the_profiled_launch():
+    """The bytes of dQ partial bench.py charges to the L2 reduction path are the ones ncu counted for the
+    profiled launch (profiles/bwd_main_kernel_llama2_7b.md: 1.107 GB), and ragged / unmasked shapes follow
+    the executed tile pairs."""
+    sys.path.insert(0, str(ROOT))
+    import bench
+    from paper_2606_10415_b200 import workloads
+    r = bench.reduction_path(workloads.ALL_CONFIGS["llama2_7b"], 0.4, {"sm_mhz": 1600.0})
+    assert r["bytes_per_launch"] == 32 * 528 * 128 * 128 * 4 == 1107296256
+    assert abs(r["achieved"] - 1107296256 / 0.4e-3 / 1e9) < 1e-6
+    assert abs(r["peak"] - 20.7 * 148 * 1.6) < 1e-6 and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-12
+    full = bench.reduction_path(workloads.ALL_CONFIGS["llama2_7b_full_mask_off"], 0.7, {})
+    assert full["bytes_per_launch"] == 32 * 32 * 32 * 128 * 128 * 4 and "frac" not in full
+    ragged = bench.reduction_path(workloads.ALL_CONFIGS["llama2_7b_s3000_ragged"], 0.2, {"sm_mhz": 1600.0})
+    assert ragged["bytes_per_launch"] == 32 * (24 * 25 // 2) * 128 * 128 * 4
