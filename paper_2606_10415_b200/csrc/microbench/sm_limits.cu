@@ -7,6 +7,7 @@
 //   sm_limits reduce [grid]            bytes per clock and SM of fp32 add-reductions into L2 (bulk and red.v4),
 //                                      of plain stores and of bulk stores
 //   sm_limits loadlat [grid]           latency of a 32 KB bulk load behind 0-32 KB of queued bulk reductions
+//   sm_limits mixed [grid]             bulk reductions with 32 KB bulk loads running beside them (the kernel's mix)
 //   sm_limits dsmem [grid]             bytes per clock and SM of stores into the partner CTA's shared memory
 //                                      (clusters of two), alone and beside bulk reductions into L2
 //
@@ -377,6 +378,50 @@ __global__ void __launch_bounds__(160, 1) dsmem_kernel(float *g, int reps, int w
     cluster_sync_all();  // the partner may still be storing into this CTA's shared memory
 }
 
+// ------------------------------------------------------------------------------------------- mixed
+// The main kernel's own mix: thread 0 loads 32 KB tiles back to back (one at a time, as many bytes as are reduced)
+// while thread 32 keeps two 8 KB bulk reductions in flight.  out[2*cta] = cycles, out[2*cta+1] = bytes loaded.
+__global__ void __launch_bounds__(128, 1) mixed_kernel(float *g, const uint8_t *src, int reps, int with_loads, long long *out) {
+    extern __shared__ __align__(1024) uint8_t raw[];
+    __shared__ uint64_t bar;
+    __shared__ int stop_flag;
+    const int tid = threadIdx.x;
+    for (int i = tid; i < 64 * 1024 / 4; i += blockDim.x) reinterpret_cast<float *>(raw)[i] = 1.0f;
+    if (tid == 0) {
+        mbar_init(&bar, 1);
+        mbar_fence_init();
+        stop_flag = 0;
+    }
+    fence_proxy_async_smem();
+    __syncthreads();
+    volatile int *stop = &stop_flag;
+    float *dst = g + (static_cast<size_t>(blockIdx.x) << 18);
+    if (tid == 32) {
+        const long long t0 = clock64();
+        for (int n = 0; n < reps; ++n) {
+            bulk_reduce_add_f32(dst + static_cast<size_t>(n % 16) * 2048, raw + (n % 4) * 8192, 8192);
+            bulk_commit_group();
+            bulk_wait_group_read<1>();
+        }
+        bulk_wait_group_all();
+        out[2 * blockIdx.x] = clock64() - t0;
+        *stop = 1;
+    } else if (tid == 0 && with_loads) {
+        long long bytes = 0;
+        uint32_t phase = 0;
+        while (!*stop) {
+            mbar_arrive_expect_tx(&bar, 32768);
+            bulk_load_1d(raw + 65536, src + (static_cast<size_t>(blockIdx.x) * 64 + (bytes >> 15) % 64) * 32768, 32768, &bar);
+            uint32_t spins = 0;
+            while (!mbar_try_wait(&bar, phase) && ++spins < (1u << 26)) {}
+            phase ^= 1;
+            bytes += 32768;
+        }
+        out[2 * blockIdx.x + 1] = bytes;
+    }
+    __syncthreads();
+}
+
 bool check(const char *what) {
     const cudaError_t e = cudaDeviceSynchronize();
     if (e != cudaSuccess) std::printf("%s: %s\n", what, cudaGetErrorString(e));
@@ -454,6 +499,29 @@ int main(int argc, char **argv) {
                 std::printf("grid %3d, red.v4 from registers beside it      : 32 KB load latency avg %6lld, worst %6lld cycles\n", grid,
                             avg / grid, worst);
         }
+    } else if (!std::strcmp(mode, "mixed")) {
+        const int grid = argc > 2 ? std::atoi(argv[2]) : 1, reps = 2000;
+        if (grid < 1 || grid > 148) return 2;
+        float *g;
+        uint8_t *src;
+        cudaMalloc(&g, static_cast<size_t>(148) << 20);
+        cudaMemset(g, 0, static_cast<size_t>(148) << 20);
+        cudaMalloc(&src, static_cast<size_t>(148) * 64 * 32768);
+        cudaMemset(src, 0, static_cast<size_t>(148) * 64 * 32768);
+        cudaFuncSetAttribute(mixed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+        for (int with_loads = 0; with_loads <= 1; ++with_loads) {
+            cudaMemset(out, 0, 148 * 2 * sizeof(long long));
+            for (int rep = 0; rep < 2; ++rep) mixed_kernel<<<grid, 128, 100 * 1024>>>(g, src, reps, with_loads, out);
+            if (!check("mixed")) return 1;
+            long long h[296], worst = 0, loaded = 0;
+            cudaMemcpy(h, out, grid * 2 * sizeof(long long), cudaMemcpyDeviceToHost);
+            for (int i = 0; i < grid; ++i) {
+                worst = h[2 * i] > worst ? h[2 * i] : worst;
+                loaded += h[2 * i + 1];
+            }
+            std::printf("grid %3d: bulk reductions %6.2f B/clock/SM with bulk loads of %6.2f B/clock/SM beside them\n", grid,
+                        8192.0 * reps / worst, static_cast<double>(loaded) / grid / worst);
+        }
     } else if (!std::strcmp(mode, "dsmem")) {
         const int grid = argc > 2 ? std::atoi(argv[2]) : 2, reps = 2000;
         if (grid < 2 || grid > 148 || (grid & 1)) return 2;
@@ -491,7 +559,7 @@ int main(int argc, char **argv) {
                         m[0] ? 2048.0 * 4 * reps / worst : 0.0, static_cast<double>(red) / grid / worst);
         }
     } else {
-        std::printf("usage: sm_limits products [reps] [grid] | reduce [grid] | loadlat [grid] | dsmem [grid]\n");
+        std::printf("usage: sm_limits products [reps] [grid] | reduce [grid] | loadlat [grid] | dsmem [grid] | mixed [grid]\n");
         return 2;
     }
     return 0;
