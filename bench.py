@@ -37,7 +37,7 @@ NOMINAL_FP16_TFLOPS = 2250.0  # datasheet dense figure, context only
 # dram__bytes_read.sum + dram__bytes_write.sum of one bwd_main_kernel launch, per workload, from an ncu capture of
 # that workload's own launch (one kernel, one launch); workloads without a capture report no traffic figure
 MAIN_KERNEL_DRAM_BYTES = {"llama2_7b": 291.4e6, "baichuan2_13b": 377.6e6, "qwen25_32b_gqa": 442.3e6,
-                          "llama2_70b_gqa": 3602.8e6}
+                          "llama2_70b_gqa": 1451.8e6}
 # (rows, weight rows, weight columns): the paper's GEMM profile shapes at sequence length 2048
 GEMM_SHAPES = [(2048, 4096, 4096), (2048, 11008, 4096), (2048, 4096, 11008), (2048, 6656, 6656), (2048, 8192, 8192)]
 FALLBACK_PEAK_TFLOPS = 1590.0

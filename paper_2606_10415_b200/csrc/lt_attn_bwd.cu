@@ -1197,7 +1197,7 @@ static int sm_count() {
         return 148;
     return sms;
 }
-static int heads_per_item(int B, int Hq, int Hkv, int S, int causal) {
+static int heads_per_item(int B, int Hq, int Hkv, int S, int D, int causal) {
     const int sms = sm_count();
     const long long split_below_items = sms + sms / 2;  // split when there are fewer than 1.5 whole-group items per SM
     const long long split_target_items = 2 * sms;       // and then aim at two items per SM (every item pays a pipeline fill)
@@ -1206,10 +1206,21 @@ static int heads_per_item(int B, int Hq, int Hkv, int S, int causal) {
     const long long n_tiles = padded_rows(S) / kTileRows;
     const long long n_base = static_cast<long long>(B) * Hkv * n_tiles;
     const long long iters = static_cast<long long>(B) * Hq * (causal ? n_tiles * (n_tiles + 1) / 2 : n_tiles * n_tiles);
-    if (G == 1 || n_base >= split_below_items || iters < split_min_iterations) return G;
-    const long long split = (split_target_items + n_base - 1) / n_base;
-    const int hs = static_cast<int>(split < G ? split : G);
-    return (G + hs - 1) / hs;
+    if (G == 1 || iters < split_min_iterations) return G;
+    if (n_base < split_below_items) {
+        const long long split = (split_target_items + n_base - 1) / n_base;
+        const int hs = static_cast<int>(split < G ? split : G);
+        return (G + hs - 1) / hs;
+    }
+    // Enough whole-group items to fill the SMs, but too few to form L2-sized batches (a batch needs two items per
+    // SM) while the working set is several times the L2: the accumulator rows of the heads in flight would be
+    // fetched and written back again and again.  Two items per key tile make room for batches (measured: LLaMA-2-70B
+    // layer, B = 2: 3.6 GB of DRAM traffic and 1.78 ms per call whole, 1.69 ms split; +12 % at S = 8192; the
+    // Qwen2.5-32B layer, whose working set is 1.4 L2s, is slower split).
+    const double unit_bytes = static_cast<double>(padded_rows(S)) * D * (2.0 * 2 + G * (2.0 * 2 + 4));
+    const double working_set = unit_bytes * B * Hkv;
+    if (n_base < 4LL * sms && working_set > 2.0 * 126.0e6 && G >= 2) return (G + 1) / 2;
+    return G;
 }
 
 template <int D, bool kBf16>
@@ -1233,7 +1244,7 @@ static int launch_bwd(const lt_half *Q, const lt_half *K, const lt_half *V, cons
     uint4 *delta_ext = reinterpret_cast<uint4 *>(ws + kStatusBytes);
     uint4 *lse_ext = reinterpret_cast<uint4 *>(ws + kStatusBytes + ext_bytes);
     float *dq_acc = reinterpret_cast<float *>(ws + kStatusBytes + 2 * ext_bytes);
-    const int hpi = saved_p ? Hq / Hkv : heads_per_item(B, Hq, Hkv, S, causal);
+    const int hpi = saved_p ? Hq / Hkv : heads_per_item(B, Hq, Hkv, S, D, causal);
     const int parts = (Hq / Hkv + hpi - 1) / hpi;
     const size_t kv_floats = static_cast<size_t>(B) * Hkv * S_pad * D;
     float *dk_acc = nullptr, *dv_acc = nullptr;
@@ -1368,7 +1379,7 @@ size_t lt_attn_bwd_workspace_bytes(int B, int Hq, int Hkv, int S, int D) {
     size_t bytes = lt::kStatusBytes + 2 * lt::round256(n_rows * 16) + lt::round256(n_rows * D * 4);
     // fp32 dK / dV sums for shapes whose groups are split over work items (either mask; sized for the
     // unmasked case, which splits no less often)
-    if (lt::heads_per_item(B, Hq, Hkv, S, 1) < Hq / Hkv || lt::heads_per_item(B, Hq, Hkv, S, 0) < Hq / Hkv)
+    if (lt::heads_per_item(B, Hq, Hkv, S, D, 1) < Hq / Hkv || lt::heads_per_item(B, Hq, Hkv, S, D, 0) < Hq / Hkv)
         bytes += 2 * lt::round256(static_cast<size_t>(B) * Hkv * static_cast<size_t>(lt::padded_rows(S)) * D * 4);
     return bytes;
 }
@@ -1376,7 +1387,7 @@ size_t lt_attn_bwd_workspace_bytes(int B, int Hq, int Hkv, int S, int D) {
 int lt_attn_bwd_num_launches(int B, int Hq, int Hkv, int S, int D, int causal) {
     if (lt::check_shape(B, Hq, Hkv, S, D, 1.0f) != LT_OK) return 0;
     // preprocess, main, dQ conversion; plus the dK/dV conversion when groups are split over work items
-    return lt::heads_per_item(B, Hq, Hkv, S, causal) < Hq / Hkv ? 4 : 3;
+    return lt::heads_per_item(B, Hq, Hkv, S, D, causal) < Hq / Hkv ? 4 : 3;
 }
 
 static int bwd_entry(const lt_half *Q, const lt_half *K, const lt_half *V, const lt_half *O, const lt_half *dO,

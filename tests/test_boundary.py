@@ -60,6 +60,9 @@ def test_launch_counts(binding):
     assert binding.lt_attn_bwd_num_launches(1, 32, 32, 4096, 128, True) == 3
     assert binding.lt_attn_bwd_num_launches(1, 40, 8, 4096, 128, True) == 3
     assert binding.lt_attn_bwd_num_launches(1, 40, 8, 2048, 128, True) == 4
+    # groups are also split when whole-group items are too few for L2-sized batches on a working set of several L2s
+    assert binding.lt_attn_bwd_num_launches(2, 64, 8, 4096, 128, True) == 4
+    assert binding.lt_attn_bwd_num_launches(4, 64, 8, 4096, 128, True) == 3
     assert binding.lt_attn_bwd_num_launches(1, 2, 2, 128, 96, True) == 0
     assert binding.lt_attn_fwd_num_launches() == 1
 
