@@ -1213,13 +1213,15 @@ static int heads_per_item(int B, int Hq, int Hkv, int S, int D, int causal) {
         return (G + hs - 1) / hs;
     }
     // Enough whole-group items to fill the SMs, but too few to form L2-sized batches (a batch needs two items per
-    // SM) while the working set is several times the L2: the accumulator rows of the heads in flight would be
-    // fetched and written back again and again.  Two items per key tile make room for batches (measured: LLaMA-2-70B
-    // layer, B = 2: 3.6 GB of DRAM traffic and 1.78 ms per call whole, 1.69 ms split; +12 % at S = 8192; the
-    // Qwen2.5-32B layer, whose working set is 1.4 L2s, is slower split).
+    // SM) while the working set is more than four times the L2: the accumulator rows of the heads in flight would be
+    // fetched and written back again and again.  Two items per key tile make room for batches.  Measured, whole
+    // against split, ms per call: LLaMA-2-70B layer with B = 2 1.78 / 1.69 (3.6 -> 1.45 GB of DRAM traffic), the
+    // same at S = 8192 with B = 1 3.38 / 3.02, 32 / 4 heads at S = 16384 6.06 / 5.76.  Smaller working sets lose
+    // more to the second pipeline fill and the fp32 epilogue than they gain: 32 / 8 heads at S = 8192 (2.4 L2s)
+    // 1.52 / 1.59, the same with B = 2 at S = 4096 0.86 / 0.89, the Qwen2.5-32B layer (1.4 L2s) 0.53 / 0.56.
     const double unit_bytes = static_cast<double>(padded_rows(S)) * D * (2.0 * 2 + G * (2.0 * 2 + 4));
     const double working_set = unit_bytes * B * Hkv;
-    if (n_base < 4LL * sms && working_set > 2.0 * 126.0e6 && G >= 2) return (G + 1) / 2;
+    if (n_base < 4LL * sms && working_set > 4.0 * 126.0e6) return (G + 1) / 2;
     return G;
 }
 
